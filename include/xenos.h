@@ -1,0 +1,204 @@
+/*
+ * xenos.h - C ABI of the linked-chain CNN inference library for NVIDIA B200 (sm_100a).
+ *
+ * The calls follow the paper's statement of the problem (Xenos, arXiv 2302.00282): the user
+ * supplies "a computation graph for the inference model, along with the hardware-specific
+ * information" (Section 6) built from the operators of Table 3; the library fuses
+ * Conv+Bn+Bias+Relu (Section 4.3), links adjacent operators so a producer hands its tile to
+ * the consumer in the order the consumer reads it (Section 4.1, Table 1), splits operators
+ * across the parallel units (Section 4.2, Eq. 1), and runs the optimised model, which is
+ * equivalent to the original one (Section 3).
+ *
+ * Conventions
+ *  - Plain C, no exceptions cross the boundary.  Every call returns xenos_status_t
+ *    (0 = XENOS_OK, negative = error); xenos_last_error() gives a message for the last
+ *    failing call on that graph.
+ *  - HOST pointers: every pointer inside xenos_op_desc_t, xenos_hw_info_t, id arrays, the
+ *    JSON buffer.  They are read during the call only; the caller keeps ownership.
+ *  - DEVICE pointers: the workspace given to xenos_graph_bind and the input / output
+ *    arrays given to xenos_graph_run.  The library never allocates or frees device memory;
+ *    the caller (typically PyTorch) owns all of it and owns the stream.
+ *  - There is no CPU fallback: xenos_graph_bind / xenos_graph_run fail with XENOS_E_CUDA
+ *    when no sm_100 device is usable.
+ *  - State machine: create -> add_input / add_op / mark_output -> (link)* -> (split)* ->
+ *    compile -> bind -> run* -> destroy.  A call made in the wrong state returns
+ *    XENOS_E_STATE and changes nothing.
+ */
+#ifndef XENOS_H_
+#define XENOS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define XENOS_API __attribute__((visibility("default")))
+#else
+#define XENOS_API
+#endif
+
+typedef struct xenos_graph xenos_graph_t;   /* opaque; owned by the library */
+typedef int32_t xenos_status_t;
+typedef int32_t xenos_id_t;                 /* tensor id; an operator is named by its output tensor */
+
+enum {
+    XENOS_OK = 0,
+    XENOS_E_INVALID = -1,       /* null pointer, unknown enum value, bad id                     */
+    XENOS_E_SHAPE = -2,         /* operand shapes do not fit the operator                        */
+    XENOS_E_UNSUPPORTED = -3,   /* valid request the library has no kernel for                   */
+    XENOS_E_NOT_LINKABLE = -4,  /* explicit link request that matches no Table 1 pattern         */
+    XENOS_E_BAD_SPLIT = -5,     /* split request that does not divide the operator               */
+    XENOS_E_STATE = -6,         /* call out of order                                             */
+    XENOS_E_WORKSPACE = -7,     /* workspace missing, too small or misaligned                    */
+    XENOS_E_CUDA = -8,          /* CUDA runtime / driver error, or no usable device              */
+    XENOS_E_TIMEOUT = -9,       /* a bounded device-side wait expired (status word set)          */
+    XENOS_E_BOUNDS = -10        /* a device-side index check failed (status word set)            */
+};
+
+/* Operator kinds: the Table 3 operators the CNN workloads use.  x.mul, x.mac, x.transpose,
+ * x.split and general x.matmul are not implemented and yield XENOS_E_UNSUPPORTED. */
+enum {
+    XENOS_OP_CONV = 1,            /* x.conv; groups == 1 dense, groups == Cin == Cout depthwise      */
+    XENOS_OP_FC = 2,              /* x.matmul as y = W x + B (Eq. 1); input is a [C] vector per image */
+    XENOS_OP_POOL_MAX = 3,        /* x.gampool                                                        */
+    XENOS_OP_POOL_AVG = 4,        /* x.gampool, unpadded windows only                                 */
+    XENOS_OP_POOL_GLOBAL_AVG = 5, /* x.gampool; output is a [C] vector per image                      */
+    XENOS_OP_ADD = 6,             /* x.add, two inputs of equal shape                                 */
+    XENOS_OP_CONCAT = 7,          /* x.concat along channels, inputs in argument order               */
+    XENOS_OP_RELU = 8,
+    XENOS_OP_RELU6 = 9,
+    XENOS_OP_BATCHNORM = 10       /* inference form: gamma * (x - mean) / sqrt(var + eps) + beta      */
+};
+
+enum { XENOS_ACT_NONE = 0, XENOS_ACT_RELU = 1, XENOS_ACT_RELU6 = 2 };
+enum { XENOS_DTYPE_F32 = 0, XENOS_DTYPE_BF16 = 1 };
+enum { XENOS_LAYOUT_NCHW = 0, XENOS_LAYOUT_NHWC = 1 };
+
+/* Arithmetic of a compiled graph.
+ *  FP32_CUDA_CORE: fp32 storage and fp32 FMA on CUDA cores, NCHW tensors.
+ *  BF16_TENSOR:    bf16 storage (round to nearest even), fp32 accumulation; dense and
+ *                  pointwise convolutions and FC run as implicit GEMM on tcgen05 tensor
+ *                  cores; tensors between kernels are NHWC bf16. */
+enum { XENOS_PRECISION_FP32_CUDA_CORE = 0, XENOS_PRECISION_BF16_TENSOR = 1 };
+
+/* "Hardware-specific information ... memory hierarchy, number of DSP units" (Section 6),
+ * in this device's terms.  Pass NULL to xenos_graph_create for the B200 defaults
+ * (148 SMs, 227 KB shared memory per block, 512 tensor-memory columns, 126 MB L2). */
+typedef struct {
+    int32_t sm_count;             /* parallel units the split pass deals tiles to       */
+    int32_t smem_bytes_per_cta;   /* private memory of one unit                         */
+    int32_t tmem_columns;         /* accumulator columns of one unit (fp32, 128 lanes)  */
+    int64_t l2_bytes;             /* memory shared by all units                         */
+} xenos_hw_info_t;
+
+/* One operator (Table 3).  Unused fields are zero / NULL.
+ * weight: CONV: [cout][cin/groups][kh][kw] fp32;  FC: [cout][cin] fp32.
+ * bias:   [cout] fp32 or NULL.
+ * bn_*:   CONV / FC may carry an inference BatchNorm directly (all four non-NULL), and an
+ *         activation, i.e. the already fused CBR form; alternatively BATCHNORM, RELU and
+ *         RELU6 are added as operators of their own and fused by xenos_graph_compile.
+ *         For XENOS_OP_BATCHNORM the four bn_* arrays are [C] of the input.
+ * kh must equal kw.  POOL_*: kh = window, stride, pad; POOL_AVG requires pad == 0. */
+typedef struct {
+    int32_t kind;
+    int32_t cout, kh, kw, stride, pad, groups;
+    int32_t act;
+    const float *weight;
+    const float *bias;
+    const float *bn_gamma, *bn_beta, *bn_mean, *bn_var;
+    float bn_eps;
+} xenos_op_desc_t;
+
+/* Create an empty graph.  hw may be NULL.  *out is owned by the library until
+ * xenos_graph_destroy.  Section 6 (user supplies graph + hardware information). */
+XENOS_API xenos_status_t xenos_graph_create(const xenos_hw_info_t *hw, xenos_graph_t **out);
+
+/* Declare a graph input of c x h x w per image (batch is given at compile / run).
+ * dtype / layout describe the caller's device buffer handed to xenos_graph_run:
+ * FP32_CUDA_CORE graphs take F32 NCHW; BF16_TENSOR graphs take F32 or BF16 NCHW when the
+ * input feeds a convolution with fewer than 8 input channels (an image), BF16 NHWC with a
+ * channel count that is a multiple of 8 otherwise. */
+XENOS_API xenos_status_t xenos_graph_add_input(xenos_graph_t *g, int32_t dtype, int32_t layout,
+                                               int32_t c, int32_t h, int32_t w, xenos_id_t *tensor);
+
+/* Append one operator reading `inputs` (tensor ids) and producing *out_tensor.  Shapes are
+ * inferred here: out = floor((in + 2 pad - k) / stride) + 1.  Weights are copied. */
+XENOS_API xenos_status_t xenos_graph_add_op(xenos_graph_t *g, const xenos_op_desc_t *desc,
+                                            const xenos_id_t *inputs, int32_t n_inputs,
+                                            xenos_id_t *out_tensor);
+
+/* Mark a tensor as a graph output.  The caller's buffer is dense: feature maps
+ * [batch][C][H][W] (NCHW) or [batch][H][W][C] (NHWC), vectors [batch][C].
+ * FP32 graphs: F32 NCHW.  BF16 graphs: vectors F32; feature maps BF16 NHWC. */
+XENOS_API xenos_status_t xenos_graph_mark_output(xenos_graph_t *g, xenos_id_t tensor,
+                                                 int32_t dtype, int32_t layout);
+
+/* Operator linking (Section 4.1, Table 1).
+ *  n_ops == 0: automatic scan of the whole graph for every linkable pattern.
+ *  n_ops  > 0: link exactly this producer->consumer sequence (ids of the operators' output
+ *              tensors, in execution order; BatchNorm / activation records belong to their
+ *              convolution and are not listed).  XENOS_E_NOT_LINKABLE if the sequence is
+ *              not adjacent (checked here) or matches no pattern with a kernel (checked by
+ *              xenos_graph_compile).
+ * Never called: every operator runs as its own kernel (the unlinked baseline; the
+ * Conv-Bn-Relu pre-fusion still applies, as in the paper's Section 3). */
+XENOS_API xenos_status_t xenos_graph_link(xenos_graph_t *g, const xenos_id_t *ops, int32_t n_ops);
+
+/* Operator split (Section 4.2, Eq. 1).  op == -1: automatic for every chain (output
+ * channels first, then rows / columns of the feature map; a reduction split is never
+ * chosen).  Otherwise fix the split of the chain that produces tensor `op`:
+ * parts_outc x parts_h x parts_w pieces (0 = automatic for that dimension); parts_k > 1
+ * requests a reduction (C/R/S) split and is XENOS_E_UNSUPPORTED in this version.
+ * XENOS_E_BAD_SPLIT (from this call or from compile) if a count exceeds the extent it
+ * divides or breaks a kernel limit. */
+XENOS_API xenos_status_t xenos_graph_split(xenos_graph_t *g, xenos_id_t op, int32_t parts_outc,
+                                           int32_t parts_h, int32_t parts_w, int32_t parts_k);
+
+/* Host only: pre-fusion, BatchNorm folding, link + split plans, weight packing, workspace
+ * layout.  *workspace_bytes receives the device bytes xenos_graph_bind needs. */
+XENOS_API xenos_status_t xenos_graph_compile(xenos_graph_t *g, int32_t max_batch, int32_t precision,
+                                             size_t *workspace_bytes);
+
+/* Attach a caller-owned DEVICE workspace (256-byte aligned, >= workspace_bytes) and upload
+ * the packed weights into it on `cuda_stream` (a cudaStream_t; NULL = default stream).
+ * The workspace must stay valid and unshared until destroy or the next bind. */
+XENOS_API xenos_status_t xenos_graph_bind(xenos_graph_t *g, void *workspace_dev, size_t bytes,
+                                          void *cuda_stream);
+
+/* Enqueue one inference of `batch` (<= max_batch) images on `cuda_stream`.
+ * inputs_dev / outputs_dev: HOST arrays of DEVICE pointers in declaration order.
+ * Asynchronous; does not synchronise.  Launch errors are returned, device-side status is
+ * read with xenos_graph_status. */
+XENOS_API xenos_status_t xenos_graph_run(xenos_graph_t *g, int32_t batch,
+                                         const void *const *inputs_dev, void *const *outputs_dev,
+                                         void *cuda_stream);
+
+/* Synchronise `cuda_stream` and return the device status word: XENOS_OK, or
+ * XENOS_E_TIMEOUT / XENOS_E_BOUNDS if a kernel gave up a bounded wait or failed an index
+ * check since the last call (the word is then cleared). */
+XENOS_API xenos_status_t xenos_graph_status(xenos_graph_t *g, void *cuda_stream);
+
+/* Write the compiled plan as JSON into `json` (capacity `cap`, always NUL-terminated when
+ * cap > 0); *needed receives the length including the NUL.  Contents: fused operators,
+ * chains with their Table 1 pattern, tiles, halos, grid, CTA -> tile rule, workspace
+ * offsets, and modelled bytes / FLOPs per chain.  Deterministic: equal graphs and options
+ * give byte-identical plans. */
+XENOS_API xenos_status_t xenos_graph_get_plan(const xenos_graph_t *g, char *json, size_t cap,
+                                              size_t *needed);
+
+/* Number of kernel launches one xenos_graph_run enqueues (valid after compile). */
+XENOS_API xenos_status_t xenos_graph_launch_count(const xenos_graph_t *g, int32_t *launches);
+
+XENOS_API xenos_status_t xenos_graph_destroy(xenos_graph_t *g);
+
+/* Message of the last failing call on g (never NULL; valid until the next call on g).
+ * With g == NULL: message of the last failing xenos_graph_create on this thread. */
+XENOS_API const char *xenos_last_error(const xenos_graph_t *g);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* XENOS_H_ */
