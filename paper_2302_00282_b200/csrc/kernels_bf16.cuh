@@ -1,0 +1,167 @@
+// bf16 NHWC CUDA-core kernels for the operators that are not contractions: depthwise 3x3,
+// pooling, global average, residual add and concat (x.conv depthwise, x.gampool, x.add, x.concat
+// of Table 3).  Each thread moves 8 channels (one 128-bit access) so a warp touches 512
+// contiguous bytes of a pixel's channel vector; arithmetic is fp32, storage rounds to nearest even.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kernels_f32.cuh"
+
+namespace xk {
+
+struct f8 { float v[8]; };
+
+__device__ __forceinline__ f8 unpack8(const uint4 &u) {
+    f8 r;
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        r.v[2 * i] = __uint_as_float(w[i] << 16);
+        r.v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+    return r;
+}
+
+__device__ __forceinline__ uint32_t pack2(float a, float b) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(a, b);   // .x = a (low half), .y = b
+    return *reinterpret_cast<uint32_t *>(&h);
+}
+
+__device__ __forceinline__ uint4 pack8(const f8 &r) {
+    uint4 u;
+    u.x = pack2(r.v[0], r.v[1]); u.y = pack2(r.v[2], r.v[3]);
+    u.z = pack2(r.v[4], r.v[5]); u.w = pack2(r.v[6], r.v[7]);
+    return u;
+}
+
+// Depthwise 3x3 (+ folded BatchNorm bias, activation).  w is fp32 [9][C] tap-major.
+__global__ void dw3x3_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restrict__ w,
+                             const float *__restrict__ b, __nv_bfloat16 *__restrict__ y, int N, int C, int H, int W,
+                             int P, int Q, int stride, int pad, int act) {
+    int C8 = C >> 3;
+    long long total = (long long)N * P * Q * C8;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        int c0 = (int)(i % C8) * 8;
+        long long t = i / C8;
+        int q = (int)(t % Q); t /= Q;
+        int p = (int)(t % P);
+        int n = (int)(t / P);
+        f8 acc;
+        const float4 b0 = *reinterpret_cast<const float4 *>(b + c0), b1 = *reinterpret_cast<const float4 *>(b + c0 + 4);
+        acc.v[0] = b0.x; acc.v[1] = b0.y; acc.v[2] = b0.z; acc.v[3] = b0.w;
+        acc.v[4] = b1.x; acc.v[5] = b1.y; acc.v[6] = b1.z; acc.v[7] = b1.w;
+#pragma unroll
+        for (int r = 0; r < 3; ++r) {
+            int ih = p * stride - pad + r;
+            if (ih < 0 || ih >= H) continue;
+#pragma unroll
+            for (int s = 0; s < 3; ++s) {
+                int iw = q * stride - pad + s;
+                if (iw < 0 || iw >= W) continue;
+                uint4 u = *reinterpret_cast<const uint4 *>(x + (((size_t)n * H + ih) * W + iw) * C + c0);
+                f8 xv = unpack8(u);
+                const float *wt = w + (size_t)(r * 3 + s) * C + c0;
+                const float4 w0 = *reinterpret_cast<const float4 *>(wt), w1 = *reinterpret_cast<const float4 *>(wt + 4);
+                acc.v[0] = fmaf(xv.v[0], w0.x, acc.v[0]); acc.v[1] = fmaf(xv.v[1], w0.y, acc.v[1]);
+                acc.v[2] = fmaf(xv.v[2], w0.z, acc.v[2]); acc.v[3] = fmaf(xv.v[3], w0.w, acc.v[3]);
+                acc.v[4] = fmaf(xv.v[4], w1.x, acc.v[4]); acc.v[5] = fmaf(xv.v[5], w1.y, acc.v[5]);
+                acc.v[6] = fmaf(xv.v[6], w1.z, acc.v[6]); acc.v[7] = fmaf(xv.v[7], w1.w, acc.v[7]);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc.v[j] = apply_act(acc.v[j], act);
+        *reinterpret_cast<uint4 *>(y + (((size_t)n * P + p) * Q + q) * C + c0) = pack8(acc);
+    }
+}
+
+// Max (kind 0) / average (kind 1) pooling.
+__global__ void pool_kernel(const __nv_bfloat16 *__restrict__ x, __nv_bfloat16 *__restrict__ y, int N, int C, int H,
+                            int W, int P, int Q, int k, int stride, int pad, int kind) {
+    int C8 = C >> 3;
+    long long total = (long long)N * P * Q * C8;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        int c0 = (int)(i % C8) * 8;
+        long long t = i / C8;
+        int q = (int)(t % Q); t /= Q;
+        int p = (int)(t % P);
+        int n = (int)(t / P);
+        f8 m, sum;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { m.v[j] = -INFINITY; sum.v[j] = 0.0f; }
+        int cnt = 0;
+        for (int r = 0; r < k; ++r) {
+            int ih = p * stride - pad + r;
+            if (ih < 0 || ih >= H) continue;
+            for (int s = 0; s < k; ++s) {
+                int iw = q * stride - pad + s;
+                if (iw < 0 || iw >= W) continue;
+                f8 xv = unpack8(*reinterpret_cast<const uint4 *>(x + (((size_t)n * H + ih) * W + iw) * C + c0));
+#pragma unroll
+                for (int j = 0; j < 8; ++j) { m.v[j] = fmaxf(m.v[j], xv.v[j]); sum.v[j] += xv.v[j]; }
+                ++cnt;
+            }
+        }
+        if (kind == 1) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) m.v[j] = cnt ? sum.v[j] / (float)cnt : 0.0f;
+        }
+        *reinterpret_cast<uint4 *>(y + (((size_t)n * P + p) * Q + q) * C + c0) = pack8(m);
+    }
+}
+
+// Global average over H*W: one thread per (image, 8 channels), rows summed in ascending order.
+__global__ void gap_kernel(const __nv_bfloat16 *__restrict__ x, void *__restrict__ y, int N, int C, int HW, int out_f32) {
+    int C8 = C >> 3;
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N * C8) return;
+    int c0 = (i % C8) * 8, n = i / C8;
+    f8 sum;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) sum.v[j] = 0.0f;
+    for (int r = 0; r < HW; ++r) {
+        f8 xv = unpack8(*reinterpret_cast<const uint4 *>(x + ((size_t)n * HW + r) * C + c0));
+#pragma unroll
+        for (int j = 0; j < 8; ++j) sum.v[j] += xv.v[j];
+    }
+    float inv = 1.0f / (float)HW;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) sum.v[j] *= inv;
+    if (out_f32) {
+        float *o = reinterpret_cast<float *>(y) + (size_t)n * C + c0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) o[j] = sum.v[j];
+    } else {
+        *reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(y) + (size_t)n * C + c0) = pack8(sum);
+    }
+}
+
+__global__ void add_kernel(const __nv_bfloat16 *__restrict__ a, const __nv_bfloat16 *__restrict__ b,
+                           __nv_bfloat16 *__restrict__ y, long long n8, int act) {
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n8; i += (long long)gridDim.x * blockDim.x) {
+        f8 av = unpack8(reinterpret_cast<const uint4 *>(a)[i]);
+        f8 bv = unpack8(reinterpret_cast<const uint4 *>(b)[i]);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) av.v[j] = apply_act(av.v[j] + bv.v[j], act);
+        reinterpret_cast<uint4 *>(y)[i] = pack8(av);
+    }
+}
+
+// One concat input: x [pixels][Ci] -> y [pixels][Ctot] at channel offset coff.
+__global__ void concat_part_kernel(const __nv_bfloat16 *__restrict__ x, __nv_bfloat16 *__restrict__ y,
+                                   long long pixels, int Ci, int Ctot, int coff) {
+    int C8 = Ci >> 3;
+    long long total = pixels * C8;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        long long px = i / C8;
+        int c0 = (int)(i % C8) * 8;
+        *reinterpret_cast<uint4 *>(y + px * Ctot + coff + c0) = *reinterpret_cast<const uint4 *>(x + px * Ci + c0);
+    }
+}
+
+}  // namespace xk
