@@ -1,0 +1,260 @@
+// CUDA runtime of the library: uploads the packed parameters into the caller's workspace,
+// encodes the TMA descriptors, and enqueues one kernel per launch record on the caller's stream.
+// Allocates no device memory.  (Section 3 of the Xenos paper: the runtime executes the optimised
+// model on the parallel units on top of the operator library.)
+#include <cuda.h>
+#include <cudaTypedefs.h>
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "gemm_tc.cuh"
+#include "graph.hpp"
+#include "kernels_bf16.cuh"
+#include "kernels_f32.cuh"
+
+namespace xenos {
+
+struct Runtime {
+    int device = -1;
+    int sm_count = 0;
+    std::vector<CUtensorMap> tmaps;     // one per launch record (used by gemm launches only)
+    PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
+};
+
+static xenos_status_t cuda_fail(const Graph &g, const char *what, cudaError_t e) {
+    return fail(g, XENOS_E_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+static uint32_t make_idesc(int tile_n) {
+    // kind::f16 instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, M = 128
+    uint32_t d = 0;
+    d |= 1u << 4;                       // D format f32
+    d |= 1u << 7;                       // A format bf16
+    d |= 1u << 10;                      // B format bf16
+    d |= (uint32_t)(tile_n >> 3) << 17; // N / 8
+    d |= (uint32_t)(128 >> 4) << 24;    // M / 16
+    return d;
+}
+
+void runtime_free(Graph &g) {
+    delete static_cast<Runtime *>(g.rt);
+    g.rt = nullptr;
+}
+
+xenos_status_t runtime_bind(Graph &g, void *ws, size_t bytes, void *stream_v) {
+    (void)bytes;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(g, "no CUDA device (this library has no CPU fallback)", e);
+    cudaDeviceProp prop;
+    if ((e = cudaGetDeviceProperties(&prop, dev)) != cudaSuccess) return cuda_fail(g, "cudaGetDeviceProperties", e);
+    if (prop.major != 10) return fail(g, XENOS_E_CUDA, "device is not sm_100 (B200); the kernels are built for sm_100a only");
+    runtime_free(g);
+    Runtime *rt = new Runtime();
+    g.rt = rt;
+    rt->device = dev;
+    rt->sm_count = prop.multiProcessorCount;
+    // parameters -> workspace, status words cleared
+    if (!g.param_blob.empty())
+        if ((e = cudaMemcpyAsync(ws, g.param_blob.data(), g.param_blob.size(), cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+            return cuda_fail(g, "parameter upload", e);
+    if ((e = cudaMemsetAsync(static_cast<uint8_t *>(ws) + g.status_off, 0, 256, stream)) != cudaSuccess)
+        return cuda_fail(g, "status clear", e);
+    if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return cuda_fail(g, "parameter upload sync", e);
+    g.ws = ws;
+    // TMA descriptors of the packed weight matrices
+    bool any_gemm = false;
+    int max_gemm_smem = 0, max_chain_smem = 0;
+    for (const Launch &L : g.launches) {
+        if (L.kind == LK_GEMM) { any_gemm = true; max_gemm_smem = std::max(max_gemm_smem, L.smem_bytes); }
+        if (L.kind == LK_F32_CONV_CONV_POOL) max_chain_smem = std::max(max_chain_smem, L.smem_bytes);
+    }
+    rt->tmaps.resize(g.launches.size());
+    if (any_gemm) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+        if (e != cudaSuccess || !fn || qres != cudaDriverEntryPointSuccess)
+            return fail(g, XENOS_E_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+        rt->encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+        for (size_t i = 0; i < g.launches.size(); ++i) {
+            const Launch &L = g.launches[i];
+            if (L.kind != LK_GEMM) continue;
+            cuuint64_t dims[2] = {(cuuint64_t)L.kpad, (cuuint64_t)L.npad};
+            cuuint64_t strides[1] = {(cuuint64_t)L.kpad * 2};
+            cuuint32_t box[2] = {64u, (cuuint32_t)L.tile_n};
+            cuuint32_t estr[2] = {1u, 1u};
+            void *gaddr = static_cast<uint8_t *>(ws) + L.w_off;
+            // host-side validation of every field the encoder or the copy engine would reject
+            if (((uintptr_t)gaddr & 15u) || (strides[0] & 15u) || box[1] > 256u || box[1] == 0u || L.tile_n % 16)
+                return fail(g, XENOS_E_CUDA, "internal: weight tensor map fields are misaligned");
+            CUresult r = rt->encode(&rt->tmaps[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, gaddr, dims, strides, box, estr,
+                                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) return fail(g, XENOS_E_CUDA, "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r));
+        }
+        if ((e = cudaFuncSetAttribute(xk::gemm_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_gemm_smem)) != cudaSuccess)
+            return cuda_fail(g, "cudaFuncSetAttribute(gemm)", e);
+    }
+    if (max_chain_smem > 48 * 1024)
+        if ((e = cudaFuncSetAttribute(xk::f32_conv_conv_pool_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_chain_smem)) != cudaSuccess)
+            return cuda_fail(g, "cudaFuncSetAttribute(f32 chain)", e);
+    return XENOS_OK;
+}
+
+static int ew_grid(long long total, int block, int sms) {
+    long long b = (total + block - 1) / block;
+    long long cap = (long long)sms * 16;
+    if (b > cap) b = cap;
+    if (b < 1) b = 1;
+    return (int)b;
+}
+
+xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *const *out, void *stream_v) {
+    Runtime *rt = static_cast<Runtime *>(g.rt);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    uint8_t *ws = static_cast<uint8_t *>(g.ws);
+    unsigned int *status = reinterpret_cast<unsigned int *>(ws + g.status_off);
+    auto ptr = [&](int t) -> void * {
+        if (t < 0) return nullptr;
+        const Tensor &x = g.tensors[t];
+        if (x.input_slot >= 0) return const_cast<void *>(in[x.input_slot]);
+        if (x.output_slot >= 0) return out[x.output_slot];
+        return ws + g.place[t].off;
+    };
+    const int sms = rt->sm_count;
+    for (size_t li = 0; li < g.launches.size(); ++li) {
+        const Launch &L = g.launches[li];
+        const int N = batch;
+        switch (L.kind) {
+        case LK_F32_CONV: {
+            long long total = (long long)N * L.K * L.P * L.Q;
+            xk::f32_conv_kernel<<<ew_grid(total, 256, sms), 256, 0, stream>>>(
+                (const float *)ptr(L.in0), (const float *)(ws + L.w_off), (const float *)(ws + L.b_off), (float *)ptr(L.out),
+                N, L.C, L.H, L.W, L.K, L.P, L.Q, L.k, L.stride, L.pad, L.groups, L.act);
+            break;
+        }
+        case LK_F32_POOL: {
+            long long total = (long long)N * L.C * L.P * L.Q;
+            xk::f32_pool_kernel<<<ew_grid(total, 256, sms), 256, 0, stream>>>(
+                (const float *)ptr(L.in0), (float *)ptr(L.out), N, L.C, L.H, L.W, L.P, L.Q, L.pool_k, L.pool_stride, L.pool_pad, L.pool_kind);
+            break;
+        }
+        case LK_F32_GAP: {
+            long long warps = (long long)N * L.C;
+            xk::f32_gap_kernel<<<(int)((warps * 32 + 255) / 256), 256, 0, stream>>>((const float *)ptr(L.in0), (float *)ptr(L.out), N * L.C, L.H * L.W);
+            break;
+        }
+        case LK_F32_ADD: {
+            const Tensor &t = g.tensors[L.out];
+            long long total = (long long)N * (t.is_vec ? t.c : t.c * t.h * t.w);
+            xk::f32_add_kernel<<<ew_grid(total, 256, sms), 256, 0, stream>>>((const float *)ptr(L.in0), (const float *)ptr(L.in1), (float *)ptr(L.out), total, L.act);
+            break;
+        }
+        case LK_F32_CONCAT_PART: {
+            long long total = (long long)N * L.C * L.H * L.W;
+            xk::f32_concat_part_kernel<<<ew_grid(total, 256, sms), 256, 0, stream>>>((const float *)ptr(L.in0), (float *)ptr(L.out), N, L.C, L.H * L.W, L.out_ctot, L.out_coff);
+            break;
+        }
+        case LK_F32_FC:
+            xk::f32_fc_kernel<<<(N * L.K + 255) / 256, 256, 0, stream>>>((const float *)ptr(L.in0), (const float *)(ws + L.w_off), (const float *)(ws + L.b_off), (float *)ptr(L.out), N, L.C, L.K, L.act);
+            break;
+        case LK_F32_CONV_CONV_POOL: {
+            xk::F32ChainParams p;
+            p.x = (const float *)ptr(L.in0); p.y = (float *)ptr(L.out);
+            p.w1 = (const float *)(ws + L.w_off); p.b1 = (const float *)(ws + L.b_off);
+            p.w2 = (const float *)(ws + L.w2_off); p.b2 = (const float *)(ws + L.b2_off);
+            p.N = N; p.C = L.C; p.H = L.H; p.W = L.W; p.Cmid = L.Cmid; p.P = L.P; p.Q = L.Q;
+            p.k = L.k; p.stride = L.stride; p.pad = L.pad; p.act1 = L.act; p.K2 = L.K2; p.act2 = L.act2;
+            p.pool_kind = L.pool_kind; p.pool_k = L.pool_k; p.pool_stride = L.pool_stride; p.PP = L.PP; p.PQ = L.PQ;
+            p.parts_outc = L.parts_outc; p.tile_h = L.tile_h; p.tile_w = L.tile_w; p.tiles_h = L.tiles_h; p.tiles_w = L.tiles_w;
+            p.halo_h = L.halo_h; p.halo_w = L.halo_w; p.status = status;
+            xk::f32_conv_conv_pool_kernel<<<N * L.grid, L.block, L.smem_bytes, stream>>>(p);
+            break;
+        }
+        case LK_DW: {
+            long long total = (long long)N * L.P * L.Q * (L.C / 8);
+            xk::dw3x3_kernel<<<ew_grid(total, 256, sms), 256, 0, stream>>>(
+                (const __nv_bfloat16 *)ptr(L.in0), (const float *)(ws + L.w_off), (const float *)(ws + L.b_off),
+                (__nv_bfloat16 *)ptr(L.out), N, L.C, L.H, L.W, L.P, L.Q, L.stride, L.pad, L.act);
+            break;
+        }
+        case LK_POOL: {
+            long long total = (long long)N * L.P * L.Q * (L.C / 8);
+            xk::pool_kernel<<<ew_grid(total, 256, sms), 256, 0, stream>>>(
+                (const __nv_bfloat16 *)ptr(L.in0), (__nv_bfloat16 *)ptr(L.out), N, L.C, L.H, L.W, L.P, L.Q, L.pool_k, L.pool_stride, L.pool_pad, L.pool_kind);
+            break;
+        }
+        case LK_GAP: {
+            int total = N * (L.C / 8);
+            xk::gap_kernel<<<(total + 127) / 128, 128, 0, stream>>>((const __nv_bfloat16 *)ptr(L.in0), ptr(L.out), N, L.C, L.H * L.W, L.out_dtype == XENOS_DTYPE_F32);
+            break;
+        }
+        case LK_ADD: {
+            const Tensor &t = g.tensors[L.out];
+            long long n8 = (long long)N * (t.is_vec ? t.c : t.c * t.h * t.w) / 8;
+            xk::add_kernel<<<ew_grid(n8, 256, sms), 256, 0, stream>>>((const __nv_bfloat16 *)ptr(L.in0), (const __nv_bfloat16 *)ptr(L.in1), (__nv_bfloat16 *)ptr(L.out), n8, L.act);
+            break;
+        }
+        case LK_CONCAT_PART: {
+            long long pixels = (long long)N * L.H * L.W;
+            xk::concat_part_kernel<<<ew_grid(pixels * (L.C / 8), 256, sms), 256, 0, stream>>>((const __nv_bfloat16 *)ptr(L.in0), (__nv_bfloat16 *)ptr(L.out), pixels, L.C, L.out_ctot, L.out_coff);
+            break;
+        }
+        case LK_GEMM: {
+            xk::GemmParams p;
+            std::memset(&p, 0, sizeof p);
+            for (int s = 0; s < 2; ++s) {
+                const ASeg &a = L.seg[s];
+                xk::GemmSeg &d = p.seg[s];
+                d.mode = a.mode; d.src = ptr(a.tensor); d.C = a.C; d.H = a.H; d.W = a.W; d.k = a.k; d.stride = a.stride; d.pad = a.pad;
+                d.kelems = a.kelems; d.kblocks = a.kblocks; d.src_f32 = a.src_dtype == XENOS_DTYPE_F32; d.dw_act = a.dw_act;
+                d.dw_w = (const float *)(ws + a.dw_w_off); d.dw_b = (const float *)(ws + a.dw_b_off);
+            }
+            p.bias = (const float *)(ws + L.b_off);
+            p.skip = (const __nv_bfloat16 *)ptr(L.skip);
+            p.skip_ctot = L.skip >= 0 ? g.tensors[L.skip].c : 0;
+            p.out = ptr(L.out); p.status = status;
+            p.batch = N; p.P = L.P; p.Q = L.Q; p.rpi = L.rows_per_image;
+            p.map_mode = L.map_mode; p.tile_rows = L.tile_rows; p.imgs_per_tile = L.imgs_per_tile;
+            p.th = L.patch_th; p.tw = L.patch_tw; p.rh = L.patch_rh; p.rw = L.patch_rw; p.tiles_y = L.tiles_y; p.tiles_x = L.tiles_x;
+            p.pool_k = L.pool_k; p.pool_stride = L.pool_stride; p.pool_pad = L.pool_pad; p.PP = L.PP; p.PQ = L.PQ;
+            p.kblocks = L.kblocks; p.stages = L.stages; p.tile_n = L.tile_n; p.n_tiles = L.n_tiles; p.N = L.K;
+            p.act = L.act; p.act2 = L.act2; p.epi = L.epi; p.out_ctot = L.out_ctot; p.out_coff = L.out_coff;
+            p.out_f32 = L.out_dtype == XENOS_DTYPE_F32;
+            p.idesc = make_idesc(L.tile_n);
+            int m_tiles;
+            if (L.epi == EPI_POOL) m_tiles = N * L.tiles_y * L.tiles_x;
+            else if (L.epi == EPI_GAP) m_tiles = (N + L.imgs_per_tile - 1) / L.imgs_per_tile;
+            else m_tiles = (int)(((long long)N * L.rows_per_image + 127) / 128);
+            xk::gemm_chain_kernel<<<m_tiles * L.n_tiles, 192, L.smem_bytes, stream>>>(rt->tmaps[li], p);
+            break;
+        }
+        default:
+            return fail(g, XENOS_E_UNSUPPORTED, "internal: launch record without a kernel");
+        }
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return cuda_fail(g, "kernel launch", e);
+    }
+    return XENOS_OK;
+}
+
+xenos_status_t runtime_status(Graph &g, void *stream_v) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    cudaError_t e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) return cuda_fail(g, "stream synchronize", e);
+    unsigned int word = 0;
+    uint8_t *ws = static_cast<uint8_t *>(g.ws);
+    if ((e = cudaMemcpy(&word, ws + g.status_off, 4, cudaMemcpyDeviceToHost)) != cudaSuccess) return cuda_fail(g, "status read", e);
+    if (word == 0) return XENOS_OK;
+    cudaMemset(ws + g.status_off, 0, 4);
+    int code = -(int)(word & 0xffu);
+    return fail(g, code, code == XENOS_E_TIMEOUT ? "a kernel gave up a bounded wait" : "a kernel failed an index check");
+}
+
+}  // namespace xenos
