@@ -1,0 +1,283 @@
+"""Benchmark: images/s of one linked CNN graph on B200, with roofline and CPU-oracle context.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload NAME]
+
+A step is one pass of the whole hot path (every linked chain of the graph) over one batch of
+seeded synthetic images.  Default workload: MobileNetV1-style depthwise-separable graph,
+width 1.0, 224x224, batch 32, bf16 activations with fp32 accumulation, linked execution.
+Prints ONE JSON line (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from xenos_workloads import graphs  # noqa: E402
+
+WORKLOADS = {
+    "mobilenet_v1_b32": (1, 32), "mobilenet_v1_b1": (1, 1),
+    "resnet18_b32": (2, 32), "resnet18_b1": (2, 1),
+    "squeezenet11_b32": (3, 32), "squeezenet11_b1": (3, 1),
+    "resnet50_stress_b64": (4, 64), "single_chain_b1": (0, 1),
+}
+L2_FLUSH_BYTES = 256 << 20
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d.get("bf16_tflops_sustained", d["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        q = "clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown," \
+            "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap"
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits", "-lms", "100",
+                                          "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.t.join(timeout=2)
+        mhz, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 6:
+                continue
+            try:
+                mhz.append(float(r[0])); mx = float(r[1])
+            except ValueError:
+                continue
+            for n, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return dict(sm_mhz=float(np.median(mhz)) if mhz else None, sm_max_mhz=mx, reasons=sorted(reasons), samples=len(mhz))
+
+
+def reference_arm(args, spec, batch):
+    """Times the CPU oracle (as it stands) on the host cores: one step = a bounded sample of the batch."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle as xo
+    from oracle import interp
+    P = graphs.make_params(spec)
+    sample = min(batch, args.ref_images)
+    x = graphs.make_input(spec, sample)
+    for _ in range(min(args.warmup, 1)):
+        interp.run_graph(spec, P, x[:1])
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        interp.run_graph(spec, P, x)
+    dt = time.perf_counter() - t0
+    val = sample * args.steps / dt
+    line = dict(impl="reference", metric="images/sec per linked CNN graph", value=val, unit="images/s", n_gpus=args.gpus,
+                steps=args.steps, warmup=args.warmup, ms_per_step=1e3 * dt / args.steps, higher_is_better=True,
+                scaling="weak", vs_baseline=None, dtype="f32", data="synthetic",
+                config=dict(workload=args.workload, graph=spec.name, global_batch=batch, mode="cpu oracle, one operator at a time"),
+                cpu_baseline=dict(value=val, unit="images/s", cores=xo.num_threads(), kind="oracle",
+                                  sample=f"{sample} of {batch} images per step"),
+                e2e=dict(value=val, unit="images/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="xenos")
+    ap.add_argument("--workload", default="mobilenet_v1_b32", choices=sorted(WORKLOADS))
+    ap.add_argument("--ref-images", type=int, default=8, help="images per step of the CPU oracle arm")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--unlinked", action="store_true", help="time the unlinked execution as the main arm")
+    args = ap.parse_args()
+    cfg, batch = WORKLOADS[args.workload]
+    spec, _ = graphs.config(cfg)
+    if args.impl == "reference":
+        reference_arm(args, spec, batch)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2302_00282_b200 import binding as xb
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    fp32 = spec.precision == "fp32"
+    P = graphs.make_params(spec)
+    x = graphs.make_input(spec, batch)
+
+    def make(linked):
+        g, ids = xb.graph_from_spec(spec, P, in_dtype=xb.DTYPE_F32 if fp32 else xb.DTYPE_BF16, in_layout=xb.LAYOUT_NCHW)
+        if linked:
+            g.link()
+        nbytes = g.compile(batch, xb.PRECISION_FP32_CUDA_CORE if fp32 else xb.PRECISION_BF16_TENSOR)
+        ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device="cuda")
+        g.bind(ws.data_ptr(), ws.numel(), torch.cuda.current_stream().cuda_stream)
+        return g, ws
+
+    stream = torch.cuda.current_stream().cuda_stream
+    x_host = torch.from_numpy(x) if fp32 else torch.from_numpy(x).to(torch.bfloat16)
+    x_pin = x_host.pin_memory()
+    x_dev = x_host.cuda()
+    oshape = spec.shapes[spec.output]
+    if len(oshape) == 1:
+        out_dev = torch.empty((batch, oshape[0]), dtype=torch.float32, device="cuda")
+    elif fp32:
+        out_dev = torch.empty((batch,) + tuple(oshape), dtype=torch.float32, device="cuda")
+    else:
+        out_dev = torch.empty((batch, oshape[1], oshape[2], oshape[0]), dtype=torch.bfloat16, device="cuda")
+    out_pin = torch.empty_like(out_dev, device="cpu").pin_memory()
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+
+    def time_steps(g, steps, warmup, e2e=False):
+        for _ in range(warmup):
+            g.run(batch, [x_dev.data_ptr()], [out_dev.data_ptr()], stream)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        ends = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        for i in range(steps):
+            flush.fill_(i & 0xFF)                    # evict L2 between timed steps (outside the timed interval)
+            starts[i].record()
+            if e2e:
+                x_dev.copy_(x_pin, non_blocking=True)
+            g.run(batch, [x_dev.data_ptr()], [out_dev.data_ptr()], stream)
+            if e2e:
+                out_pin.copy_(out_dev, non_blocking=True)
+            ends[i].record()
+        torch.cuda.synchronize()
+        g.status(stream)
+        total_ms = sum(s.elapsed_time(e) for s, e in zip(starts, ends))
+        if world > 1:
+            t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            total_ms = float(t.item())
+            dist.barrier()
+        torch.cuda.synchronize()
+        return total_ms
+
+    g_main, ws_main = make(not args.unlinked)
+    sampler = ClockSampler(local)
+    sampler.start()
+    total_ms = time_steps(g_main, args.steps, args.warmup)
+    clocks = sampler.stop()
+    value = world * batch * args.steps / (total_ms * 1e-3)
+    e2e_ms = time_steps(g_main, max(3, args.steps // 4), 3, e2e=True)
+    e2e_val = world * batch * max(3, args.steps // 4) / (e2e_ms * 1e-3)
+
+    # the other arm (unlinked when the main arm is linked) on the same inputs, fewer steps
+    g_other, ws_other = make(args.unlinked)
+    osteps = max(3, args.steps // 4)
+    other_ms = time_steps(g_other, osteps, 3)
+    other_val = world * batch * osteps / (other_ms * 1e-3)
+
+    # per-launch device times of the main arm -> roofline of the dominant kernel
+    plan = g_main.plan()
+    reps = 5
+    acc = np.zeros(len(plan["launches"]))
+    for i in range(reps + 1):
+        flush.fill_(i)
+        ms = g_main.profile(batch, [x_dev.data_ptr()], [out_dev.data_ptr()], stream)
+        if i:
+            acc += np.array(ms)
+    acc /= reps
+    peaks = measured_peaks()
+    by_kind = {}
+    for L, ms in zip(plan["launches"], acc):
+        d = by_kind.setdefault(L["kind"], dict(ms=0.0, bytes=0.0, flops=0.0, launches=0))
+        d["ms"] += float(ms); d["bytes"] += L["bytes"]; d["flops"] += L["flops"]; d["launches"] += 1
+    dom = max(by_kind, key=lambda k: by_kind[k]["ms"])
+    dk = by_kind[dom]
+    t_mem = dk["bytes"] / (peaks["hbm_gbs"] * 1e9)
+    t_tc = dk["flops"] / (peaks["bf16_tflops"] * 1e12)
+    if t_tc > t_mem and not fp32:
+        roof = dict(bound="tensor", achieved=dk["flops"] / (dk["ms"] * 1e-3) / 1e12, peak=peaks["bf16_tflops"], unit="TFLOP/s")
+    else:
+        roof = dict(bound="hbm", achieved=dk["bytes"] / (dk["ms"] * 1e-3) / 1e9, peak=peaks["hbm_gbs"], unit="GB/s")
+    roof.update(frac=roof["achieved"] / roof["peak"], traffic=None, kernel=dom, launches_per_step=dk["launches"],
+                avg_launch_us=1e3 * dk["ms"] / dk["launches"], peak_source=peaks["source"],
+                algorithmic_bytes_per_step=dk["bytes"], flops_per_step=dk["flops"])
+    chains = []
+    for c in plan["chains"]:
+        ms = float(sum(acc[i] for i in c["launches"]))
+        tm, tt = c["bytes_linked"] / (peaks["hbm_gbs"] * 1e9), c["flops"] / (peaks["bf16_tflops"] * 1e12)
+        chains.append(dict(id=c["id"], kind=c["kind"], us=1e3 * ms, bound="tensor" if tt > tm else "hbm",
+                           frac=(max(tm, tt) * 1e3) / ms if ms > 0 else None))
+
+    line = dict(metric="images/sec per linked CNN graph", value=value, unit="images/s", n_gpus=world, steps=args.steps,
+                warmup=args.warmup, ms_per_step=total_ms / args.steps, higher_is_better=True, scaling="weak",
+                vs_baseline=None, dtype="f32" if fp32 else "bf16", data="synthetic",
+                config=dict(workload=args.workload, graph=spec.name, global_batch=batch * world, input=list(spec.in_shape),
+                            mode="unlinked" if args.unlinked else "linked", l2="flushed between timed steps (256 MiB write)",
+                            parallelism="replicas only" if world > 1 else "single GPU"),
+                clocks=clocks,
+                e2e=dict(value=e2e_val, unit="images/s", h2d_bytes_per_step=x_pin.numel() * x_pin.element_size(),
+                         d2h_bytes_per_step=out_pin.numel() * out_pin.element_size()),
+                gpu_launches=g_main.launch_count() * args.steps,
+                roofline=roof,
+                linked_vs_unlinked=dict(other_mode="linked" if args.unlinked else "unlinked", other_value=other_val,
+                                        speedup=(value / other_val) if not args.unlinked else (other_val / value),
+                                        launches_linked=(g_other if args.unlinked else g_main).launch_count(),
+                                        launches_unlinked=(g_main if args.unlinked else g_other).launch_count(),
+                                        model_bytes_linked=plan["bytes_linked"], model_bytes_unlinked=plan["bytes_unlinked"]),
+                chains=chains)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle as xo
+        from oracle import interp
+        sample = min(batch, 16)
+        interp.run_graph(spec, P, x[:1])
+        t0 = time.perf_counter()
+        interp.run_graph(spec, P, x[:sample])
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = dict(value=sample / dt, unit="images/s", cores=xo.num_threads(), kind="oracle",
+                                    sample=f"{sample} of {batch} images, one pass, {dt:.1f} s")
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

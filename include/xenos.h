@@ -176,6 +176,15 @@ XENOS_API xenos_status_t xenos_graph_run(xenos_graph_t *g, int32_t batch,
                                          const void *const *inputs_dev, void *const *outputs_dev,
                                          void *cuda_stream);
 
+/* Like xenos_graph_run, but brackets every kernel launch with CUDA events on `cuda_stream`,
+ * synchronises, and writes the device time of launch i (milliseconds) to ms_per_launch[i]
+ * (HOST array of n_launches = xenos_graph_launch_count entries).  This is the PROFILING step
+ * of the paper's Algorithm 1 ("Enumerating Partition Schemes") for one fixed scheme; it
+ * creates and destroys CUDA events, allocates no device memory, and is not for hot loops. */
+XENOS_API xenos_status_t xenos_graph_profile(xenos_graph_t *g, int32_t batch,
+                                             const void *const *inputs_dev, void *const *outputs_dev,
+                                             void *cuda_stream, float *ms_per_launch, int32_t n_launches);
+
 /* Synchronise `cuda_stream` and return the device status word: XENOS_OK, or
  * XENOS_E_TIMEOUT / XENOS_E_BOUNDS if a kernel gave up a bounded wait or failed an index
  * check since the last call (the word is then cleared). */

@@ -229,6 +229,24 @@ xenos_status_t xenos_graph_run(xenos_graph_t *gp, int32_t batch, const void *con
     XENOS_GUARD_END(gp)
 }
 
+xenos_status_t xenos_graph_profile(xenos_graph_t *gp, int32_t batch, const void *const *inputs_dev,
+                                   void *const *outputs_dev, void *cuda_stream, float *ms_per_launch,
+                                   int32_t n_launches) {
+    if (!gp) return XENOS_E_INVALID;
+    XENOS_GUARD_BEGIN
+    Graph &g = gp->g;
+    if (g.state != ST_BOUND) return fail(g, XENOS_E_STATE, "profile before bind");
+    if (batch < 1 || batch > g.max_batch) return fail(g, XENOS_E_INVALID, "profile: batch exceeds max_batch given to compile");
+    if (!inputs_dev || !outputs_dev || !ms_per_launch) return fail(g, XENOS_E_INVALID, "profile: NULL pointer");
+    if (n_launches != (int32_t)g.launches.size()) return fail(g, XENOS_E_INVALID, "profile: n_launches must equal xenos_graph_launch_count");
+    for (size_t i = 0; i < g.inputs.size(); ++i)
+        if (!inputs_dev[i]) return fail(g, XENOS_E_INVALID, "profile: NULL input pointer");
+    for (size_t i = 0; i < g.outputs.size(); ++i)
+        if (!outputs_dev[i]) return fail(g, XENOS_E_INVALID, "profile: NULL output pointer");
+    return runtime_run(g, batch, inputs_dev, outputs_dev, cuda_stream, ms_per_launch);
+    XENOS_GUARD_END(gp)
+}
+
 xenos_status_t xenos_graph_status(xenos_graph_t *gp, void *cuda_stream) {
     if (!gp) return XENOS_E_INVALID;
     XENOS_GUARD_BEGIN

@@ -191,7 +191,8 @@ void emit_plan_json(Graph &g);
 uint16_t f32_to_bf16_rne(float f);
 // runtime.cu
 xenos_status_t runtime_bind(Graph &g, void *ws, size_t bytes, void *stream);
-xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *const *out, void *stream);
+xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *const *out, void *stream,
+                           float *ms_per_launch = nullptr);
 xenos_status_t runtime_status(Graph &g, void *stream);
 void runtime_free(Graph &g);
 

@@ -115,7 +115,8 @@ static int ew_grid(long long total, int block, int sms) {
     return (int)b;
 }
 
-xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *const *out, void *stream_v) {
+xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *const *out, void *stream_v,
+                           float *ms_per_launch) {
     Runtime *rt = static_cast<Runtime *>(g.rt);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     uint8_t *ws = static_cast<uint8_t *>(g.ws);
@@ -128,6 +129,13 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
         return ws + g.place[t].off;
     };
     const int sms = rt->sm_count;
+    std::vector<cudaEvent_t> ev;
+    if (ms_per_launch) {
+        ev.resize(g.launches.size() + 1);
+        for (auto &e : ev)
+            if (cudaEventCreate(&e) != cudaSuccess) return fail(g, XENOS_E_CUDA, "cudaEventCreate failed");
+        cudaEventRecord(ev[0], stream);
+    }
     for (size_t li = 0; li < g.launches.size(); ++li) {
         const Launch &L = g.launches[li];
         const int N = batch;
@@ -240,6 +248,16 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
         }
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return cuda_fail(g, "kernel launch", e);
+        if (ms_per_launch) cudaEventRecord(ev[li + 1], stream);
+    }
+    if (ms_per_launch) {
+        cudaError_t e = cudaStreamSynchronize(stream);
+        for (size_t li = 0; li < g.launches.size(); ++li) {
+            ms_per_launch[li] = 0.0f;
+            if (e == cudaSuccess) cudaEventElapsedTime(&ms_per_launch[li], ev[li], ev[li + 1]);
+        }
+        for (auto &x : ev) cudaEventDestroy(x);
+        if (e != cudaSuccess) return cuda_fail(g, "profile synchronize", e);
     }
     return XENOS_OK;
 }

@@ -1,0 +1,273 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs.  fp32 CUDA-core graphs: max relative error <= 1e-4; bf16 tensor-core graphs:
+max abs error <= 2e-2 * max|output|."""
+import numpy as np
+import pytest
+
+import oracle as xo
+from oracle import interp
+from xenos_workloads import gen, graphs
+from xenos_workloads.graphs import GraphSpec
+
+from gpu_util import GpuGraph, abs_err_scaled, log, rel_err_fp32
+
+pytestmark = pytest.mark.gpu
+BF16_TOL = 2e-2
+FP32_TOL = 1e-4
+
+
+def check_bf16(name, spec, batch, linked=True, in_mode="f32_nchw", seed=gen.DEFAULT_SEED, max_batch=None,
+               splits=(), images=None, links=None):
+    P = graphs.make_params(spec, seed)
+    x = graphs.make_input(spec, batch, seed)
+    if in_mode != "f32_nchw":
+        x = xo.round_bf16(x)          # the device buffer holds bf16 values; the oracle reads the same numbers
+    gg = GpuGraph(spec, P, max_batch or batch, linked=linked, in_mode=in_mode, splits=splits, links=links)
+    y = gg.run(x)
+    sel = list(range(batch)) if images is None else images
+    o = interp.run_graph(spec, P, x[sel])
+    err = abs_err_scaled(y[sel], o)
+    nan = int(np.isnan(y).sum())
+    log(dict(test=name, batch=batch, linked=linked, err=err, nan=nan, launches=gg.g.launch_count(), omax=float(np.abs(o).max())))
+    assert nan == 0, f"{name}: {nan} NaN outputs (unwritten elements)"
+    assert err <= BF16_TOL, f"{name}: scaled abs err {err:.3e}"
+    return y, o, gg
+
+
+# ---- fp32 CUDA-core chain (benchmark config 0) ---------------------------------------------------
+@pytest.mark.parametrize("linked", [True, False])
+@pytest.mark.parametrize("hw,batch", [(32, 1), (30, 3), (9, 2)])
+def test_fp32_single_chain(linked, hw, batch):
+    spec = graphs.single_chain(hw=hw)
+    P = graphs.make_params(spec)
+    x = graphs.make_input(spec, batch)
+    gg = GpuGraph(spec, P, batch, linked=linked)
+    y = gg.run(x)
+    o = interp.run_graph(spec, P, x)
+    err = rel_err_fp32(y, o)
+    log(dict(test="fp32_single_chain", hw=hw, batch=batch, linked=linked, err=err))
+    assert not np.isnan(y).any()
+    assert err <= FP32_TOL
+
+
+@pytest.mark.parametrize("split", [dict(parts_outc=4, parts_h=2, parts_w=1), dict(parts_outc=1, parts_h=16, parts_w=16),
+                                   dict(parts_outc=32, parts_h=1, parts_w=1), dict(parts_outc=2, parts_h=4, parts_w=8)])
+def test_fp32_chain_explicit_splits_agree_bitwise(split):
+    """Eq. 1: an output-channel / row / column split changes no value."""
+    spec = graphs.single_chain()
+    P = graphs.make_params(spec)
+    x = graphs.make_input(spec, 2)
+    base = GpuGraph(spec, P, 2, linked=True).run(x)
+    y = GpuGraph(spec, P, 2, linked=True, splits=[("mp", split)]).run(x)
+    assert np.array_equal(y, base)
+    assert rel_err_fp32(y, interp.run_graph(spec, P, x)) <= FP32_TOL
+
+
+def test_fp32_mode_runs_other_graphs_unlinked():
+    spec = graphs.squeezenet11(hw=47, classes=10, scale=4)
+    spec.precision = "fp32"
+    P = graphs.make_params(spec)
+    x = graphs.make_input(spec, 2)
+    y = GpuGraph(spec, P, 2, linked=False).run(x)
+    assert rel_err_fp32(y, interp.run_graph(spec, P, x)) <= FP32_TOL
+
+
+# ---- bf16: single operators ----------------------------------------------------------------------
+def _one(build, cin, hw):
+    g = GraphSpec("unit", (cin, hw, hw))
+    build(g)
+    return g
+
+
+CONV_CASES = [
+    # cin, hw, cout, k, stride, pad, batch
+    (64, 16, 64, 1, 1, 0, 2),       # pointwise: a plain matmul, one K block
+    (128, 9, 32, 1, 1, 0, 3),       # two K blocks, ragged M tail (243 rows)
+    (16, 12, 48, 3, 1, 1, 2),       # taps share K blocks (C = 16)
+    (48, 10, 24, 3, 2, 1, 2),       # C = 48: chunks straddle K blocks; stride 2
+    (64, 14, 320, 3, 1, 1, 1),      # two N tiles
+    (32, 8, 40, 1, 2, 0, 2),        # strided 1x1 (projection shape), N not a multiple of 16
+    (8, 20, 16, 7, 2, 3, 1),        # 7x7
+    (256, 7, 1000, 1, 1, 0, 2),     # classifier-like: ragged N = 1000
+]
+
+
+@pytest.mark.parametrize("case", CONV_CASES)
+def test_bf16_conv(case):
+    cin, hw, cout, k, st, pad, batch = case
+    spec = _one(lambda g: g.cbr("c", "input", cout, k, st, pad, act="relu"), cin, hw)
+    check_bf16(f"conv{case}", spec, batch, linked=False, in_mode="bf16_nhwc")
+
+
+def test_bf16_conv1x1_equals_matmul():
+    spec = _one(lambda g: g.conv("c", "input", 64, 1), 64, 8)
+    P = graphs.make_params(spec)
+    x = xo.round_bf16(graphs.make_input(spec, 2))
+    y = GpuGraph(spec, P, 2, linked=False, in_mode="bf16_nhwc").run(x)
+    w = xo.round_bf16(P["c"]["w"])[:, :, 0, 0].astype(np.float64)
+    ref = np.einsum("kc,nchw->nkhw", w, x.astype(np.float64))
+    # inputs and weights are exactly representable, accumulation is fp32, the store rounds to bf16
+    assert np.abs(y - ref).max() <= 2 ** -8 * np.abs(ref).max() + 1e-6
+
+
+@pytest.mark.parametrize("stem", [(3, 2, 1, 32, 33), (7, 2, 3, 64, 40), (3, 2, 0, 64, 31)])
+@pytest.mark.parametrize("in_mode", ["f32_nchw", "bf16_nchw"])
+def test_bf16_stem(stem, in_mode):
+    k, st, pad, cout, hw = stem
+    spec = _one(lambda g: g.cbr("stem", "input", cout, k, st, pad, act="relu6"), 3, hw)
+    check_bf16(f"stem{stem}{in_mode}", spec, 2, linked=False, in_mode=in_mode)
+
+
+@pytest.mark.parametrize("c,hw,stride", [(32, 12, 1), (64, 11, 2), (8, 5, 1)])
+def test_bf16_depthwise(c, hw, stride):
+    spec = _one(lambda g: g.cbr("dw", "input", c, 3, stride, 1, groups=c, act="relu6"), c, hw)
+    check_bf16(f"dw{c}_{hw}_{stride}", spec, 2, linked=False, in_mode="bf16_nhwc")
+
+
+@pytest.mark.parametrize("k,st,pad", [(3, 2, 1), (3, 2, 0), (2, 2, 0)])
+def test_bf16_maxpool(k, st, pad):
+    spec = _one(lambda g: g.pool("mp", "input", "maxpool", k, st, pad), 16, 13)
+    y, o, _ = check_bf16(f"maxpool{k}{st}{pad}", spec, 2, linked=False, in_mode="bf16_nhwc")
+    assert np.array_equal(y, o)          # comparisons only: exact
+
+
+def test_bf16_gap_add_concat_fc():
+    def build(g):
+        a = g.cbr("a", "input", 24, 1)
+        b = g.cbr("b", "input", 24, 3, 1, 1)
+        s = g.add("s", a, b)
+        s = g.act("s.relu", s, "relu")
+        c = g.concat("cat", [s, a])
+        v = g.gap("gap", c)
+        g.fc("fc", v, 10)
+    spec = _one(build, 16, 9)
+    check_bf16("gap_add_concat_fc", spec, 3, linked=False, in_mode="bf16_nhwc")
+
+
+# ---- bf16: linked chains -------------------------------------------------------------------------
+@pytest.mark.parametrize("c,cout,hw,stride,batch", [(32, 64, 14, 1, 2), (64, 128, 15, 2, 3), (8, 16, 6, 1, 1), (128, 320, 7, 1, 2)])
+@pytest.mark.parametrize("linked", [True, False])
+def test_bf16_dw_pw(c, cout, hw, stride, batch, linked):
+    def build(g):
+        x = g.cbr("dw", "input", c, 3, stride, 1, groups=c, act="relu6")
+        g.cbr("pw", x, cout, 1, act="relu6")
+    spec = _one(build, c, hw)
+    _, _, gg = check_bf16(f"dw_pw{(c, cout, hw, stride)}", spec, batch, linked=linked, in_mode="bf16_nhwc")
+    assert gg.g.launch_count() == (1 if linked else 2)
+
+
+def test_bf16_dw_pw_gap_fc():
+    def build(g):
+        x = g.cbr("dw", "input", 64, 3, 1, 1, groups=64, act="relu6")
+        x = g.cbr("pw", x, 128, 1, act="relu6")
+        x = g.gap("gap", x)
+        g.fc("fc", x, 24)
+    spec = _one(build, 64, 7)
+    _, _, gg = check_bf16("dw_pw_gap_fc", spec, 5, linked=True, in_mode="bf16_nhwc")
+    assert gg.g.launch_count() == 2
+
+
+@pytest.mark.parametrize("k,st,pad,pk,ps,pp,hw", [(3, 1, 1, 3, 2, 1, 20), (3, 2, 0, 3, 2, 0, 31), (1, 1, 0, 2, 2, 0, 16)])
+def test_bf16_conv_maxpool(k, st, pad, pk, ps, pp, hw):
+    def build(g):
+        x = g.cbr("c", "input", 32, k, st, pad)
+        g.pool("mp", x, "maxpool", pk, ps, pp)
+    spec = _one(build, 16, hw)
+    _, _, gg = check_bf16(f"conv_maxpool{(k, st, pad, pk, ps, pp, hw)}", spec, 2, linked=True, in_mode="bf16_nhwc")
+    assert gg.g.launch_count() == 1
+
+
+def test_bf16_stem_maxpool_linked():
+    def build(g):
+        x = g.cbr("stem", "input", 64, 7, 2, 3)
+        g.pool("mp", x, "maxpool", 3, 2, 1)
+    spec = _one(build, 3, 64)
+    _, _, gg = check_bf16("stem_maxpool", spec, 2, linked=True)
+    assert gg.g.launch_count() == 1
+
+
+def test_bf16_conv_gap_linked():
+    def build(g):
+        x = g.cbr("cls", "input", 40, 1, act=None, bn=False, bias=True)
+        g.gap("gap", x)
+    spec = _one(build, 64, 7)
+    _, _, gg = check_bf16("conv_gap", spec, 5, linked=True, in_mode="bf16_nhwc")
+    assert gg.g.launch_count() == 1
+
+
+@pytest.mark.parametrize("proj", [False, True])
+def test_bf16_shortcut_block(proj):
+    def build(g):
+        c = 32
+        y = g.cbr("c1", "input", 64 if proj else c, 3, 2 if proj else 1, 1)
+        y = g.cbr("c2", y, 64 if proj else c, 3, 1, 1, act=None)
+        skip = "input"
+        if proj:
+            skip = g.cbr("proj", "input", 64, 1, 2, 0, act=None)
+        y = g.add("add", y, skip)
+        g.act("relu", y, "relu")
+    spec = _one(build, 32, 14)
+    _, _, gg = check_bf16(f"shortcut_proj{proj}", spec, 2, linked=True, in_mode="bf16_nhwc")
+    assert gg.g.launch_count() == 2      # c1, then {c2 [+proj] + add + relu}
+
+
+@pytest.mark.parametrize("pool", [False, True])
+def test_bf16_fire_module(pool):
+    def build(g):
+        sq = g.cbr("sq", "input", 16, 1, bn=False, bias=True)
+        e1 = g.cbr("e1", sq, 64, 1, bn=False, bias=True)
+        e3 = g.cbr("e3", sq, 64, 3, 1, 1, bn=False, bias=True)
+        x = g.concat("cat", [e1, e3])
+        if pool:
+            g.pool("mp", x, "maxpool", 3, 2, 0)
+    spec = _one(build, 64, 15)
+    _, _, gg = check_bf16(f"fire_pool{pool}", spec, 2, linked=True, in_mode="bf16_nhwc")
+    assert gg.g.launch_count() == 2      # squeeze, then {expand1x1, expand3x3, concat [, pool]}
+
+
+def test_bf16_linked_equals_unlinked_closely():
+    spec = graphs.mobilenet_v1(hw=64, width=0.5, classes=16)
+    yl, o, _ = check_bf16("mbv1_small_linked", spec, 3, linked=True)
+    yu, _, _ = check_bf16("mbv1_small_unlinked", spec, 3, linked=False)
+    assert abs_err_scaled(yl, yu) <= 1e-2
+
+
+def test_bf16_batch_smaller_than_max_batch():
+    spec = graphs.mobilenet_v1(hw=32, width=0.25, classes=16)
+    check_bf16("mbv1_batch3_of_8", spec, 3, linked=True, max_batch=8)
+
+
+# ---- bf16: whole graphs ---------------------------------------------------------------------------
+@pytest.mark.parametrize("linked", [True, False])
+@pytest.mark.parametrize("name,kw", [("mobilenet_v1", dict(hw=64, width=0.25, classes=24)),
+                                     ("resnet18", dict(hw=64, base=16, classes=24)),
+                                     ("squeezenet11", dict(hw=63, classes=24, scale=2)),
+                                     ("resnet50_stress", dict(hw=64, base=8, blocks=(2, 1, 1, 1)))])
+def test_bf16_small_graphs(name, kw, linked):
+    spec = getattr(graphs, name)(**kw)
+    check_bf16(f"{name}_small", spec, 3, linked=linked)
+
+
+@pytest.mark.parametrize("linked", [True, False])
+@pytest.mark.parametrize("cfg", [1, 2, 3])
+def test_bf16_full_configs_batch1(cfg, linked):
+    spec, _ = graphs.config(cfg)
+    check_bf16(f"cfg{cfg}_n1", spec, 1, linked=linked, in_mode="bf16_nchw")
+
+
+def test_bf16_mobilenet_batch32_bench_configuration():
+    """The configuration bench.py times: MobileNetV1 1.0, batch 32, linked, bf16 NCHW images."""
+    spec, _ = graphs.config(1)
+    check_bf16("cfg1_n32", spec, 32, linked=True, in_mode="bf16_nchw", images=[0, 17, 31])
+
+
+@pytest.mark.parametrize("cfg", [2, 3])
+def test_bf16_full_configs_batch32_sampled(cfg):
+    spec, _ = graphs.config(cfg)
+    check_bf16(f"cfg{cfg}_n32", spec, 32, linked=True, in_mode="bf16_nchw", images=[0, 31])
+
+
+def test_bf16_stress_graph_batch64_sampled():
+    """Config 4 at full size; the oracle evaluates images 0 and 63 (images are independent)."""
+    spec, _ = graphs.config(4)
+    check_bf16("cfg4_n64", spec, 64, linked=True, in_mode="bf16_nchw", images=[0, 63])
