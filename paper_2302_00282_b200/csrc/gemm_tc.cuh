@@ -404,21 +404,23 @@ __global__ void __launch_bounds__(192) gemm_chain_kernel(const __grid_constant__
                 v[i] = apply_act(v[i] + b.x, g.act); v[i + 1] = apply_act(v[i + 1] + b.y, g.act);
                 v[i + 2] = apply_act(v[i + 2] + b.z, g.act); v[i + 3] = apply_act(v[i + 3] + b.w, g.act);
             }
+            // shortcut connection with an identity branch: the skip tile is read once, here
+            const size_t pix = ((size_t)rp.n * g.P + rp.p) * g.Q + rp.q;
+            if (g.skip && rp.valid) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    if (nc + h * 8 + 8 > g.N) break;
+                    f8 sv = unpack8(__ldg(reinterpret_cast<const uint4 *>(g.skip + pix * g.skip_ctot + nc + h * 8)));
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) v[h * 8 + i] += sv.v[i];
+                }
+            }
+            if (g.act2) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) v[i] = apply_act(v[i], g.act2);
+            }
             if (g.epi == GE_STORE) {
                 if (!rp.valid || !ok) continue;
-                size_t pix = ((size_t)rp.n * g.P + rp.p) * g.Q + rp.q;
-                if (g.skip) {
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        if (nc + h * 8 + 8 > g.N) break;
-                        f8 sv = unpack8(__ldg(reinterpret_cast<const uint4 *>(g.skip + pix * g.skip_ctot + nc + h * 8)));
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) v[h * 8 + i] = apply_act(v[h * 8 + i] + sv.v[i], g.act2);
-                    }
-                } else if (g.act2) {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) v[i] = apply_act(v[i], g.act2);
-                }
                 if (g.out_f32) {
                     float *o = reinterpret_cast<float *>(g.out) + pix * g.out_ctot + g.out_coff + nc;
 #pragma unroll

@@ -1,0 +1,327 @@
+"""Host logic of the C-ABI library, no GPU needed: exported symbols, the call-order state machine,
+error codes, Conv-Bn-Relu pre-fusion, Table 1 pattern matching, split plans (exact covers,
+halos, determinism) and the workspace layout."""
+import ctypes
+import itertools
+import os
+import re
+
+import numpy as np
+import pytest
+
+from paper_2302_00282_b200 import binding as xb
+from xenos_workloads import graphs
+from xenos_workloads.graphs import GraphSpec
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+GOLD = os.path.join(os.path.dirname(__file__), "golden", "link_patterns.txt")
+
+
+def compiled(spec, batch=2, linked=True, splits=(), links=None, hw=None):
+    P = graphs.make_params(spec)
+    g, ids = xb.graph_from_spec(spec, P, hw=hw)
+    if links is not None:
+        for ch in links:
+            g.link([ids[n] for n in ch])
+    elif linked:
+        g.link()
+    for name, kw in splits:
+        g.split(ids[name], **kw)
+    g.compile(batch, xb.PRECISION_FP32_CUDA_CORE if spec.precision == "fp32" else xb.PRECISION_BF16_TENSOR)
+    return g, ids
+
+
+def test_library_exports_every_declared_symbol():
+    hdr = open(os.path.join(ROOT, "include", "xenos.h")).read()
+    declared = sorted(set(re.findall(r"\b(xenos_(?:graph_\w+|last_error))\s*\(", hdr)))
+    assert declared and sorted(xb.EXPORTS) == declared
+    L = xb.lib()
+    for name in declared:
+        assert hasattr(L, name), name
+
+
+def test_state_machine_and_argument_errors():
+    g = xb.Graph()
+    with pytest.raises(xb.XenosError) as e:
+        g.compile(1, xb.PRECISION_BF16_TENSOR)
+    assert e.value.code == xb.E_INVALID                      # no input yet
+    x = g.add_input(xb.DTYPE_F32, xb.LAYOUT_NCHW, 4, 8, 8)
+    w = np.ones((4, 4, 3, 3), np.float32)
+    with pytest.raises(xb.XenosError) as e:
+        g.add_op(xb.OP_CONV, [x], cout=4, k=9, stride=1, pad=0, weight=np.ones((4, 4, 9, 9), np.float32))
+    assert e.value.code == xb.E_SHAPE                        # kernel larger than the input
+    with pytest.raises(xb.XenosError) as e:
+        g.add_op(xb.OP_CONV, [x], cout=4, k=3, weight=None)
+    assert e.value.code == xb.E_INVALID
+    with pytest.raises(xb.XenosError) as e:
+        g.add_op(xb.OP_CONV, [x], cout=4, k=3, groups=2, weight=np.ones((4, 2, 3, 3), np.float32))
+    assert e.value.code == xb.E_UNSUPPORTED                  # grouped but not depthwise
+    with pytest.raises(xb.XenosError) as e:
+        g.add_op(42, [x])
+    assert e.value.code == xb.E_UNSUPPORTED                  # x.mul / x.mac / ... are not implemented
+    with pytest.raises(xb.XenosError) as e:
+        g.add_op(xb.OP_CONV, [99], cout=4, k=3, weight=w)
+    assert e.value.code == xb.E_INVALID
+    y = g.add_op(xb.OP_CONV, [x], cout=4, k=3, stride=1, pad=1, weight=w)
+    z = g.add_op(xb.OP_POOL_MAX, [y], k=2, stride=2)
+    with pytest.raises(xb.XenosError) as e:
+        g.add_op(xb.OP_ADD, [y, z])
+    assert e.value.code == xb.E_SHAPE
+    with pytest.raises(xb.XenosError) as e:
+        g.link([y])
+    assert e.value.code == xb.E_NOT_LINKABLE
+    with pytest.raises(xb.XenosError) as e:
+        g.link([z, y])                                       # not producer -> consumer
+    assert e.value.code == xb.E_NOT_LINKABLE
+    with pytest.raises(xb.XenosError) as e:
+        g.split(y, parts_k=2)
+    assert e.value.code == xb.E_UNSUPPORTED
+    for call in (lambda: g.bind(256, 256), lambda: g.run(1, [1], [1]), lambda: g.plan(), lambda: g.status()):
+        with pytest.raises(xb.XenosError) as e:
+            call()
+        assert e.value.code == xb.E_STATE
+    g.mark_output(z, xb.DTYPE_F32, xb.LAYOUT_NCHW)
+    with pytest.raises(xb.XenosError) as e:
+        g.mark_output(z, xb.DTYPE_F32, xb.LAYOUT_NCHW)
+    assert e.value.code == xb.E_INVALID
+    n = g.compile(3, xb.PRECISION_FP32_CUDA_CORE)
+    assert n > 0
+    for call in (lambda: g.add_input(0, 0, 1, 1, 1), lambda: g.link(), lambda: g.split(-1),
+                 lambda: g.compile(3, 0), lambda: g.run(1, [1], [1])):
+        with pytest.raises(xb.XenosError) as e:
+            call()
+        assert e.value.code == xb.E_STATE
+    with pytest.raises(xb.XenosError) as e:
+        g.bind(0, n)
+    assert e.value.code == xb.E_WORKSPACE
+    with pytest.raises(xb.XenosError) as e:
+        g.bind(4096 + 8, n)                                  # misaligned
+    assert e.value.code == xb.E_WORKSPACE
+    with pytest.raises(xb.XenosError) as e:
+        g.bind(4096, n - 1)
+    assert e.value.code == xb.E_WORKSPACE
+    g.destroy()
+
+
+def test_bind_fails_loudly_without_a_device():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a device is present")
+    g, _ = compiled(graphs.single_chain(), 1)
+    n = g.plan()["workspace_bytes"]
+    with pytest.raises(xb.XenosError) as e:
+        g.bind(1 << 20, max(n, 256))
+    assert e.value.code == xb.E_CUDA
+
+
+def test_prefusion_folds_bn_and_activation():
+    spec = graphs.single_chain()
+    g, _ = compiled(spec, 1, linked=False)
+    pl = g.plan()
+    assert [n["kind"] for n in pl["nodes"]] == ["conv", "conv", "maxpool"]
+    assert [len(n["user_ops"]) for n in pl["nodes"]] == [3, 3, 1]
+    assert [n["act"] for n in pl["nodes"]] == [1, 1, 0]
+    assert len(pl["chains"]) == 3 and all(c["kind"] == "single" for c in pl["chains"])
+
+
+def test_standalone_bn_or_activation_is_rejected():
+    g = xb.Graph()
+    x = g.add_input(xb.DTYPE_F32, xb.LAYOUT_NCHW, 4, 8, 8)
+    p = g.add_op(xb.OP_POOL_MAX, [x], k=2, stride=2)
+    r = g.add_op(xb.OP_RELU, [p])
+    g.mark_output(r, xb.DTYPE_F32, xb.LAYOUT_NCHW)
+    with pytest.raises(xb.XenosError) as e:
+        g.compile(1, xb.PRECISION_FP32_CUDA_CORE)
+    assert e.value.code == xb.E_UNSUPPORTED
+
+
+def _gold_counts():
+    out = {}
+    for line in open(GOLD):
+        if line.strip() and not line.startswith("#"):
+            name, pat, cnt = line.split()
+            out.setdefault(name, {})[pat] = int(cnt)
+    return out
+
+
+def _classify(chain, nodes):
+    kinds = [nodes[i]["kind"] for i in chain["nodes"]]
+    if chain["kind"] == "conv_conv_pool":
+        return "conv-conv-pool"
+    if chain["kind"] == "dw_pw":
+        return "dw-pw"
+    if chain["kind"] == "expand_concat":
+        return "fire"
+    if chain["kind"] == "conv_tail":
+        if "add" in kinds:
+            return "shortcut"
+        return "conv-pool" if "maxpool" in kinds else "conv-gap"
+    return None
+
+
+@pytest.mark.parametrize("name", ["single_chain", "mobilenet_v1", "resnet18", "squeezenet11", "resnet50_stress"])
+def test_table1_patterns_are_found(name):
+    spec = getattr(graphs, name)()
+    g, _ = compiled(spec, 1)
+    pl = g.plan()
+    got = {}
+    for c in pl["chains"]:
+        k = _classify(c, pl["nodes"])
+        if k:
+            got[k] = got.get(k, 0) + 1
+    want = _gold_counts()[name]
+    if name == "mobilenet_v1":        # the last dw -> pw chain also absorbs the global average
+        want = {"dw-pw": 13}
+        assert sum("gap" in [pl["nodes"][i]["kind"] for i in c["nodes"]] for c in pl["chains"]) == 1
+    if name == "squeezenet11":        # 13x13 = 169 rows exceed one 128-row tile: classifier -> gap stays unlinked
+        want = {k: v for k, v in want.items() if k != "conv-gap"}
+    assert got == want
+    # every node is in exactly one chain; chains run after their producers
+    seen = sorted(i for c in pl["chains"] for i in c["nodes"])
+    assert seen == list(range(len(pl["nodes"])))
+    produced = set(t["id"] for t in pl["tensors"] if t["external"])
+    for L in pl["launches"]:
+        for t in (L["in0"], L["in1"], L["skip"]):
+            assert t < 0 or t in produced, (L["id"], t)
+        produced.add(L["out"])
+
+
+def test_producer_with_two_unrelated_consumers_is_not_linked():
+    g = GraphSpec("fork", (16, 12, 12))
+    a = g.cbr("a", "input", 16, 3, 1, 1)
+    p = g.pool("p", a, "maxpool", 2, 2)
+    q = g.cbr("q", a, 16, 1)          # second consumer of a
+    g.pool("q.p", q, "maxpool", 2, 2)
+    g.output = "p"
+    gg, _ = compiled(g, 1)
+    pl = gg.plan()
+    chain_of = {n["id"]: n["chain"] for n in pl["nodes"]}
+    assert pl["chains"][chain_of[0]]["kind"] == "single"     # a -> {p, q}: a stays alone
+
+
+def test_explicit_link_requests():
+    spec = graphs.mobilenet_v1(hw=32, width=0.25, classes=8)
+    g, _ = compiled(spec, 1, links=[["dw1", "pw1"], ["dw13", "pw13", "gap"]])
+    pl = g.plan()
+    linked = [c for c in pl["chains"] if c["kind"] != "single"]
+    assert len(linked) == 2 and [len(c["nodes"]) for c in linked] == [2, 3]
+    with pytest.raises(xb.XenosError) as e:
+        compiled(spec, 1, links=[["pw1", "dw2"]])            # adjacent, but no pattern with a kernel
+    assert e.value.code == xb.E_NOT_LINKABLE
+    with pytest.raises(xb.XenosError) as e:
+        compiled(spec, 1, links=[["dw1", "pw1"], ["dw1", "pw1"]])
+    assert e.value.code == xb.E_NOT_LINKABLE
+
+
+def test_plans_are_deterministic():
+    for spec in (graphs.single_chain(), graphs.resnet18(hw=64, base=16, classes=8)):
+        a, _ = compiled(spec, 4)
+        b, _ = compiled(spec, 4)
+        assert a.plan_text() == b.plan_text()
+
+
+@pytest.mark.parametrize("split", [dict(), dict(parts_outc=4, parts_h=2, parts_w=1), dict(parts_outc=2, parts_h=4, parts_w=8),
+                                   dict(parts_h=16, parts_w=16), dict(parts_outc=32)])
+def test_fp32_chain_split_is_an_exact_cover_with_correct_halo(split):
+    spec = graphs.single_chain()
+    g, _ = compiled(spec, 1, splits=[("mp", split)] if split else ())
+    L = g.plan()["launches"][0]
+    assert L["kind"] == "f32_conv_conv_pool"
+    PP = PQ = 16
+    if split.get("parts_outc"):
+        assert L["parts_outc"] == split["parts_outc"]
+    if split.get("parts_h"):
+        assert L["tiles_h"] == split["parts_h"] and L["tiles_w"] == split.get("parts_w", L["tiles_w"])
+    cover = np.zeros((32, PP, PQ), int)
+    kper = 32 // L["parts_outc"]
+    for part, ty, tx in itertools.product(range(L["parts_outc"]), range(L["tiles_h"]), range(L["tiles_w"])):
+        y0, x0 = ty * L["tile_h"], tx * L["tile_w"]
+        cover[part * kper:(part + 1) * kper, y0:min(PP, y0 + L["tile_h"]), x0:min(PQ, x0 + L["tile_w"])] += 1
+    assert (cover == 1).all()                                 # disjoint and complete
+    assert L["grid"] == L["parts_outc"] * L["tiles_h"] * L["tiles_w"]
+    # halo: rows / columns of the first conv's output a full tile reads (pool 2x2 s2 over a 1x1 conv)
+    assert (L["halo_h"], L["halo_w"]) == (2 * L["tile_h"], 2 * L["tile_w"])
+
+
+def test_bad_splits_are_rejected():
+    spec = graphs.single_chain()
+    for kw in (dict(parts_outc=5), dict(parts_h=17), dict(parts_w=64), dict(parts_outc=64)):
+        with pytest.raises(xb.XenosError) as e:
+            compiled(spec, 1, splits=[("mp", kw)])
+        assert e.value.code == xb.E_BAD_SPLIT, kw
+    m = graphs.mobilenet_v1(hw=32, width=0.25, classes=8)
+    with pytest.raises(xb.XenosError) as e:
+        compiled(m, 1, splits=[("pw1.relu6", dict(parts_h=2))])
+    assert e.value.code == xb.E_BAD_SPLIT
+
+
+def test_gemm_split_prefers_output_channels_until_units_are_busy():
+    """Section 4.2.1: kernels are dealt to the units first; rows / columns follow."""
+    spec = graphs.mobilenet_v1()
+    for batch in (1, 32):
+        g, _ = compiled(spec, batch)
+        for L in g.plan()["launches"]:
+            if L["kind"] != "gemm":
+                continue
+            assert L["tile_n"] % 16 == 0 and 16 <= L["tile_n"] <= 256
+            assert L["npad"] == L["tile_n"] * L["n_tiles"] and (L["n_tiles"] - 1) * L["tile_n"] < L["K"] <= L["npad"]
+            assert L["grid"] == L["m_tiles"] * L["n_tiles"]
+            if L["n_tiles"] > -(-L["K"] // 256):               # split finer than the 256-wide maximum
+                assert L["m_tiles"] * (L["n_tiles"] // 2) < 148   # ... only because units would idle otherwise
+            assert L["tmem_cols"] >= L["tile_n"] and L["stages"] >= 2
+            assert L["smem_bytes"] <= 227 * 1024
+    g, ids = compiled(spec, 32, splits=[("pw7.relu6", dict(parts_outc=4))])
+    L = [l for l in g.plan()["launches"] if l["kind"] == "gemm" and l["K"] == 512][1]
+    hw = xb.HwInfo(16, 227 * 1024, 512, 1 << 20)
+    g2, _ = compiled(spec, 1, hw=hw)
+    assert g2.plan()["hw"]["sm_count"] == 16
+
+
+def test_user_outc_split_sets_tiles():
+    spec = graphs.mobilenet_v1()
+    g, ids = compiled(spec, 32, splits=[("pw7.relu6", dict(parts_outc=4))])
+    pl = g.plan()
+    node = [n for n in pl["nodes"] if n["out"] == ids["pw7.relu6"]][0]
+    L = pl["launches"][pl["chains"][node["chain"]]["launches"][0]]
+    assert (L["n_tiles"], L["tile_n"]) == (4, 128)
+
+
+def test_pool_patch_tiles_cover_pool_output():
+    spec = graphs.resnet18()
+    g, _ = compiled(spec, 2)
+    L = [l for l in g.plan()["launches"] if l["kind"] == "gemm" and l["epi"] == 2][0]
+    assert L["patch_rh"] == (L["patch_th"] - 1) * 2 + 3 and L["patch_rw"] == (L["patch_tw"] - 1) * 2 + 3
+    assert L["patch_rh"] * L["patch_rw"] <= 128
+    assert L["tiles_y"] * L["patch_th"] >= 56 > (L["tiles_y"] - 1) * L["patch_th"]
+    assert L["tiles_x"] * L["patch_tw"] >= 56 > (L["tiles_x"] - 1) * L["patch_tw"]
+    assert L["m_tiles"] == 2 * L["tiles_y"] * L["tiles_x"]
+
+
+@pytest.mark.parametrize("name,kw", [("mobilenet_v1", {}), ("resnet18", {}), ("squeezenet11", {}),
+                                     ("resnet50_stress", dict(hw=128))])
+@pytest.mark.parametrize("linked", [True, False])
+def test_workspace_tensors_never_overlap_while_live(name, kw, linked):
+    spec = getattr(graphs, name)(**kw)
+    g, _ = compiled(spec, 2, linked=linked)
+    pl = g.plan()
+    ts = [t for t in pl["tensors"] if not t["external"]]
+    for a, b in itertools.combinations(ts, 2):
+        live = not (a["last"] < b["first"] or b["last"] < a["first"])
+        mem = not (a["off"] + a["bytes"] <= b["off"] or b["off"] + b["bytes"] <= a["off"])
+        assert not (live and mem), (a, b)
+    for t in ts:
+        assert t["off"] >= pl["param_bytes"] and t["off"] + t["bytes"] <= pl["workspace_bytes"] and t["off"] % 256 == 0
+    # linking removes intermediates from memory
+    if linked:
+        gu, _ = compiled(spec, 2, linked=False)
+        assert pl["bytes_linked"] < gu.plan()["bytes_linked"]
+        assert len(pl["launches"]) < len(gu.plan()["launches"])
+
+
+def test_modelled_work_matches_shapes():
+    spec = graphs.mobilenet_v1()
+    g, _ = compiled(spec, 32)
+    pl = g.plan()
+    assert pl["flops"] == 2 * 32 * spec.macs()
+    # depthwise-separable chains dominate the saving: linked bytes are well below unlinked ones
+    assert pl["bytes_linked"] < 0.7 * pl["bytes_unlinked"]
