@@ -4,7 +4,7 @@
 // (the operator split of Section 4.2: output channels first, then rows / columns).
 //   warp 0      : TMA producer for the weight tile (cp.async.bulk.tensor, 128-byte swizzle)
 //   warp 1      : allocates tensor memory, one lane issues tcgen05.mma (bf16 x bf16 -> fp32)
-//   warps 2..5  : produce the activation operand straight into shared memory in the layout the
+//   warps 2..9  : produce the activation operand straight into shared memory in the layout the
 //                 tensor core reads (K-major, 128-byte swizzle) - the paper's "write in the
 //                 order the next operator reads" (Section 4.1) - then run the epilogue
 // The activation operand of one 64-wide K block comes from one of
@@ -56,7 +56,7 @@ struct GemmParams {
     int batch, P, Q, rpi;
     int map_mode, tile_rows, imgs_per_tile;
     int th, tw, rh, rw, tiles_y, tiles_x, pool_k, pool_stride, pool_pad, PP, PQ;
-    int kblocks, stages, tile_n, n_tiles, N;
+    int kblocks, stages, tile_n, n_tiles, N, pipe_bytes;
     int act, act2, epi, out_ctot, out_coff, out_f32, skip_ctot;
     uint32_t idesc;
 };
@@ -146,7 +146,9 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float *v) {
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+constexpr int kProducerThreads = 256;           // warps 2..9
+constexpr int kThreads = 64 + kProducerThreads;
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 // ---- row <-> pixel -----------------------------------------------------------------------------
 struct RowPos { int valid, n, p, q; };
@@ -175,111 +177,180 @@ __device__ __forceinline__ RowPos map_row(const GemmParams &g, int mt, int r) {
     return o;
 }
 
-// ---- A-operand producers: each of the 128 producer threads fills one row (128 bytes) of the stage
+// ---- A-operand producers ------------------------------------------------------------------------
+// A stage is 128 rows x 128 bytes; 16-byte chunk j of row r sits at r*128 + ((j ^ (r & 7)) << 4),
+// which is what a 128-byte-swizzle TMA load would have written and what the MMA descriptor expects.
 __device__ __forceinline__ uint32_t a_chunk_addr(uint32_t a_base, int row, int j) {
     return a_base + row * 128 + ((j ^ (row & 7)) << 4);
 }
 
-struct GatherState { int tap_r, tap_s, cc; };   // position of the next 8-channel chunk inside the segment
+// One lane polls, the warp follows: keeps 32x fewer pollers on the barrier word.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, int lane) {
+    int ok = 1;
+    if (lane == 0) ok = mbar_wait(bar, parity) ? 1 : 0;
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    return ok != 0;
+}
+// Every lane has fenced its own writes; one arrival per warp.
+__device__ __forceinline__ void warp_arrive(uint32_t bar, int lane) {
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar);
+}
 
-__device__ __forceinline__ void produce_gather(const GemmSeg &sg, GatherState &st, const RowPos &rp, uint32_t a_base, int row) {
-    const __nv_bfloat16 *src = reinterpret_cast<const __nv_bfloat16 *>(sg.src);
-    int C8 = sg.C >> 3;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const void *ptr = src;
-        uint32_t bytes = 0;
-        if (rp.valid && st.tap_r < sg.k) {
-            int ih = rp.p * sg.stride - sg.pad + st.tap_r, iw = rp.q * sg.stride - sg.pad + st.tap_s;
-            if (ih >= 0 && ih < sg.H && iw >= 0 && iw < sg.W) {
-                ptr = src + (((size_t)rp.n * sg.H + ih) * sg.W + iw) * sg.C + st.cc * 8;
-                bytes = 16;
-            }
-        }
-        cp_async16(a_chunk_addr(a_base, row, j), ptr, bytes);
-        if (st.tap_r < sg.k && ++st.cc == C8) {
-            st.cc = 0;
-            if (++st.tap_s == sg.k) { st.tap_s = 0; ++st.tap_r; }
-        }
+struct GatherState { int tap_r, tap_s, cc; };   // (tap, channel chunk) of a thread's next 8-channel chunk
+
+__device__ __forceinline__ void gather_advance(GatherState &st, int n, int C8, int k) {
+    if (st.tap_r >= k) return;
+    st.cc += n;
+    while (st.cc >= C8 && st.tap_r < k) {
+        st.cc -= C8;
+        if (++st.tap_s == k) { st.tap_s = 0; ++st.tap_r; }
     }
 }
 
-// K order of the stem: element e = (r * k + s) * C + c of an NCHW image, fp32 or bf16.
-__device__ __forceinline__ void produce_stem(const GemmSeg &sg, int kb_local, const RowPos &rp, uint32_t a_base, int row) {
-    int e = kb_local * kTileK;
+// gather: thread = (row, half); it copies chunks 4*half .. 4*half+3 of its row with 16-byte cp.async
+__device__ __forceinline__ void produce_gather(const GemmSeg &sg, GatherState st, const int4 ri, uint32_t a_base,
+                                               int row, int half) {
+    const __nv_bfloat16 *src = reinterpret_cast<const __nv_bfloat16 *>(sg.src);
+    const int C8 = sg.C >> 3;
+    const int ih0 = ri.z * sg.stride - sg.pad, iw0 = ri.w * sg.stride - sg.pad;
+    const __nv_bfloat16 *img = src + (size_t)ri.y * sg.H * sg.W * sg.C;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const void *ptr = src;
+        uint32_t bytes = 0;
+        if (ri.x && st.tap_r < sg.k) {
+            int ih = ih0 + st.tap_r, iw = iw0 + st.tap_s;
+            if (ih >= 0 && ih < sg.H && iw >= 0 && iw < sg.W) {
+                ptr = img + ((size_t)ih * sg.W + iw) * sg.C + st.cc * 8;
+                bytes = 16;
+            }
+        }
+        cp_async16(a_chunk_addr(a_base, row, half * 4 + i), ptr, bytes);
+        gather_advance(st, 1, C8, sg.k);
+    }
+}
+
+// stem: K element e = (r * k + s) * C + c of an NCHW image (fp32 or bf16); thread = (row, half)
+__device__ __forceinline__ void produce_stem(const GemmSeg &sg, int kb_local, const int4 ri, uint32_t a_base,
+                                             int row, int half) {
+    int e = kb_local * kTileK + half * 32;
     int tap = e / sg.C, c = e - tap * sg.C;
     int r = tap / sg.k, s = tap - r * sg.k;
+    const int ih0 = ri.z * sg.stride - sg.pad, iw0 = ri.w * sg.stride - sg.pad;
+    const size_t img = (size_t)ri.y * sg.C * sg.H * sg.W;
+    const float *sf = reinterpret_cast<const float *>(sg.src) + img;
+    const __nv_bfloat16 *sh = reinterpret_cast<const __nv_bfloat16 *>(sg.src) + img;
 #pragma unroll 1
-    for (int j = 0; j < 8; ++j) {
+    for (int j = 0; j < 4; ++j) {
         f8 v;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             float x = 0.0f;
-            if (rp.valid && r < sg.k) {
-                int ih = rp.p * sg.stride - sg.pad + r, iw = rp.q * sg.stride - sg.pad + s;
+            if (ri.x && r < sg.k) {
+                int ih = ih0 + r, iw = iw0 + s;
                 if (ih >= 0 && ih < sg.H && iw >= 0 && iw < sg.W) {
-                    size_t idx = (((size_t)rp.n * sg.C + c) * sg.H + ih) * sg.W + iw;
-                    x = sg.src_f32 ? reinterpret_cast<const float *>(sg.src)[idx]
-                                   : __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(sg.src)[idx]);
+                    int off = (c * sg.H + ih) * sg.W + iw;
+                    x = sg.src_f32 ? __ldg(sf + off) : __bfloat162float(sh[off]);
                 }
             }
             v.v[i] = x;
             if (++c == sg.C) { c = 0; if (++s == sg.k) { s = 0; ++r; } }
         }
-        st_shared16(a_chunk_addr(a_base, row, j), pack8(v));
+        st_shared16(a_chunk_addr(a_base, row, half * 4 + j), pack8(v));
     }
 }
 
-// Depthwise 3x3 + bias + activation for 64 channels of one output pixel, rounded to bf16.
-__device__ __forceinline__ void produce_dw(const GemmSeg &sg, int kb_local, const RowPos &rp, uint32_t a_base, int row) {
-    const __nv_bfloat16 *src = reinterpret_cast<const __nv_bfloat16 *>(sg.src);
-#pragma unroll 1
-    for (int j = 0; j < 8; ++j) {
-        int c0 = kb_local * kTileK + j * 8;
-        uint4 outv = make_uint4(0u, 0u, 0u, 0u);
-        if (rp.valid && c0 < sg.C) {
-            f8 acc;
-            const float4 b0 = *reinterpret_cast<const float4 *>(sg.dw_b + c0), b1 = *reinterpret_cast<const float4 *>(sg.dw_b + c0 + 4);
-            acc.v[0] = b0.x; acc.v[1] = b0.y; acc.v[2] = b0.z; acc.v[3] = b0.w;
-            acc.v[4] = b1.x; acc.v[5] = b1.y; acc.v[6] = b1.z; acc.v[7] = b1.w;
+// depthwise 3x3 + bias + activation, rounded to bf16 and stored in the consumer's operand layout.
+// thread = (chunk j of 8 channels, row group); it owns rows rg, rg+32, rg+64, rg+96 so that the
+// nine tap weights of its 8 channels are fetched once per K block and four independent pixel
+// loads are in flight per tap.
+struct DwRows { long long base[4]; unsigned mask[4]; };
+
+__device__ __forceinline__ void dw_rows_init(const GemmSeg &sg, const int4 *rowtab, int rg, DwRows &dr) {
 #pragma unroll
-            for (int r = 0; r < 3; ++r) {
-                int ih = rp.p * sg.stride - sg.pad + r;
-                if (ih < 0 || ih >= sg.H) continue;
+    for (int i = 0; i < 4; ++i) {
+        const int4 ri = rowtab[rg + 32 * i];
+        int ih0 = ri.z * sg.stride - sg.pad, iw0 = ri.w * sg.stride - sg.pad;
+        unsigned m = 0;
+        if (ri.x) {
 #pragma unroll
-                for (int s = 0; s < 3; ++s) {
-                    int iw = rp.q * sg.stride - sg.pad + s;
-                    if (iw < 0 || iw >= sg.W) continue;
-                    f8 xv = unpack8(__ldg(reinterpret_cast<const uint4 *>(src + (((size_t)rp.n * sg.H + ih) * sg.W + iw) * sg.C + c0)));
-                    const float *wt = sg.dw_w + (size_t)(r * 3 + s) * sg.C + c0;
-                    const float4 w0 = __ldg(reinterpret_cast<const float4 *>(wt)), w1 = __ldg(reinterpret_cast<const float4 *>(wt + 4));
-                    acc.v[0] = fmaf(xv.v[0], w0.x, acc.v[0]); acc.v[1] = fmaf(xv.v[1], w0.y, acc.v[1]);
-                    acc.v[2] = fmaf(xv.v[2], w0.z, acc.v[2]); acc.v[3] = fmaf(xv.v[3], w0.w, acc.v[3]);
-                    acc.v[4] = fmaf(xv.v[4], w1.x, acc.v[4]); acc.v[5] = fmaf(xv.v[5], w1.y, acc.v[5]);
-                    acc.v[6] = fmaf(xv.v[6], w1.z, acc.v[6]); acc.v[7] = fmaf(xv.v[7], w1.w, acc.v[7]);
-                }
-            }
+            for (int r = 0; r < 3; ++r)
 #pragma unroll
-            for (int i = 0; i < 8; ++i) acc.v[i] = apply_act(acc.v[i], sg.dw_act);
-            outv = pack8(acc);
+                for (int s = 0; s < 3; ++s)
+                    if (ih0 + r >= 0 && ih0 + r < sg.H && iw0 + s >= 0 && iw0 + s < sg.W) m |= 1u << (r * 3 + s);
         }
-        st_shared16(a_chunk_addr(a_base, row, j), outv);
+        if (ri.x) m |= 1u << 9;        // bit 9: the row is a real output pixel
+        dr.mask[i] = m;
+        dr.base[i] = (((long long)ri.y * sg.H + ih0) * sg.W + iw0) * sg.C;
+    }
+}
+
+__device__ __forceinline__ void produce_dw(const GemmSeg &sg, int kb_local, const DwRows &dr, uint32_t a_base, int j, int rg) {
+    const int c0 = kb_local * kTileK + j * 8;
+    if (c0 >= sg.C) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) st_shared16(a_chunk_addr(a_base, rg + 32 * i, j), make_uint4(0u, 0u, 0u, 0u));
+        return;
+    }
+    const __nv_bfloat16 *src = reinterpret_cast<const __nv_bfloat16 *>(sg.src) + c0;
+    float acc[4][8];
+    {
+        const float4 b0 = __ldg(reinterpret_cast<const float4 *>(sg.dw_b + c0)), b1 = __ldg(reinterpret_cast<const float4 *>(sg.dw_b + c0 + 4));
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            acc[i][0] = b0.x; acc[i][1] = b0.y; acc[i][2] = b0.z; acc[i][3] = b0.w;
+            acc[i][4] = b1.x; acc[i][5] = b1.y; acc[i][6] = b1.z; acc[i][7] = b1.w;
+        }
+    }
+#pragma unroll
+    for (int t = 0; t < 9; ++t) {
+        const float *wt = sg.dw_w + (size_t)t * sg.C + c0;
+        const float4 w0 = __ldg(reinterpret_cast<const float4 *>(wt)), w1 = __ldg(reinterpret_cast<const float4 *>(wt + 4));
+        const int toff = ((t / 3) * sg.W + (t % 3)) * sg.C;
+        uint4 xv[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            xv[i] = make_uint4(0u, 0u, 0u, 0u);
+            if (dr.mask[i] & (1u << t)) xv[i] = __ldg(reinterpret_cast<const uint4 *>(src + dr.base[i] + toff));
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const f8 x = unpack8(xv[i]);
+            acc[i][0] = fmaf(x.v[0], w0.x, acc[i][0]); acc[i][1] = fmaf(x.v[1], w0.y, acc[i][1]);
+            acc[i][2] = fmaf(x.v[2], w0.z, acc[i][2]); acc[i][3] = fmaf(x.v[3], w0.w, acc[i][3]);
+            acc[i][4] = fmaf(x.v[4], w1.x, acc[i][4]); acc[i][5] = fmaf(x.v[5], w1.y, acc[i][5]);
+            acc[i][6] = fmaf(x.v[6], w1.z, acc[i][6]); acc[i][7] = fmaf(x.v[7], w1.w, acc[i][7]);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        uint4 o = make_uint4(0u, 0u, 0u, 0u);
+        if (dr.mask[i]) {
+            f8 r;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) r.v[c] = apply_act(acc[i][c], sg.dw_act);
+            o = pack8(r);
+        }
+        st_shared16(a_chunk_addr(a_base, rg + 32 * i, j), o);
     }
 }
 
 // ---- the kernel --------------------------------------------------------------------------------
-__global__ void __launch_bounds__(192) gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const GemmParams g) {
+// Shared memory: [stages x (A 16 KB | B tile_n x 128 B)] [staging, if larger] [barriers] [row table]
+__global__ void __launch_bounds__(kThreads, 2) gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const GemmParams g) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t sbase = (raw + 1023u) & ~1023u;
     uint8_t *sm = smem_raw + (sbase - raw);
     const int stage_bytes = kABytes + g.tile_n * 128;
-    const uint32_t bar_base = sbase + g.stages * stage_bytes;
+    const int pipe_bytes = g.pipe_bytes;            // >= stages * stage_bytes and >= the epilogue staging need
+    const uint32_t bar_base = sbase + pipe_bytes;
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto empty_bar = [&](int s) { return bar_base + 8u * (kMaxStages + s); };
     const uint32_t accum_bar = bar_base + 8u * (2 * kMaxStages);
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(sm + g.stages * stage_bytes + 8 * (2 * kMaxStages + 1));
-    int *abort_flag = reinterpret_cast<int *>(tmem_slot + 1);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(sm + pipe_bytes + 8 * (2 * kMaxStages + 1));
+    int4 *rowtab = reinterpret_cast<int4 *>(sm + pipe_bytes + 128);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int mt = blockIdx.x / g.n_tiles, nt = blockIdx.x - mt * g.n_tiles;
@@ -287,15 +358,18 @@ __global__ void __launch_bounds__(192) gemm_chain_kernel(const __grid_constant__
     while ((int)tmem_cols < g.tile_n) tmem_cols <<= 1;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < g.stages; ++s) { mbar_init(full_bar(s), 128 + 1); mbar_init(empty_bar(s), 1); }
+        for (int s = 0; s < g.stages; ++s) { mbar_init(full_bar(s), kProducerThreads / 32 + 1); mbar_init(empty_bar(s), 1); }
         mbar_init(accum_bar, 1);
-        *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (threadIdx.x >= 64 && threadIdx.x < 64 + kTileM) {
+        const RowPos rp = map_row(g, mt, threadIdx.x - 64);
+        rowtab[threadIdx.x - 64] = make_int4(rp.valid, rp.n, rp.p, rp.q);
     }
     tc_fence_before();
     __syncthreads();
@@ -314,7 +388,7 @@ __global__ void __launch_bounds__(192) gemm_chain_kernel(const __grid_constant__
                 mbar_arrive_expect_tx(full_bar(s), (uint32_t)g.tile_n * 128u);
                 tma_load_2d(sbase + s * stage_bytes + kABytes, &tmB, kb * kTileK, nt * g.tile_n, full_bar(s));
             }
-            if (!ok) { atomicCAS(g.status, 0u, kStatusTimeout); atomicExch(abort_flag, 1); }
+            if (!ok) atomicCAS(g.status, 0u, kStatusTimeout);
         }
     } else if (warp == 1) {
         // ---- MMA issue ----
@@ -333,94 +407,107 @@ __global__ void __launch_bounds__(192) gemm_chain_kernel(const __grid_constant__
                 umma_commit(empty_bar(s));
             }
             if (ok) umma_commit(accum_bar);
-            else { atomicCAS(g.status, 0u, kStatusTimeout); atomicExch(abort_flag, 1); }
+            else atomicCAS(g.status, 0u, kStatusTimeout);
         }
     } else {
         // ---- activation operand, then epilogue ----
-        const int row = (warp & 3) * 32 + lane;          // also the tensor-memory lane this thread reads
-        const RowPos rp = map_row(g, mt, row);
-        GatherState gs[2] = {{0, 0, 0}, {0, 0, 0}};
-        const int lag = g.stages >= 3 ? 2 : 1;
+        const int pt = threadIdx.x - 64;                 // 0..255
+        const int grow = pt & 127, ghalf = pt >> 7;      // gather / stem mapping
+        const int dj = pt & 7, drg = pt >> 3;            // depthwise mapping
+        const int4 ri = rowtab[grow];
+        GatherState gs0 = {0, 0, 0}, gs1 = {0, 0, 0};
+        if (g.seg[0].mode == GA_GATHER && ghalf) gather_advance(gs0, 4, g.seg[0].C >> 3, g.seg[0].k);
+        if (g.seg[1].mode == GA_GATHER && ghalf) gather_advance(gs1, 4, g.seg[1].C >> 3, g.seg[1].k);
+        DwRows dr;
+        if (g.seg[0].mode == GA_DW) dw_rows_init(g.seg[0], rowtab, drg, dr);
+        const int lag = g.stages >= 3 ? 2 : (g.stages == 2 ? 1 : 0);
         int pend = 0, pend_first = 0;
         auto retire_oldest = [&]() {
             fence_proxy_async();
-            mbar_arrive(full_bar(pend_first % g.stages));
+            warp_arrive(full_bar(pend_first % g.stages), lane);
             ++pend_first; --pend;
         };
         for (int kb = 0; kb < g.kblocks && ok; ++kb) {
             int s = kb % g.stages;
             uint32_t ph = (kb / g.stages) & 1;
-            ok = mbar_wait(empty_bar(s), ph ^ 1u);
+            ok = mbar_wait_warp(empty_bar(s), ph ^ 1u, lane);
             if (!ok) break;
-            int si = kb < g.seg[0].kblocks ? 0 : 1;
-            int kbl = kb - (si ? g.seg[0].kblocks : 0);
-            const GemmSeg &sg = g.seg[si];
+            const bool first = kb < g.seg[0].kblocks;
+            const GemmSeg &sg = first ? g.seg[0] : g.seg[1];
+            const int kbl = first ? kb : kb - g.seg[0].kblocks;
             uint32_t a_base = sbase + s * stage_bytes;
             if (sg.mode == GA_GATHER) {
-                produce_gather(sg, gs[si], rp, a_base, row);
+                if (first) { produce_gather(sg, gs0, ri, a_base, grow, ghalf); gather_advance(gs0, 8, sg.C >> 3, sg.k); }
+                else { produce_gather(sg, gs1, ri, a_base, grow, ghalf); gather_advance(gs1, 8, sg.C >> 3, sg.k); }
                 cp_async_commit();
                 ++pend;
                 if (pend > lag) {
-                    if (lag == 2) cp_async_wait<2>(); else cp_async_wait<1>();
+                    if (lag == 2) cp_async_wait<2>(); else if (lag == 1) cp_async_wait<1>(); else cp_async_wait<0>();
                     retire_oldest();
                 }
             } else {
                 if (pend) { cp_async_wait<0>(); while (pend) retire_oldest(); }
                 pend_first = kb + 1;
-                if (sg.mode == GA_DW) produce_dw(sg, kbl, rp, a_base, row);
-                else produce_stem(sg, kbl, rp, a_base, row);
+                if (sg.mode == GA_DW) produce_dw(sg, kbl, dr, a_base, dj, drg);
+                else produce_stem(sg, kbl, ri, a_base, grow, ghalf);
                 fence_proxy_async();
-                mbar_arrive(full_bar(s));
+                warp_arrive(full_bar(s), lane);
             }
         }
         cp_async_wait<0>();
         if (ok) { while (pend) retire_oldest(); }
-        else if (lane == 0) { atomicCAS(g.status, 0u, kStatusTimeout); atomicExch(abort_flag, 1); }
+        else if (lane == 0) atomicCAS(g.status, 0u, kStatusTimeout);
 
-        // ---- epilogue ----
-        if (ok) ok = mbar_wait(accum_bar, 0);
-        ok = __all_sync(0xffffffffu, ok);     // warp-uniform from here on (tcgen05.ld is warp-collective)
-        if (!ok && lane == 0) { atomicCAS(g.status, 0u, kStatusTimeout); atomicExch(abort_flag, 1); }
+        // ---- epilogue: warp w reads tensor-memory lanes 32*(w%4).., the two warps that share a
+        // lane quarter take alternate 16-column chunks ----
+        if (ok) ok = mbar_wait_warp(accum_bar, 0, lane);
+        if (!ok && lane == 0) atomicCAS(g.status, 0u, kStatusTimeout);
         tc_fence_after();
-        const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+        const int quarter = warp & 3, chalf = (warp - 2) >> 2;
+        const int row = quarter * 32 + lane;
+        const int4 rq = rowtab[row];
+        const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
         const int n0 = nt * g.tile_n;
         const int nchunks = g.tile_n / 16;
-        // staging area for the pool / global-average epilogues reuses the pipeline buffers: every
-        // MMA has retired (accum barrier) so nothing reads or writes them any more
+        // staging for the pool / global-average epilogues reuses the pipeline buffers: every MMA has
+        // retired (accum barrier), so nothing reads or writes them any more
         const uint32_t stg = sbase;
         const int pool_pitch = g.tile_n * 2 + 16;
-        for (int ch = 0; ch < nchunks; ++ch) {
+        const size_t pix = ((size_t)rq.y * g.P + rq.z) * g.Q + rq.w;
+        for (int c2 = 0; c2 * 2 < nchunks; ++c2) {
+            const int ch = c2 * 2 + chalf;
+            const bool live = ch < nchunks;
             float v[16];
-            if (ok) tmem_ld16(t_lane + ch * 16, v);
+            if (ok && live) tmem_ld16(t_lane + ch * 16, v);
             else {
 #pragma unroll
                 for (int i = 0; i < 16; ++i) v[i] = 0.0f;
             }
             const int nc = n0 + ch * 16;
+            if (live) {
 #pragma unroll
-            for (int i = 0; i < 16; i += 4) {
-                float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (nc + i < g.N) b = __ldg(reinterpret_cast<const float4 *>(g.bias + nc + i));
-                v[i] = apply_act(v[i] + b.x, g.act); v[i + 1] = apply_act(v[i + 1] + b.y, g.act);
-                v[i + 2] = apply_act(v[i + 2] + b.z, g.act); v[i + 3] = apply_act(v[i + 3] + b.w, g.act);
-            }
-            // shortcut connection with an identity branch: the skip tile is read once, here
-            const size_t pix = ((size_t)rp.n * g.P + rp.p) * g.Q + rp.q;
-            if (g.skip && rp.valid) {
+                for (int i = 0; i < 16; i += 4) {
+                    const float4 b = __ldg(reinterpret_cast<const float4 *>(g.bias + nc + i));   // bias is padded to npad
+                    v[i] = apply_act(v[i] + b.x, g.act); v[i + 1] = apply_act(v[i + 1] + b.y, g.act);
+                    v[i + 2] = apply_act(v[i + 2] + b.z, g.act); v[i + 3] = apply_act(v[i + 3] + b.w, g.act);
+                }
+                // shortcut connection with an identity branch: the skip tile is read once, here
+                if (g.skip && rq.x) {
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    if (nc + h * 8 + 8 > g.N) break;
-                    f8 sv = unpack8(__ldg(reinterpret_cast<const uint4 *>(g.skip + pix * g.skip_ctot + nc + h * 8)));
+                    for (int h = 0; h < 2; ++h) {
+                        if (nc + h * 8 + 8 > g.N) break;
+                        f8 sv = unpack8(__ldg(reinterpret_cast<const uint4 *>(g.skip + pix * g.skip_ctot + nc + h * 8)));
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) v[h * 8 + i] += sv.v[i];
+                        for (int i = 0; i < 8; ++i) v[h * 8 + i] += sv.v[i];
+                    }
+                }
+                if (g.act2) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) v[i] = apply_act(v[i], g.act2);
                 }
             }
-            if (g.act2) {
-#pragma unroll
-                for (int i = 0; i < 16; ++i) v[i] = apply_act(v[i], g.act2);
-            }
             if (g.epi == GE_STORE) {
-                if (!rp.valid || !ok) continue;
+                if (!rq.x || !ok || !live) continue;
                 if (g.out_f32) {
                     float *o = reinterpret_cast<float *>(g.out) + pix * g.out_ctot + g.out_coff + nc;
 #pragma unroll
@@ -437,28 +524,30 @@ __global__ void __launch_bounds__(192) gemm_chain_kernel(const __grid_constant__
                     }
                 }
             } else if (g.epi == GE_POOL) {
+                if (!live) continue;
                 // rows outside the conv output never win a max
                 f8 lo, hi;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) { lo.v[i] = rp.valid ? v[i] : -INFINITY; hi.v[i] = rp.valid ? v[8 + i] : -INFINITY; }
+                for (int i = 0; i < 8; ++i) { lo.v[i] = rq.x ? v[i] : -INFINITY; hi.v[i] = rq.x ? v[8 + i] : -INFINITY; }
                 st_shared16(stg + row * pool_pitch + ch * 32, pack8(lo));
                 st_shared16(stg + row * pool_pitch + ch * 32 + 16, pack8(hi));
             } else {
-                // global average: 16 columns at a time through shared memory, rows summed in ascending order
+                // global average: two 16-column chunks at a time through shared memory, rows summed in ascending order
                 epi_bar();
-                float *sf = reinterpret_cast<float *>(sm);
+                float *sf = reinterpret_cast<float *>(sm) + chalf * (kTileM * 17);
 #pragma unroll
-                for (int i = 0; i < 16; ++i) sf[row * 17 + i] = rp.valid ? v[i] : 0.0f;
+                for (int i = 0; i < 16; ++i) sf[row * 17 + i] = (rq.x && live) ? v[i] : 0.0f;
                 epi_bar();
-                int t = threadIdx.x - 64;
-                for (int item = t; item < g.imgs_per_tile * 16; item += 128) {
-                    int img = item >> 4, c = item & 15;
-                    int n = mt * g.imgs_per_tile + img;
-                    if (n >= g.batch || nc + c >= g.N || !ok) continue;
+                for (int item = threadIdx.x - 64; item < g.imgs_per_tile * 32; item += kProducerThreads) {
+                    const int img = item >> 5, c = item & 31;
+                    const int n = mt * g.imgs_per_tile + img;
+                    const int col = n0 + c2 * 32 + c;
+                    if (n >= g.batch || col >= g.N || c2 * 2 + (c >> 4) >= nchunks || !ok) continue;
+                    const float *sc = reinterpret_cast<float *>(sm) + (c >> 4) * (kTileM * 17) + (c & 15);
                     float acc = 0.0f;
-                    for (int r = 0; r < g.rpi; ++r) acc += sf[(img * g.rpi + r) * 17 + c];
+                    for (int r = 0; r < g.rpi; ++r) acc += sc[(img * g.rpi + r) * 17];
                     acc /= (float)g.rpi;
-                    size_t oi = (size_t)n * g.out_ctot + g.out_coff + nc + c;
+                    const size_t oi = (size_t)n * g.out_ctot + g.out_coff + col;
                     if (g.out_f32) reinterpret_cast<float *>(g.out)[oi] = acc;
                     else reinterpret_cast<__nv_bfloat16 *>(g.out)[oi] = __float2bfloat16_rn(acc);
                 }
@@ -466,24 +555,23 @@ __global__ void __launch_bounds__(192) gemm_chain_kernel(const __grid_constant__
         }
         if (g.epi == GE_POOL) {
             epi_bar();
-            int per = g.tiles_y * g.tiles_x;
-            int n = mt / per, tt = mt - n * per;
-            int ty = tt / g.tiles_x, tx = tt - ty * g.tiles_x;
-            int c8n = g.tile_n / 8;
-            int t = threadIdx.x - 64;
-            for (int item = t; item < g.th * g.tw * c8n; item += 128) {
-                int c8 = item % c8n, o = item / c8n;
-                int oy = o / g.tw, ox = o - oy * g.tw;
-                int gy = ty * g.th + oy, gx = tx * g.tw + ox;
-                int col = n0 + c8 * 8;
+            const int per = g.tiles_y * g.tiles_x;
+            const int n = mt / per, tt = mt - n * per;
+            const int ty = tt / g.tiles_x, tx = tt - ty * g.tiles_x;
+            const int c8n = g.tile_n / 8;
+            for (int item = threadIdx.x - 64; item < g.th * g.tw * c8n; item += kProducerThreads) {
+                const int c8 = item % c8n, o = item / c8n;
+                const int oy = o / g.tw, ox = o - oy * g.tw;
+                const int gy = ty * g.th + oy, gx = tx * g.tw + ox;
+                const int col = n0 + c8 * 8;
                 if (gy >= g.PP || gx >= g.PQ || col + 8 > g.N || n >= g.batch || !ok) continue;
                 f8 m;
 #pragma unroll
                 for (int i = 0; i < 8; ++i) m.v[i] = -INFINITY;
                 for (int dy = 0; dy < g.pool_k; ++dy)
                     for (int dx = 0; dx < g.pool_k; ++dx) {
-                        int r = (oy * g.pool_stride + dy) * g.rw + ox * g.pool_stride + dx;
-                        f8 xv = unpack8(ld_shared16(stg + r * pool_pitch + c8 * 16));
+                        const int r = (oy * g.pool_stride + dy) * g.rw + ox * g.pool_stride + dx;
+                        const f8 xv = unpack8(ld_shared16(stg + r * pool_pitch + c8 * 16));
 #pragma unroll
                         for (int i = 0; i < 8; ++i) m.v[i] = fmaxf(m.v[i], xv.v[i]);
                     }

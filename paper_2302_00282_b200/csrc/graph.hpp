@@ -121,7 +121,7 @@ struct Launch {
     int epi = EPI_STORE;
     int skip = -1;                // tensor id added in the epilogue (identity shortcut)
     int out_dtype = XENOS_DTYPE_BF16;
-    int stages = 0, smem_bytes = 0, tmem_cols = 0;
+    int stages = 0, smem_bytes = 0, tmem_cols = 0, pipe_bytes = 0;
     // ---- fp32 linked chain (conv kxk -> conv1x1 -> pool)
     int Cmid = 0, K2 = 0, act2 = 0;
     int parts_outc = 1, tile_h = 0, tile_w = 0, tiles_h = 0, tiles_w = 0;   // tile of POOL outputs

@@ -648,11 +648,14 @@ struct Lower {
         int stage_bytes = 16384 + L.tile_n * 128;
         int budget = std::min(g.hw.smem_bytes_per_cta, 227 * 1024) / 2 - 4096;   // two CTAs per SM overlap epilogue and main loop
         L.stages = std::max(2, std::min(6, budget / stage_bytes));
-        L.stages = std::min(L.stages, std::max(2, L.kblocks));
-        L.smem_bytes = L.stages * stage_bytes + 2048;
+        L.stages = std::max(1, std::min(L.stages, L.kblocks));
+        // the pool / global-average epilogues stage the tile in the (by then idle) pipeline buffers
+        int staging = L.epi == EPI_POOL ? 128 * (L.tile_n * 2 + 16) : (L.epi == EPI_GAP ? 2 * 128 * 17 * 4 : 0);
+        L.pipe_bytes = (int)align_up((size_t)std::max(L.stages * stage_bytes, staging), 1024);
+        L.smem_bytes = L.pipe_bytes + 128 + 2048 + 1024;     // + barriers, row table, alignment slack
         if (L.smem_bytes > g.hw.smem_bytes_per_cta) return fail(g, XENOS_E_BAD_SPLIT, "split: pipeline does not fit shared memory");
         L.grid = L.m_tiles * L.n_tiles;
-        L.block = 192;
+        L.block = 320;
         // --- pack weights + bias
         L.w_off = blob_reserve(g, (size_t)L.npad * L.kpad * 2);
         L.b_off = blob_reserve(g, (size_t)L.npad * 4);

@@ -98,11 +98,17 @@ xenos_status_t runtime_bind(Graph &g, void *ws, size_t bytes, void *stream_v) {
                                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
             if (r != CUDA_SUCCESS) return fail(g, XENOS_E_CUDA, "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r));
         }
-        if ((e = cudaFuncSetAttribute(xk::gemm_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_gemm_smem)) != cudaSuccess)
-            return cuda_fail(g, "cudaFuncSetAttribute(gemm)", e);
     }
-    if (max_chain_smem > 48 * 1024)
-        if ((e = cudaFuncSetAttribute(xk::f32_conv_conv_pool_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_chain_smem)) != cudaSuccess)
+    // The opt-in limit is a per-function, per-device setting shared by every graph in the process:
+    // always raise it to the device maximum so that binding one graph never lowers it for another.
+    const int optin = (int)prop.sharedMemPerBlockOptin;
+    if (max_gemm_smem > optin || max_chain_smem > optin)
+        return fail(g, XENOS_E_CUDA, "a kernel of this plan needs more shared memory than the device offers");
+    if (any_gemm)
+        if ((e = cudaFuncSetAttribute(xk::gemm_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin)) != cudaSuccess)
+            return cuda_fail(g, "cudaFuncSetAttribute(gemm)", e);
+    if (max_chain_smem > 0)
+        if ((e = cudaFuncSetAttribute(xk::f32_conv_conv_pool_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin)) != cudaSuccess)
             return cuda_fail(g, "cudaFuncSetAttribute(f32 chain)", e);
     return XENOS_OK;
 }
@@ -232,7 +238,7 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
             p.map_mode = L.map_mode; p.tile_rows = L.tile_rows; p.imgs_per_tile = L.imgs_per_tile;
             p.th = L.patch_th; p.tw = L.patch_tw; p.rh = L.patch_rh; p.rw = L.patch_rw; p.tiles_y = L.tiles_y; p.tiles_x = L.tiles_x;
             p.pool_k = L.pool_k; p.pool_stride = L.pool_stride; p.pool_pad = L.pool_pad; p.PP = L.PP; p.PQ = L.PQ;
-            p.kblocks = L.kblocks; p.stages = L.stages; p.tile_n = L.tile_n; p.n_tiles = L.n_tiles; p.N = L.K;
+            p.kblocks = L.kblocks; p.stages = L.stages; p.pipe_bytes = L.pipe_bytes; p.tile_n = L.tile_n; p.n_tiles = L.n_tiles; p.N = L.K;
             p.act = L.act; p.act2 = L.act2; p.epi = L.epi; p.out_ctot = L.out_ctot; p.out_coff = L.out_coff;
             p.out_f32 = L.out_dtype == XENOS_DTYPE_F32;
             p.idesc = make_idesc(L.tile_n);
@@ -240,7 +246,7 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
             if (L.epi == EPI_POOL) m_tiles = N * L.tiles_y * L.tiles_x;
             else if (L.epi == EPI_GAP) m_tiles = (N + L.imgs_per_tile - 1) / L.imgs_per_tile;
             else m_tiles = (int)(((long long)N * L.rows_per_image + 127) / 128);
-            xk::gemm_chain_kernel<<<m_tiles * L.n_tiles, 192, L.smem_bytes, stream>>>(rt->tmaps[li], p);
+            xk::gemm_chain_kernel<<<m_tiles * L.n_tiles, xk::kThreads, L.smem_bytes, stream>>>(rt->tmaps[li], p);
             break;
         }
         default:
