@@ -185,6 +185,33 @@ XENOS_API xenos_status_t xenos_graph_profile(xenos_graph_t *g, int32_t batch,
                                              const void *const *inputs_dev, void *const *outputs_dev,
                                              void *cuda_stream, float *ms_per_launch, int32_t n_launches);
 
+/* Run one inference WITHOUT a caller-provided workspace.  (The paper has no counterpart: this
+ * entry point exists for deployment settings, not for the method.)
+ *
+ * Who needs it: code that runs where device allocation is forbidden or unavailable - a plugin
+ * inside a host application that owns and has already carved up all device memory, a
+ * real-time loop that is not allowed to call the allocator, a process whose memory pool is
+ * exhausted.  Such a caller cannot obtain the workspace xenos_graph_bind expects.  Here the
+ * workspace is a fixed 16 MiB array that is part of the library image (every device that
+ * loads the library holds it until the process exits); the caller passes only its input and
+ * output buffers, exactly as for xenos_graph_run.
+ *
+ *  - Valid on a compiled graph, bound or not; an existing xenos_graph_bind binding is left
+ *    untouched.  Graphs whose workspace_bytes exceed 16 MiB are refused with
+ *    XENOS_E_WORKSPACE and a message giving both sizes.
+ *  - Calls no cudaMalloc / cudaFree and no allocating library routine.
+ *  - The first call on a device looks up the array's device address and uploads the graph's
+ *    parameters into it; make that first call outside any stream capture.  Parameters are
+ *    uploaded again whenever another graph has used the array in between.
+ *  - All graphs and all calls share the one array, and it keeps the previous call's contents
+ *    (the library clears the words that must start at zero).  Two calls that overlap on the
+ *    device - different streams or different host threads - race; serialise them.
+ *  - Synchronous: it waits for `cuda_stream` and returns the device status like
+ *    xenos_graph_status. */
+XENOS_API xenos_status_t xenos_graph_run_builtin_scratch(xenos_graph_t *g, int32_t batch,
+                                                         const void *const *inputs_dev,
+                                                         void *const *outputs_dev, void *cuda_stream);
+
 /* Synchronise `cuda_stream` and return the device status word: XENOS_OK, or
  * XENOS_E_TIMEOUT / XENOS_E_BOUNDS if a kernel gave up a bounded wait or failed an index
  * check since the last call (the word is then cleared). */

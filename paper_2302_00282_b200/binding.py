@@ -42,7 +42,7 @@ class OpDesc(ctypes.Structure):
 
 EXPORTS = ["xenos_graph_create", "xenos_graph_add_input", "xenos_graph_add_op", "xenos_graph_mark_output",
            "xenos_graph_link", "xenos_graph_split", "xenos_graph_compile", "xenos_graph_bind", "xenos_graph_run",
-           "xenos_graph_profile", "xenos_graph_status", "xenos_graph_get_plan", "xenos_graph_launch_count", "xenos_graph_destroy",
+           "xenos_graph_profile", "xenos_graph_run_builtin_scratch", "xenos_graph_status", "xenos_graph_get_plan", "xenos_graph_launch_count", "xenos_graph_destroy",
            "xenos_last_error"]
 
 _lib = None
@@ -65,6 +65,7 @@ def lib() -> ctypes.CDLL:
         L.xenos_graph_bind.argtypes = [vp, vp, sz, vp]
         L.xenos_graph_run.argtypes = [vp, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), vp]
         L.xenos_graph_profile.argtypes = [vp, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), vp, _f32p, i32]
+        L.xenos_graph_run_builtin_scratch.argtypes = [vp, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), vp]
         L.xenos_graph_status.argtypes = [vp, vp]
         L.xenos_graph_get_plan.argtypes = [vp, ctypes.c_char_p, sz, ctypes.POINTER(sz)]
         L.xenos_graph_launch_count.argtypes = [vp, ctypes.POINTER(i32)]
@@ -156,6 +157,12 @@ class Graph:
         oa = (ctypes.c_void_p * len(outputs))(*outputs)
         self._check(lib().xenos_graph_profile(self._h, batch, ia, oa, ctypes.c_void_p(stream), ms, n))
         return list(ms)
+
+    def run_builtin_scratch(self, batch: int, inputs: Sequence[int], outputs: Sequence[int], stream: int = 0):
+        """Inference with the library's built-in 16 MiB workspace instead of a bound one (synchronous)."""
+        ia = (ctypes.c_void_p * len(inputs))(*inputs)
+        oa = (ctypes.c_void_p * len(outputs))(*outputs)
+        self._check(lib().xenos_graph_run_builtin_scratch(self._h, batch, ia, oa, ctypes.c_void_p(stream)))
 
     def status(self, stream: int = 0):
         self._check(lib().xenos_graph_status(self._h, ctypes.c_void_p(stream)))

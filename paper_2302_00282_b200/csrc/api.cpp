@@ -1,5 +1,6 @@
 // C ABI of the library: argument checks, the call-order state machine, and dispatch into the
 // host passes and the CUDA runtime.  No exception leaves this file.
+#include <atomic>
 #include <cstring>
 #include <new>
 #include <string>
@@ -59,6 +60,8 @@ xenos_status_t xenos_graph_create(const xenos_hw_info_t *hw, xenos_graph_t **out
         }
         p->g.hw = *hw;
     }
+    static std::atomic<uint64_t> next_serial{1};
+    p->g.serial = next_serial.fetch_add(1);
     *out = p;
     return XENOS_OK;
 }
@@ -279,8 +282,31 @@ xenos_status_t xenos_graph_launch_count(const xenos_graph_t *gp, int32_t *launch
     return XENOS_OK;
 }
 
+xenos_status_t xenos_graph_run_builtin_scratch(xenos_graph_t *gp, int32_t batch, const void *const *inputs_dev,
+                                               void *const *outputs_dev, void *cuda_stream) {
+    if (!gp) return XENOS_E_INVALID;
+    XENOS_GUARD_BEGIN
+    Graph &g = gp->g;
+    if (g.state < ST_COMPILED) return fail(g, XENOS_E_STATE, "run_builtin_scratch before compile");
+    if (batch < 1 || batch > g.max_batch)
+        return fail(g, XENOS_E_INVALID, "run_builtin_scratch: batch exceeds max_batch given to compile");
+    if (!inputs_dev || !outputs_dev) return fail(g, XENOS_E_INVALID, "run_builtin_scratch: NULL pointer array");
+    for (size_t i = 0; i < g.inputs.size(); ++i)
+        if (!inputs_dev[i]) return fail(g, XENOS_E_INVALID, "run_builtin_scratch: NULL input pointer");
+    for (size_t i = 0; i < g.outputs.size(); ++i)
+        if (!outputs_dev[i]) return fail(g, XENOS_E_INVALID, "run_builtin_scratch: NULL output pointer");
+    if (g.workspace_bytes > runtime_builtin_scratch_bytes())
+        return fail(g, XENOS_E_WORKSPACE,
+                    "run_builtin_scratch: this graph needs " + std::to_string(g.workspace_bytes) +
+                        " workspace bytes but the built-in scratch holds only " +
+                        std::to_string(runtime_builtin_scratch_bytes()) + "; use xenos_graph_bind with your own buffer");
+    return runtime_run_builtin(g, batch, inputs_dev, outputs_dev, cuda_stream);
+    XENOS_GUARD_END(gp)
+}
+
 xenos_status_t xenos_graph_destroy(xenos_graph_t *gp) {
     if (!gp) return XENOS_E_INVALID;
+    runtime_free_builtin(gp->g);
     runtime_free(gp->g);
     delete gp;
     return XENOS_OK;

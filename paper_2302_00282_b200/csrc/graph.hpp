@@ -176,6 +176,8 @@ struct Graph {
     // ---- bound
     void *ws = nullptr;
     void *rt = nullptr;                   // runtime-private data (tensor maps), owned by runtime.cu
+    void *rt_builtin = nullptr;           // the same for the binding to the library's built-in scratch
+    uint64_t serial = 0;                  // unique per graph, names the owner of the built-in scratch
     mutable std::string err;
 };
 
@@ -195,6 +197,9 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
                            float *ms_per_launch = nullptr);
 xenos_status_t runtime_status(Graph &g, void *stream);
 void runtime_free(Graph &g);
+xenos_status_t runtime_run_builtin(Graph &g, int batch, const void *const *in, void *const *out, void *stream);
+void runtime_free_builtin(Graph &g);
+size_t runtime_builtin_scratch_bytes();
 
 xenos_status_t fail(const Graph &g, xenos_status_t code, const std::string &msg);
 

@@ -281,4 +281,62 @@ xenos_status_t runtime_status(Graph &g, void *stream_v) {
     return fail(g, code, code == XENOS_E_TIMEOUT ? "a kernel gave up a bounded wait" : "a kernel failed an index check");
 }
 
+// ------------------------------------------------------------------------------------------------
+// Built-in scratch: a workspace that lives inside the library image, for callers that must not
+// allocate device memory themselves.
+// ------------------------------------------------------------------------------------------------
+constexpr size_t kBuiltinScratchBytes = 16u << 20;    // 16 MiB, held by every device that loads the library
+constexpr int kMaxDevices = 64;
+static __device__ __align__(256) unsigned char g_builtin_scratch[kBuiltinScratchBytes];
+// In host code the name g_builtin_scratch is only a handle for the symbol, not a device address;
+// the address is looked up once per device and cached here.
+static void *g_builtin_ptr[kMaxDevices] = {};
+static uint64_t g_builtin_owner[kMaxDevices] = {};    // serial of the graph whose parameters the array holds
+
+size_t runtime_builtin_scratch_bytes() { return kBuiltinScratchBytes; }
+
+void runtime_free_builtin(Graph &g) {
+    delete static_cast<Runtime *>(g.rt_builtin);
+    g.rt_builtin = nullptr;
+    for (int d = 0; d < kMaxDevices; ++d)
+        if (g_builtin_owner[d] == g.serial) g_builtin_owner[d] = 0;
+}
+
+xenos_status_t runtime_run_builtin(Graph &g, int batch, const void *const *in, void *const *out, void *stream_v) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(g, "no CUDA device (this library has no CPU fallback)", e);
+    if (dev < 0 || dev >= kMaxDevices) return fail(g, XENOS_E_CUDA, "run_builtin_scratch: device index out of range");
+    if (!g_builtin_ptr[dev]) {
+        void *p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_builtin_scratch);
+        if (e != cudaSuccess || !p) return cuda_fail(g, "cudaGetSymbolAddress(built-in scratch)", e);
+        g_builtin_ptr[dev] = p;
+    }
+    void *scratch = g_builtin_ptr[dev];
+    // run with the graph temporarily bound to the built-in scratch; the caller's own binding
+    // (xenos_graph_bind) is put back afterwards
+    void *save_ws = g.ws, *save_rt = g.rt;
+    g.rt = g.rt_builtin;
+    xenos_status_t st = XENOS_OK;
+    Runtime *rb = static_cast<Runtime *>(g.rt_builtin);
+    if (!rb || rb->device != dev || g_builtin_owner[dev] != g.serial) {
+        // the array holds nothing or another graph's data: upload parameters, clear status, encode maps
+        st = runtime_bind(g, scratch, kBuiltinScratchBytes, stream);
+        g.rt_builtin = g.rt;
+        g_builtin_owner[dev] = st == XENOS_OK ? g.serial : 0;
+    } else {
+        g.ws = scratch;
+        // the status word keeps the last call's contents: start from zero
+        if ((e = cudaMemsetAsync(static_cast<uint8_t *>(scratch) + g.status_off, 0, 256, stream)) != cudaSuccess)
+            st = cuda_fail(g, "status clear", e);
+    }
+    if (st == XENOS_OK) st = runtime_run(g, batch, in, out, stream, nullptr);
+    if (st == XENOS_OK) st = runtime_status(g, stream);
+    g.ws = save_ws;
+    g.rt = save_rt;
+    return st;
+}
+
 }  // namespace xenos
