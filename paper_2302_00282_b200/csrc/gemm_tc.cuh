@@ -1,22 +1,27 @@
-// Linked-chain implicit GEMM on the 5th-generation tensor cores (sm_100a).
+// Linked-chain implicit GEMM on the 5th-generation tensor cores (sm_100a), persistent form.
 //
-// One CTA owns a 128-row tile of output pixels and a slice of <= 256 output channels
-// (the operator split of Section 4.2: output channels first, then rows / columns).
-//   warp 0      : TMA producer for the weight tile (cp.async.bulk.tensor, 128-byte swizzle)
-//   warp 1      : allocates tensor memory, one lane issues tcgen05.mma (bf16 x bf16 -> fp32)
-//   warps 2..9  : produce the activation operand straight into shared memory in the layout the
-//                 tensor core reads (K-major, 128-byte swizzle) - the paper's "write in the
-//                 order the next operator reads" (Section 4.1) - then run the epilogue
+// One CTA per SM walks over the tiles of a chain (tile = 128 output pixels x tile_n <= 256 output
+// channels: the operator split of Section 4.2 of the Xenos paper, output channels first, then
+// rows / columns), so that tensor-memory allocation, barrier set-up and descriptor fetches are
+// paid once and the stages of neighbouring tiles overlap:
+//   warp 0        : TMA producer - weight tiles (128-byte swizzle) and, for linked depthwise
+//                   chains, the input halo tile of the depthwise stage (4-D box, zero fill = padding)
+//   warp 1        : one lane issues tcgen05.mma (bf16 x bf16 -> fp32) into one of two
+//                   tensor-memory accumulators
+//   warps 2..9    : produce the activation operand straight into shared memory in the layout the
+//                   tensor core reads (K-major, 128-byte swizzle) - the paper's "write in the
+//                   order the next operator reads" (Section 4.1)
+//   warps 10..13  : epilogue of the previous tile, overlapped with the production of the next
 // The activation operand of one 64-wide K block comes from one of
 //   gather : a k x k / strided / padded window of an NHWC bf16 tensor (16-byte cp.async, zero fill)
 //   stem   : a k x k window of a small-channel NCHW image (scalar loads, converted to bf16)
-//   dw     : a depthwise 3x3 + bias + activation computed on the fly (linked dw -> pw)
+//   dw     : a depthwise 3x3 + bias + activation computed from the halo tile in shared memory
 // and a second gather segment can append the K blocks of a shortcut 1x1 convolution, so the
 // residual sum of a shortcut connection happens in the accumulator.
-// Epilogues: bias, activation, identity-shortcut add, then a coalesced store at a channel
-// offset (concat needs no kernel), a max pool over the tile's patch, or a global average.
+// Epilogues: bias, activation, identity-shortcut add, then a store at a channel offset (concat
+// needs no kernel), a max pool over the tile's patch, or a global average.
 //
-// Every wait on an mbarrier is bounded; on expiry the CTA records XENOS_E_TIMEOUT in the status
+// Every wait on an mbarrier is bounded; on expiry the role records XENOS_E_TIMEOUT in the status
 // word and leaves through the common exit (tensor memory is always released).
 #pragma once
 
@@ -37,6 +42,10 @@ constexpr int kTileM = 128;
 constexpr int kTileK = 64;
 constexpr int kABytes = kTileM * kTileK * 2;    // 16 KB per stage
 constexpr int kMaxStages = 6;
+constexpr int kMaxHaloStages = 4;
+constexpr int kProducerThreads = 256;           // warps 2..9
+constexpr int kEpilogueThreads = 128;           // warps 10..13
+constexpr int kThreads = 64 + kProducerThreads + kEpilogueThreads;
 constexpr unsigned kStatusTimeout = 0x80000000u | 9u;
 constexpr unsigned kStatusBounds = 0x80000000u | 10u;
 constexpr int kSpinLimit = 1 << 22;             // try_wait polls before a wait gives up
@@ -54,9 +63,15 @@ struct GemmParams {
     void *out;
     unsigned int *status;
     int batch, P, Q, rpi;
-    int map_mode, tile_rows, imgs_per_tile;
-    int th, tw, rh, rw, tiles_y, tiles_x, pool_k, pool_stride, pool_pad, PP, PQ;
-    int kblocks, stages, tile_n, n_tiles, N, pipe_bytes;
+    int map_mode, tile_rows;
+    // PATCH tiles: ni images x rh x rw positions of the conv output, origin (ty*step_y - off_y, tx*step_x - off_x)
+    int ni, rh, rw, tiles_y, tiles_x, step_y, step_x, off_y, off_x;
+    int pool_k, pool_stride, PP, PQ, pth, ptw;     // max-pool epilogue: pth x ptw pool outputs per tile
+    int gap_imgs, gap_rpi;                         // global-average epilogue: whole images per tile
+    int kblocks, stages, tile_n, n_tiles, m_tiles, N;
+    int acc_stride, tmem_cols;                     // two accumulators, acc_stride columns apart
+    int hstages, halo_bytes, halo_stride, halo_h, halo_w, halo_cb;   // depthwise halo ring
+    int off_halo, off_stg, off_bar;                // shared-memory offsets from the 1024-aligned base
     int act, act2, epi, out_ctot, out_coff, out_f32, skip_ctot;
     uint32_t idesc;
 };
@@ -86,6 +101,18 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     }
     return false;
 }
+// One lane polls, the warp follows: keeps 32x fewer pollers on the barrier word.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, int lane) {
+    int ok = 1;
+    if (lane == 0) ok = mbar_wait(bar, parity) ? 1 : 0;
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    return ok != 0;
+}
+// Every lane has finished (and fenced) its own accesses; one arrival per warp.
+__device__ __forceinline__ void warp_arrive(uint32_t bar, int lane) {
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar);
+}
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -110,6 +137,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm,
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(dst), "l"(tm), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+// c0 (the innermost coordinate) must be a multiple of 8 elements; the others may be negative
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *tm, int c0, int c1, int c2, int c3, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
 
 // K-major operand tile with 128-byte swizzle: rows 128 bytes apart, 8-row groups 1024 bytes apart.
@@ -146,9 +179,7 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float *v) {
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-constexpr int kProducerThreads = 256;           // warps 2..9
-constexpr int kThreads = 64 + kProducerThreads;
-__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 // ---- row <-> pixel -----------------------------------------------------------------------------
 struct RowPos { int valid, n, p, q; };
@@ -165,14 +196,15 @@ __device__ __forceinline__ RowPos map_row(const GemmParams &g, int mt, int r) {
             o.valid = 1;
         }
     } else {
-        int per = g.tiles_y * g.tiles_x;
-        o.n = mt / per;
-        int t = mt - o.n * per;
-        int ty = t / g.tiles_x, tx = t - ty * g.tiles_x;
-        int dy = r / g.rw, dx = r - dy * g.rw;
-        o.p = ty * g.th * g.pool_stride - g.pool_pad + dy;
-        o.q = tx * g.tw * g.pool_stride - g.pool_pad + dx;
-        o.valid = (r < g.rh * g.rw) && o.n < g.batch && o.p >= 0 && o.p < g.P && o.q >= 0 && o.q < g.Q;
+        const int per = g.tiles_y * g.tiles_x, area = g.rh * g.rw;
+        const int grp = mt / per, t = mt - grp * per;
+        const int ty = t / g.tiles_x, tx = t - ty * g.tiles_x;
+        const int img = r / area, rem = r - img * area;
+        const int dy = rem / g.rw, dx = rem - dy * g.rw;
+        o.n = grp * g.ni + img;
+        o.p = ty * g.step_y - g.off_y + dy;
+        o.q = tx * g.step_x - g.off_x + dx;
+        o.valid = (img < g.ni) && o.n < g.batch && o.p >= 0 && o.p < g.P && o.q >= 0 && o.q < g.Q;
     }
     return o;
 }
@@ -182,19 +214,6 @@ __device__ __forceinline__ RowPos map_row(const GemmParams &g, int mt, int r) {
 // which is what a 128-byte-swizzle TMA load would have written and what the MMA descriptor expects.
 __device__ __forceinline__ uint32_t a_chunk_addr(uint32_t a_base, int row, int j) {
     return a_base + row * 128 + ((j ^ (row & 7)) << 4);
-}
-
-// One lane polls, the warp follows: keeps 32x fewer pollers on the barrier word.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, int lane) {
-    int ok = 1;
-    if (lane == 0) ok = mbar_wait(bar, parity) ? 1 : 0;
-    ok = __shfl_sync(0xffffffffu, ok, 0);
-    return ok != 0;
-}
-// Every lane has fenced its own writes; one arrival per warp.
-__device__ __forceinline__ void warp_arrive(uint32_t bar, int lane) {
-    __syncwarp();
-    if (lane == 0) mbar_arrive(bar);
 }
 
 struct GatherState { int tap_r, tap_s, cc; };   // (tap, channel chunk) of a thread's next 8-channel chunk
@@ -209,17 +228,17 @@ __device__ __forceinline__ void gather_advance(GatherState &st, int n, int C8, i
 }
 
 // gather: thread = (row, half); it copies chunks 4*half .. 4*half+3 of its row with 16-byte cp.async
-__device__ __forceinline__ void produce_gather(const GemmSeg &sg, GatherState st, const int4 ri, uint32_t a_base,
+__device__ __forceinline__ void produce_gather(const GemmSeg &sg, GatherState st, const RowPos &rp, uint32_t a_base,
                                                int row, int half) {
     const __nv_bfloat16 *src = reinterpret_cast<const __nv_bfloat16 *>(sg.src);
     const int C8 = sg.C >> 3;
-    const int ih0 = ri.z * sg.stride - sg.pad, iw0 = ri.w * sg.stride - sg.pad;
-    const __nv_bfloat16 *img = src + (size_t)ri.y * sg.H * sg.W * sg.C;
+    const int ih0 = rp.p * sg.stride - sg.pad, iw0 = rp.q * sg.stride - sg.pad;
+    const __nv_bfloat16 *img = src + (size_t)rp.n * sg.H * sg.W * sg.C;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const void *ptr = src;
         uint32_t bytes = 0;
-        if (ri.x && st.tap_r < sg.k) {
+        if (rp.valid && st.tap_r < sg.k) {
             int ih = ih0 + st.tap_r, iw = iw0 + st.tap_s;
             if (ih >= 0 && ih < sg.H && iw >= 0 && iw < sg.W) {
                 ptr = img + ((size_t)ih * sg.W + iw) * sg.C + st.cc * 8;
@@ -232,13 +251,13 @@ __device__ __forceinline__ void produce_gather(const GemmSeg &sg, GatherState st
 }
 
 // stem: K element e = (r * k + s) * C + c of an NCHW image (fp32 or bf16); thread = (row, half)
-__device__ __forceinline__ void produce_stem(const GemmSeg &sg, int kb_local, const int4 ri, uint32_t a_base,
+__device__ __forceinline__ void produce_stem(const GemmSeg &sg, int kb_local, const RowPos &rp, uint32_t a_base,
                                              int row, int half) {
     int e = kb_local * kTileK + half * 32;
     int tap = e / sg.C, c = e - tap * sg.C;
     int r = tap / sg.k, s = tap - r * sg.k;
-    const int ih0 = ri.z * sg.stride - sg.pad, iw0 = ri.w * sg.stride - sg.pad;
-    const size_t img = (size_t)ri.y * sg.C * sg.H * sg.W;
+    const int ih0 = rp.p * sg.stride - sg.pad, iw0 = rp.q * sg.stride - sg.pad;
+    const size_t img = (size_t)rp.n * sg.C * sg.H * sg.W;
     const float *sf = reinterpret_cast<const float *>(sg.src) + img;
     const __nv_bfloat16 *sh = reinterpret_cast<const __nv_bfloat16 *>(sg.src) + img;
 #pragma unroll 1
@@ -247,7 +266,7 @@ __device__ __forceinline__ void produce_stem(const GemmSeg &sg, int kb_local, co
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             float x = 0.0f;
-            if (ri.x && r < sg.k) {
+            if (rp.valid && r < sg.k) {
                 int ih = ih0 + r, iw = iw0 + s;
                 if (ih >= 0 && ih < sg.H && iw >= 0 && iw < sg.W) {
                     int off = (c * sg.H + ih) * sg.W + iw;
@@ -261,39 +280,19 @@ __device__ __forceinline__ void produce_stem(const GemmSeg &sg, int kb_local, co
     }
 }
 
-// depthwise 3x3 + bias + activation, rounded to bf16 and stored in the consumer's operand layout.
-// thread = (chunk j of 8 channels, row group); it owns rows rg, rg+32, rg+64, rg+96 so that the
-// nine tap weights of its 8 channels are fetched once per K block and four independent pixel
-// loads are in flight per tap.
-struct DwRows { long long base[4]; unsigned mask[4]; };
-
-__device__ __forceinline__ void dw_rows_init(const GemmSeg &sg, const int4 *rowtab, int rg, DwRows &dr) {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int4 ri = rowtab[rg + 32 * i];
-        int ih0 = ri.z * sg.stride - sg.pad, iw0 = ri.w * sg.stride - sg.pad;
-        unsigned m = 0;
-        if (ri.x) {
-#pragma unroll
-            for (int r = 0; r < 3; ++r)
-#pragma unroll
-                for (int s = 0; s < 3; ++s)
-                    if (ih0 + r >= 0 && ih0 + r < sg.H && iw0 + s >= 0 && iw0 + s < sg.W) m |= 1u << (r * 3 + s);
-        }
-        if (ri.x) m |= 1u << 9;        // bit 9: the row is a real output pixel
-        dr.mask[i] = m;
-        dr.base[i] = (((long long)ri.y * sg.H + ih0) * sg.W + iw0) * sg.C;
-    }
-}
-
-__device__ __forceinline__ void produce_dw(const GemmSeg &sg, int kb_local, const DwRows &dr, uint32_t a_base, int j, int rg) {
+// depthwise 3x3 + bias + activation from the halo tile in shared memory ([image][y][x][cb channels],
+// dense), rounded to bf16 and stored in the consumer's operand layout.
+// thread = (chunk j of 8 channels, row group); it owns rows rg, rg+32, rg+64, rg+96 so that the nine
+// tap weights of its 8 channels are fetched once per K block.
+__device__ __forceinline__ void produce_dw(const GemmSeg &sg, const GemmParams &g, int kb_local, uint32_t halo,
+                                           const int (&hoff)[4], uint32_t a_base, int j, int rg) {
     const int c0 = kb_local * kTileK + j * 8;
-    if (c0 >= sg.C) {
+    const int cbytes = g.halo_cb * 2;
+    if (c0 >= sg.C || j * 8 >= g.halo_cb) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) st_shared16(a_chunk_addr(a_base, rg + 32 * i, j), make_uint4(0u, 0u, 0u, 0u));
         return;
     }
-    const __nv_bfloat16 *src = reinterpret_cast<const __nv_bfloat16 *>(sg.src) + c0;
     float acc[4][8];
     {
         const float4 b0 = __ldg(reinterpret_cast<const float4 *>(sg.dw_b + c0)), b1 = __ldg(reinterpret_cast<const float4 *>(sg.dw_b + c0 + 4));
@@ -303,20 +302,16 @@ __device__ __forceinline__ void produce_dw(const GemmSeg &sg, int kb_local, cons
             acc[i][4] = b1.x; acc[i][5] = b1.y; acc[i][6] = b1.z; acc[i][7] = b1.w;
         }
     }
+    const uint32_t hb = halo + j * 16;
 #pragma unroll
     for (int t = 0; t < 9; ++t) {
         const float *wt = sg.dw_w + (size_t)t * sg.C + c0;
         const float4 w0 = __ldg(reinterpret_cast<const float4 *>(wt)), w1 = __ldg(reinterpret_cast<const float4 *>(wt + 4));
-        const int toff = ((t / 3) * sg.W + (t % 3)) * sg.C;
-        uint4 xv[4];
+        const int toff = ((t / 3) * g.halo_w + (t % 3)) * cbytes;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            xv[i] = make_uint4(0u, 0u, 0u, 0u);
-            if (dr.mask[i] & (1u << t)) xv[i] = __ldg(reinterpret_cast<const uint4 *>(src + dr.base[i] + toff));
-        }
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const f8 x = unpack8(xv[i]);
+            if (hoff[i] < 0) continue;
+            const f8 x = unpack8(ld_shared16(hb + hoff[i] + toff));
             acc[i][0] = fmaf(x.v[0], w0.x, acc[i][0]); acc[i][1] = fmaf(x.v[1], w0.y, acc[i][1]);
             acc[i][2] = fmaf(x.v[2], w0.z, acc[i][2]); acc[i][3] = fmaf(x.v[3], w0.w, acc[i][3]);
             acc[i][4] = fmaf(x.v[4], w1.x, acc[i][4]); acc[i][5] = fmaf(x.v[5], w1.y, acc[i][5]);
@@ -325,51 +320,47 @@ __device__ __forceinline__ void produce_dw(const GemmSeg &sg, int kb_local, cons
     }
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        uint4 o = make_uint4(0u, 0u, 0u, 0u);
-        if (dr.mask[i]) {
-            f8 r;
+        f8 r;
 #pragma unroll
-            for (int c = 0; c < 8; ++c) r.v[c] = apply_act(acc[i][c], sg.dw_act);
-            o = pack8(r);
-        }
-        st_shared16(a_chunk_addr(a_base, rg + 32 * i, j), o);
+        for (int c = 0; c < 8; ++c) r.v[c] = apply_act(acc[i][c], sg.dw_act);
+        st_shared16(a_chunk_addr(a_base, rg + 32 * i, j), hoff[i] < 0 ? make_uint4(0u, 0u, 0u, 0u) : pack8(r));
     }
 }
 
 // ---- the kernel --------------------------------------------------------------------------------
-// Shared memory: [stages x (A 16 KB | B tile_n x 128 B)] [staging, if larger] [barriers] [row table]
-__global__ void __launch_bounds__(kThreads, 2) gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const GemmParams g) {
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmH, const GemmParams g) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t sbase = (raw + 1023u) & ~1023u;
     uint8_t *sm = smem_raw + (sbase - raw);
     const int stage_bytes = kABytes + g.tile_n * 128;
-    const int pipe_bytes = g.pipe_bytes;            // >= stages * stage_bytes and >= the epilogue staging need
-    const uint32_t bar_base = sbase + pipe_bytes;
+    const uint32_t bar_base = sbase + g.off_bar;
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto empty_bar = [&](int s) { return bar_base + 8u * (kMaxStages + s); };
-    const uint32_t accum_bar = bar_base + 8u * (2 * kMaxStages);
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(sm + pipe_bytes + 8 * (2 * kMaxStages + 1));
-    int4 *rowtab = reinterpret_cast<int4 *>(sm + pipe_bytes + 128);
+    auto accf_bar = [&](int b) { return bar_base + 8u * (2 * kMaxStages + b); };
+    auto acce_bar = [&](int b) { return bar_base + 8u * (2 * kMaxStages + 2 + b); };
+    auto hfull_bar = [&](int s) { return bar_base + 8u * (2 * kMaxStages + 4 + s); };
+    auto hempty_bar = [&](int s) { return bar_base + 8u * (2 * kMaxStages + 4 + kMaxHaloStages + s); };
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(sm + g.off_bar + 8 * (2 * kMaxStages + 4 + 2 * kMaxHaloStages));
+    volatile int *fail_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int mt = blockIdx.x / g.n_tiles, nt = blockIdx.x - mt * g.n_tiles;
-    uint32_t tmem_cols = 32;
-    while ((int)tmem_cols < g.tile_n) tmem_cols <<= 1;
+    const int total_tiles = g.m_tiles * g.n_tiles;
+    const bool dw_mode = g.seg[0].mode == GA_DW;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < g.stages; ++s) { mbar_init(full_bar(s), kProducerThreads / 32 + 1); mbar_init(empty_bar(s), 1); }
-        mbar_init(accum_bar, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), kEpilogueThreads / 32); }
+        for (int s = 0; s < g.hstages; ++s) { mbar_init(hfull_bar(s), 1); mbar_init(hempty_bar(s), kProducerThreads / 32); }
+        *fail_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
+        if (dw_mode) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmH) : "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(tmem_cols) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)g.tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    if (threadIdx.x >= 64 && threadIdx.x < 64 + kTileM) {
-        const RowPos rp = map_row(g, mt, threadIdx.x - 64);
-        rowtab[threadIdx.x - 64] = make_int4(rp.valid, rp.n, rp.p, rp.q);
     }
     tc_fence_before();
     __syncthreads();
@@ -378,214 +369,262 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_chain_kernel(const __grid_co
     bool ok = true;
 
     if (warp == 0) {
-        // ---- weight tiles by TMA ----
+        // ---- TMA: weight tiles, and the depthwise halo tiles ----
         if (lane == 0) {
-            for (int kb = 0; kb < g.kblocks && ok; ++kb) {
-                int s = kb % g.stages;
-                uint32_t ph = (kb / g.stages) & 1;
-                ok = mbar_wait(empty_bar(s), ph ^ 1u);
-                if (!ok) break;
-                mbar_arrive_expect_tx(full_bar(s), (uint32_t)g.tile_n * 128u);
-                tma_load_2d(sbase + s * stage_bytes + kABytes, &tmB, kb * kTileK, nt * g.tile_n, full_bar(s));
+            int it = 0;
+            for (int ti = blockIdx.x; ti < total_tiles && ok; ti += gridDim.x) {
+                const int mt = ti / g.n_tiles, nt = ti - mt * g.n_tiles;
+                int hx = 0, hy = 0, hn = 0;
+                if (dw_mode) {
+                    const int per = g.tiles_y * g.tiles_x, grp = mt / per, t = mt - grp * per;
+                    const int ty = t / g.tiles_x, tx = t - ty * g.tiles_x;
+                    hn = grp * g.ni;
+                    hy = (ty * g.step_y - g.off_y) * g.seg[0].stride - g.seg[0].pad;
+                    hx = (tx * g.step_x - g.off_x) * g.seg[0].stride - g.seg[0].pad;
+                }
+                for (int kb = 0; kb < g.kblocks && ok; ++kb, ++it) {
+                    if (dw_mode) {
+                        const int hs = it % g.hstages;
+                        ok = mbar_wait(hempty_bar(hs), ((it / g.hstages) & 1) ^ 1u);
+                        if (!ok) break;
+                        mbar_arrive_expect_tx(hfull_bar(hs), (uint32_t)g.halo_bytes);
+                        tma_load_4d(sbase + g.off_halo + hs * g.halo_stride, &tmH, kb * kTileK, hx, hy, hn, hfull_bar(hs));
+                    }
+                    const int s = it % g.stages;
+                    ok = mbar_wait(empty_bar(s), ((it / g.stages) & 1) ^ 1u);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(full_bar(s), (uint32_t)g.tile_n * 128u);
+                    tma_load_2d(sbase + s * stage_bytes + kABytes, &tmB, kb * kTileK, nt * g.tile_n, full_bar(s));
+                }
             }
             if (!ok) atomicCAS(g.status, 0u, kStatusTimeout);
         }
     } else if (warp == 1) {
         // ---- MMA issue ----
         if (lane == 0) {
-            for (int kb = 0; kb < g.kblocks && ok; ++kb) {
-                int s = kb % g.stages;
-                uint32_t ph = (kb / g.stages) & 1;
-                ok = mbar_wait(full_bar(s), ph);
+            int it = 0, i = 0;
+            for (int ti = blockIdx.x; ti < total_tiles && ok; ti += gridDim.x, ++i) {
+                const int b = i & 1;
+                ok = mbar_wait(acce_bar(b), ((i >> 1) & 1) ^ 1u);      // the epilogue has drained this accumulator
                 if (!ok) break;
                 tc_fence_after();
-                uint32_t a = sbase + s * stage_bytes, b = a + kABytes;
+                const uint32_t d_tmem = tmem_base + b * g.acc_stride;
+                for (int kb = 0; kb < g.kblocks && ok; ++kb, ++it) {
+                    const int s = it % g.stages;
+                    ok = mbar_wait(full_bar(s), (it / g.stages) & 1);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t a = sbase + s * stage_bytes, bb = a + kABytes;
 #pragma unroll
-                for (int k4 = 0; k4 < kTileK / 16; ++k4)
-                    umma_bf16(tmem_base, umma_desc_sw128(a + k4 * 32), umma_desc_sw128(b + k4 * 32), g.idesc,
-                              (kb > 0 || k4 > 0) ? 1u : 0u);
-                umma_commit(empty_bar(s));
+                    for (int k4 = 0; k4 < kTileK / 16; ++k4)
+                        umma_bf16(d_tmem, umma_desc_sw128(a + k4 * 32), umma_desc_sw128(bb + k4 * 32), g.idesc,
+                                  (kb > 0 || k4 > 0) ? 1u : 0u);
+                    umma_commit(empty_bar(s));
+                }
+                if (ok) umma_commit(accf_bar(b));
             }
-            if (ok) umma_commit(accum_bar);
-            else atomicCAS(g.status, 0u, kStatusTimeout);
+            if (!ok) atomicCAS(g.status, 0u, kStatusTimeout);
         }
-    } else {
-        // ---- activation operand, then epilogue ----
+    } else if (warp < 2 + kProducerThreads / 32) {
+        // ---- activation operand ----
         const int pt = threadIdx.x - 64;                 // 0..255
         const int grow = pt & 127, ghalf = pt >> 7;      // gather / stem mapping
         const int dj = pt & 7, drg = pt >> 3;            // depthwise mapping
-        const int4 ri = rowtab[grow];
-        GatherState gs0 = {0, 0, 0}, gs1 = {0, 0, 0};
-        if (g.seg[0].mode == GA_GATHER && ghalf) gather_advance(gs0, 4, g.seg[0].C >> 3, g.seg[0].k);
-        if (g.seg[1].mode == GA_GATHER && ghalf) gather_advance(gs1, 4, g.seg[1].C >> 3, g.seg[1].k);
-        DwRows dr;
-        if (g.seg[0].mode == GA_DW) dw_rows_init(g.seg[0], rowtab, drg, dr);
+        int hoff[4] = {-1, -1, -1, -1};                  // byte offset of each owned row's window origin in the halo tile
+        if (dw_mode) {
+            const int area = g.rh * g.rw, cbytes = g.halo_cb * 2;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int r = drg + 32 * i;
+                const int img = r / area, rem = r - img * area;
+                const int dy = rem / g.rw, dx = rem - dy * g.rw;
+                if (img < g.ni) hoff[i] = ((img * g.halo_h + dy * g.seg[0].stride) * g.halo_w + dx * g.seg[0].stride) * cbytes;
+            }
+        }
         const int lag = g.stages >= 3 ? 2 : (g.stages == 2 ? 1 : 0);
-        int pend = 0, pend_first = 0;
+        int pend = 0, pend_first = 0, it = 0;
         auto retire_oldest = [&]() {
             fence_proxy_async();
             warp_arrive(full_bar(pend_first % g.stages), lane);
             ++pend_first; --pend;
         };
-        for (int kb = 0; kb < g.kblocks && ok; ++kb) {
-            int s = kb % g.stages;
-            uint32_t ph = (kb / g.stages) & 1;
-            ok = mbar_wait_warp(empty_bar(s), ph ^ 1u, lane);
-            if (!ok) break;
-            const bool first = kb < g.seg[0].kblocks;
-            const GemmSeg &sg = first ? g.seg[0] : g.seg[1];
-            const int kbl = first ? kb : kb - g.seg[0].kblocks;
-            uint32_t a_base = sbase + s * stage_bytes;
-            if (sg.mode == GA_GATHER) {
-                if (first) { produce_gather(sg, gs0, ri, a_base, grow, ghalf); gather_advance(gs0, 8, sg.C >> 3, sg.k); }
-                else { produce_gather(sg, gs1, ri, a_base, grow, ghalf); gather_advance(gs1, 8, sg.C >> 3, sg.k); }
-                cp_async_commit();
-                ++pend;
-                if (pend > lag) {
-                    if (lag == 2) cp_async_wait<2>(); else if (lag == 1) cp_async_wait<1>(); else cp_async_wait<0>();
-                    retire_oldest();
+        for (int ti = blockIdx.x; ti < total_tiles && ok; ti += gridDim.x) {
+            const int mt = ti / g.n_tiles;
+            RowPos rp;
+            rp.valid = 0; rp.n = 0; rp.p = 0; rp.q = 0;
+            if (!dw_mode) rp = map_row(g, mt, grow);
+            GatherState gs0 = {0, 0, 0}, gs1 = {0, 0, 0};
+            if (g.seg[0].mode == GA_GATHER && ghalf) gather_advance(gs0, 4, g.seg[0].C >> 3, g.seg[0].k);
+            if (g.seg[1].mode == GA_GATHER && ghalf) gather_advance(gs1, 4, g.seg[1].C >> 3, g.seg[1].k);
+            for (int kb = 0; kb < g.kblocks && ok; ++kb, ++it) {
+                const int s = it % g.stages;
+                ok = mbar_wait_warp(empty_bar(s), ((it / g.stages) & 1) ^ 1u, lane);
+                if (!ok) break;
+                const bool first = kb < g.seg[0].kblocks;
+                const GemmSeg &sg = first ? g.seg[0] : g.seg[1];
+                const int kbl = first ? kb : kb - g.seg[0].kblocks;
+                const uint32_t a_base = sbase + s * stage_bytes;
+                if (sg.mode == GA_GATHER) {
+                    if (first) { produce_gather(sg, gs0, rp, a_base, grow, ghalf); gather_advance(gs0, 8, sg.C >> 3, sg.k); }
+                    else { produce_gather(sg, gs1, rp, a_base, grow, ghalf); gather_advance(gs1, 8, sg.C >> 3, sg.k); }
+                    cp_async_commit();
+                    ++pend;
+                    if (pend > lag) {
+                        if (lag == 2) cp_async_wait<2>(); else if (lag == 1) cp_async_wait<1>(); else cp_async_wait<0>();
+                        retire_oldest();
+                    }
+                } else {
+                    if (pend) { cp_async_wait<0>(); while (pend) retire_oldest(); }
+                    pend_first = it + 1;
+                    if (sg.mode == GA_DW) {
+                        const int hs = it % g.hstages;
+                        ok = mbar_wait_warp(hfull_bar(hs), (it / g.hstages) & 1, lane);
+                        if (!ok) break;
+                        produce_dw(sg, g, kbl, sbase + g.off_halo + hs * g.halo_stride, hoff, a_base, dj, drg);
+                        fence_proxy_async();
+                        warp_arrive(full_bar(s), lane);
+                        warp_arrive(hempty_bar(hs), lane);     // the halo tile has been read
+                    } else {
+                        produce_stem(sg, kbl, rp, a_base, grow, ghalf);
+                        fence_proxy_async();
+                        warp_arrive(full_bar(s), lane);
+                    }
                 }
-            } else {
-                if (pend) { cp_async_wait<0>(); while (pend) retire_oldest(); }
-                pend_first = kb + 1;
-                if (sg.mode == GA_DW) produce_dw(sg, kbl, dr, a_base, dj, drg);
-                else produce_stem(sg, kbl, ri, a_base, grow, ghalf);
-                fence_proxy_async();
-                warp_arrive(full_bar(s), lane);
             }
         }
         cp_async_wait<0>();
         if (ok) { while (pend) retire_oldest(); }
         else if (lane == 0) atomicCAS(g.status, 0u, kStatusTimeout);
-
-        // ---- epilogue: warp w reads tensor-memory lanes 32*(w%4).., the two warps that share a
-        // lane quarter take alternate 16-column chunks ----
-        if (ok) ok = mbar_wait_warp(accum_bar, 0, lane);
-        if (!ok && lane == 0) atomicCAS(g.status, 0u, kStatusTimeout);
-        tc_fence_after();
-        const int quarter = warp & 3, chalf = (warp - 2) >> 2;
+    } else {
+        // ---- epilogue: warp w reads tensor-memory lanes 32*(w%4).. ----
+        const int quarter = warp & 3;
         const int row = quarter * 32 + lane;
-        const int4 rq = rowtab[row];
-        const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
-        const int n0 = nt * g.tile_n;
-        const int nchunks = g.tile_n / 16;
-        // staging for the pool / global-average epilogues reuses the pipeline buffers: every MMA has
-        // retired (accum barrier), so nothing reads or writes them any more
-        const uint32_t stg = sbase;
+        const int et = threadIdx.x - (64 + kProducerThreads);      // 0..127
+        const uint32_t stg = sbase + g.off_stg;
+        float *stgf = reinterpret_cast<float *>(sm + g.off_stg);
         const int pool_pitch = g.tile_n * 2 + 16;
-        const size_t pix = ((size_t)rq.y * g.P + rq.z) * g.Q + rq.w;
-        for (int c2 = 0; c2 * 2 < nchunks; ++c2) {
-            const int ch = c2 * 2 + chalf;
-            const bool live = ch < nchunks;
-            float v[16];
-            if (ok && live) tmem_ld16(t_lane + ch * 16, v);
-            else {
+        const int nchunks = g.tile_n / 16;
+        int i = 0;
+        for (int ti = blockIdx.x; ti < total_tiles; ti += gridDim.x, ++i) {
+            const int mt = ti / g.n_tiles, nt = ti - mt * g.n_tiles;
+            const int b = i & 1;
+            // the four epilogue warps share named barriers below, so they must agree on giving up
+            if (!mbar_wait_warp(accf_bar(b), (i >> 1) & 1, lane) && lane == 0) *fail_flag = 1;
+            epi_bar();
+            if (*fail_flag) { ok = false; break; }
+            tc_fence_after();
+            const RowPos rq = map_row(g, mt, row);
+            const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * g.acc_stride;
+            const int n0 = nt * g.tile_n;
+            const size_t pix = ((size_t)rq.n * g.P + rq.p) * g.Q + rq.q;
+            for (int ch = 0; ch < nchunks; ++ch) {
+                float v[16];
+                tmem_ld16(t_lane + ch * 16, v);
+                if (ch == nchunks - 1) {
+                    // every column of this accumulator is in registers: hand it back to the MMA warp
+                    tc_fence_before();
+                    warp_arrive(acce_bar(b), lane);
+                }
+                const int nc = n0 + ch * 16;
 #pragma unroll
-                for (int i = 0; i < 16; ++i) v[i] = 0.0f;
-            }
-            const int nc = n0 + ch * 16;
-            if (live) {
-#pragma unroll
-                for (int i = 0; i < 16; i += 4) {
-                    const float4 b = __ldg(reinterpret_cast<const float4 *>(g.bias + nc + i));   // bias is padded to npad
-                    v[i] = apply_act(v[i] + b.x, g.act); v[i + 1] = apply_act(v[i + 1] + b.y, g.act);
-                    v[i + 2] = apply_act(v[i + 2] + b.z, g.act); v[i + 3] = apply_act(v[i + 3] + b.w, g.act);
+                for (int q4 = 0; q4 < 16; q4 += 4) {
+                    const float4 bz = __ldg(reinterpret_cast<const float4 *>(g.bias + nc + q4));   // bias is padded to npad
+                    v[q4] = apply_act(v[q4] + bz.x, g.act); v[q4 + 1] = apply_act(v[q4 + 1] + bz.y, g.act);
+                    v[q4 + 2] = apply_act(v[q4 + 2] + bz.z, g.act); v[q4 + 3] = apply_act(v[q4 + 3] + bz.w, g.act);
                 }
                 // shortcut connection with an identity branch: the skip tile is read once, here
-                if (g.skip && rq.x) {
+                if (g.skip && rq.valid) {
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
                         if (nc + h * 8 + 8 > g.N) break;
-                        f8 sv = unpack8(__ldg(reinterpret_cast<const uint4 *>(g.skip + pix * g.skip_ctot + nc + h * 8)));
+                        const f8 sv = unpack8(__ldg(reinterpret_cast<const uint4 *>(g.skip + pix * g.skip_ctot + nc + h * 8)));
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) v[h * 8 + i] += sv.v[i];
+                        for (int c = 0; c < 8; ++c) v[h * 8 + c] += sv.v[c];
                     }
                 }
                 if (g.act2) {
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) v[i] = apply_act(v[i], g.act2);
+                    for (int c = 0; c < 16; ++c) v[c] = apply_act(v[c], g.act2);
                 }
-            }
-            if (g.epi == GE_STORE) {
-                if (!rq.x || !ok || !live) continue;
-                if (g.out_f32) {
-                    float *o = reinterpret_cast<float *>(g.out) + pix * g.out_ctot + g.out_coff + nc;
+                if (g.epi == GE_STORE) {
+                    if (!rq.valid) continue;
+                    if (g.out_f32) {
+                        float *o = reinterpret_cast<float *>(g.out) + pix * g.out_ctot + g.out_coff + nc;
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) if (nc + i < g.N) o[i] = v[i];
+                        for (int c = 0; c < 16; ++c) if (nc + c < g.N) o[c] = v[c];
+                    } else {
+                        __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(g.out) + pix * g.out_ctot + g.out_coff + nc;
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            if (nc + h * 8 + 8 > g.N) break;
+                            f8 pv;
+#pragma unroll
+                            for (int c = 0; c < 8; ++c) pv.v[c] = v[h * 8 + c];
+                            *reinterpret_cast<uint4 *>(o + h * 8) = pack8(pv);
+                        }
+                    }
+                } else if (g.epi == GE_POOL) {
+                    // rows outside the conv output never win a max
+                    f8 lo, hi;
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) { lo.v[c] = rq.valid ? v[c] : -INFINITY; hi.v[c] = rq.valid ? v[8 + c] : -INFINITY; }
+                    st_shared16(stg + row * pool_pitch + ch * 32, pack8(lo));
+                    st_shared16(stg + row * pool_pitch + ch * 32 + 16, pack8(hi));
                 } else {
-                    __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(g.out) + pix * g.out_ctot + g.out_coff + nc;
+                    // global average: 16 columns at a time through shared memory, rows summed in ascending order
+                    epi_bar();
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        if (nc + h * 8 + 8 > g.N) break;
-                        f8 pv;
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) pv.v[i] = v[h * 8 + i];
-                        *reinterpret_cast<uint4 *>(o + h * 8) = pack8(pv);
+                    for (int c = 0; c < 16; ++c) stgf[row * 17 + c] = rq.valid ? v[c] : 0.0f;
+                    epi_bar();
+                    for (int item = et; item < g.gap_imgs * 16; item += kEpilogueThreads) {
+                        const int img = item >> 4, c = item & 15;
+                        const int n = mt * g.gap_imgs + img;
+                        if (n >= g.batch || nc + c >= g.N) continue;
+                        float acc = 0.0f;
+                        for (int r = 0; r < g.gap_rpi; ++r) acc += stgf[(img * g.gap_rpi + r) * 17 + c];
+                        acc /= (float)g.gap_rpi;
+                        const size_t oi = (size_t)n * g.out_ctot + g.out_coff + nc + c;
+                        if (g.out_f32) reinterpret_cast<float *>(g.out)[oi] = acc;
+                        else reinterpret_cast<__nv_bfloat16 *>(g.out)[oi] = __float2bfloat16_rn(acc);
                     }
                 }
-            } else if (g.epi == GE_POOL) {
-                if (!live) continue;
-                // rows outside the conv output never win a max
-                f8 lo, hi;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) { lo.v[i] = rq.x ? v[i] : -INFINITY; hi.v[i] = rq.x ? v[8 + i] : -INFINITY; }
-                st_shared16(stg + row * pool_pitch + ch * 32, pack8(lo));
-                st_shared16(stg + row * pool_pitch + ch * 32 + 16, pack8(hi));
-            } else {
-                // global average: two 16-column chunks at a time through shared memory, rows summed in ascending order
+            }
+            if (g.epi == GE_POOL) {
                 epi_bar();
-                float *sf = reinterpret_cast<float *>(sm) + chalf * (kTileM * 17);
+                const int per = g.tiles_y * g.tiles_x;
+                const int n = mt / per, tt = mt - n * per;
+                const int ty = tt / g.tiles_x, tx = tt - ty * g.tiles_x;
+                const int c8n = g.tile_n / 8;
+                for (int item = et; item < g.pth * g.ptw * c8n; item += kEpilogueThreads) {
+                    const int c8 = item % c8n, o = item / c8n;
+                    const int oy = o / g.ptw, ox = o - oy * g.ptw;
+                    const int gy = ty * g.pth + oy, gx = tx * g.ptw + ox;
+                    const int col = n0 + c8 * 8;
+                    if (gy >= g.PP || gx >= g.PQ || col + 8 > g.N || n >= g.batch) continue;
+                    f8 m;
 #pragma unroll
-                for (int i = 0; i < 16; ++i) sf[row * 17 + i] = (rq.x && live) ? v[i] : 0.0f;
-                epi_bar();
-                for (int item = threadIdx.x - 64; item < g.imgs_per_tile * 32; item += kProducerThreads) {
-                    const int img = item >> 5, c = item & 31;
-                    const int n = mt * g.imgs_per_tile + img;
-                    const int col = n0 + c2 * 32 + c;
-                    if (n >= g.batch || col >= g.N || c2 * 2 + (c >> 4) >= nchunks || !ok) continue;
-                    const float *sc = reinterpret_cast<float *>(sm) + (c >> 4) * (kTileM * 17) + (c & 15);
-                    float acc = 0.0f;
-                    for (int r = 0; r < g.rpi; ++r) acc += sc[(img * g.rpi + r) * 17];
-                    acc /= (float)g.rpi;
-                    const size_t oi = (size_t)n * g.out_ctot + g.out_coff + col;
-                    if (g.out_f32) reinterpret_cast<float *>(g.out)[oi] = acc;
-                    else reinterpret_cast<__nv_bfloat16 *>(g.out)[oi] = __float2bfloat16_rn(acc);
+                    for (int c = 0; c < 8; ++c) m.v[c] = -INFINITY;
+                    for (int dy = 0; dy < g.pool_k; ++dy)
+                        for (int dx = 0; dx < g.pool_k; ++dx) {
+                            const int r = (oy * g.pool_stride + dy) * g.rw + ox * g.pool_stride + dx;
+                            const f8 xv = unpack8(ld_shared16(stg + r * pool_pitch + c8 * 16));
+#pragma unroll
+                            for (int c = 0; c < 8; ++c) m.v[c] = fmaxf(m.v[c], xv.v[c]);
+                        }
+                    __nv_bfloat16 *o2 = reinterpret_cast<__nv_bfloat16 *>(g.out) +
+                                        (((size_t)n * g.PP + gy) * g.PQ + gx) * g.out_ctot + g.out_coff + col;
+                    *reinterpret_cast<uint4 *>(o2) = pack8(m);
                 }
+                epi_bar();          // the staging tile is free for the next tile
             }
         }
-        if (g.epi == GE_POOL) {
-            epi_bar();
-            const int per = g.tiles_y * g.tiles_x;
-            const int n = mt / per, tt = mt - n * per;
-            const int ty = tt / g.tiles_x, tx = tt - ty * g.tiles_x;
-            const int c8n = g.tile_n / 8;
-            for (int item = threadIdx.x - 64; item < g.th * g.tw * c8n; item += kProducerThreads) {
-                const int c8 = item % c8n, o = item / c8n;
-                const int oy = o / g.tw, ox = o - oy * g.tw;
-                const int gy = ty * g.th + oy, gx = tx * g.tw + ox;
-                const int col = n0 + c8 * 8;
-                if (gy >= g.PP || gx >= g.PQ || col + 8 > g.N || n >= g.batch || !ok) continue;
-                f8 m;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) m.v[i] = -INFINITY;
-                for (int dy = 0; dy < g.pool_k; ++dy)
-                    for (int dx = 0; dx < g.pool_k; ++dx) {
-                        const int r = (oy * g.pool_stride + dy) * g.rw + ox * g.pool_stride + dx;
-                        const f8 xv = unpack8(ld_shared16(stg + r * pool_pitch + c8 * 16));
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) m.v[i] = fmaxf(m.v[i], xv.v[i]);
-                    }
-                __nv_bfloat16 *o2 = reinterpret_cast<__nv_bfloat16 *>(g.out) +
-                                    (((size_t)n * g.PP + gy) * g.PQ + gx) * g.out_ctot + g.out_coff + col;
-                *reinterpret_cast<uint4 *>(o2) = pack8(m);
-            }
-        }
+        if (!ok && lane == 0) atomicCAS(g.status, 0u, kStatusTimeout);
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)g.tmem_cols) : "memory");
     }
 }
 

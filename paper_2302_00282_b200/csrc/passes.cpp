@@ -605,6 +605,9 @@ struct Lower {
             if (!pool_patch(pooln->k, pooln->stride, po.h, po.w, L.patch_th, L.patch_tw, L.patch_rh, L.patch_rw))
                 return fail(g, XENOS_E_UNSUPPORTED, "internal: pool patch does not fit");
             L.tiles_y = ceil_div(po.h, L.patch_th); L.tiles_x = ceil_div(po.w, L.patch_tw);
+            L.ni = 1;
+            L.step_y = L.patch_th * pooln->stride; L.step_x = L.patch_tw * pooln->stride;
+            L.off_y = L.off_x = pooln->pad;
             L.tile_rows = L.patch_rh * L.patch_rw;
         }
         if (gapn) {
@@ -612,6 +615,40 @@ struct Lower {
             L.epi = EPI_GAP;
             L.imgs_per_tile = 128 / L.rows_per_image;
             L.tile_rows = L.imgs_per_tile * L.rows_per_image;
+            L.gap_imgs = L.imgs_per_tile; L.gap_rpi = L.rows_per_image;
+        }
+        if (dw) {
+            // The depthwise stage reads a halo tile that TMA fetches as one 4-D box, so the tile is a
+            // patch: ni whole images when an image fits 128 rows, else th x tw output pixels of one image.
+            L.map_mode = MAP_PATCH;
+            if (L.rows_per_image <= 128) {
+                L.ni = 128 / L.rows_per_image; L.patch_rh = L.P; L.patch_rw = L.Q;
+            } else {
+                if (gapn) return fail(g, XENOS_E_UNSUPPORTED, "internal: global average needs whole images per tile");
+                L.ni = 1;
+                long best = -1;
+                for (int tw = 1; tw <= std::min(L.Q, 128); ++tw) {
+                    int th = std::min(L.P, 128 / tw);
+                    long tiles = (long)ceil_div(L.P, th) * ceil_div(L.Q, tw);
+                    // fewest tiles first; then the widest tile (longest contiguous rows in memory)
+                    if (best < 0 || tiles < best || (tiles == best && tw > L.patch_rw)) { best = tiles; L.patch_rh = th; L.patch_rw = tw; }
+                }
+            }
+            // keep one halo tile (64 channels of the input window) small enough for a 2-3 deep ring
+            auto halo_of = [&](int ni, int th, int tw) {
+                return (long)ni * ((th - 1) * dw->stride + 3) * ((tw - 1) * dw->stride + 3) * std::min(64, src.c) * 2;
+            };
+            while (L.ni > 1 && halo_of(L.ni, L.patch_rh, L.patch_rw) > 40 * 1024) --L.ni;
+            while (!gapn && L.patch_rh > 1 && halo_of(L.ni, L.patch_rh, L.patch_rw) > 76 * 1024) --L.patch_rh;
+            L.tiles_y = ceil_div(L.P, L.patch_rh); L.tiles_x = ceil_div(L.Q, L.patch_rw);
+            L.step_y = L.patch_rh; L.step_x = L.patch_rw; L.off_y = L.off_x = 0;
+            L.tile_rows = L.ni * L.patch_rh * L.patch_rw;
+            L.halo_h = (L.patch_rh - 1) * dw->stride + 3; L.halo_w = (L.patch_rw - 1) * dw->stride + 3;
+            L.halo_cb = std::min(64, src.c);
+            L.halo_bytes = L.ni * L.halo_h * L.halo_w * L.halo_cb * 2;
+            L.halo_stride = (int)align_up((size_t)L.halo_bytes, 128);
+            if (L.halo_h > 256 || L.halo_w > 256) return fail(g, XENOS_E_UNSUPPORTED, "internal: halo tile exceeds the TMA box limit");
+            if (gapn) { L.gap_imgs = L.ni; L.gap_rpi = L.rows_per_image; }
         }
         L.out = last->out;
         const Tensor &ot = g.tensors[L.out];
@@ -621,9 +658,9 @@ struct Lower {
         // --- split (Section 4.2.1: output channels first, then rows / columns of the feature map)
         const SplitRequest &rq = ch.split;
         int N16 = round_up(N, 16);
-        if (L.epi == EPI_STORE) L.m_tiles = ceil_div(g.max_batch * L.rows_per_image, 128);
+        if (L.map_mode == MAP_PATCH) L.m_tiles = ceil_div(g.max_batch, L.ni) * L.tiles_y * L.tiles_x;
         else if (L.epi == EPI_GAP) L.m_tiles = ceil_div(g.max_batch, L.imgs_per_tile);
-        else L.m_tiles = g.max_batch * L.tiles_y * L.tiles_x;
+        else L.m_tiles = ceil_div(g.max_batch * L.rows_per_image, 128);
         if (rq.user && (rq.h > 1 || rq.w > 1))
             return fail(g, XENOS_E_BAD_SPLIT, "split: tensor-core chains cut rows / columns into 128-row tiles themselves; only parts_outc can be set");
         if (rq.user && rq.outc > 0) {
@@ -635,27 +672,37 @@ struct Lower {
             L.n_tiles = ceil_div(N16, 256);
             L.tile_n = round_up(ceil_div(N16, L.n_tiles), 16);
             // kernels are dealt to idle units first: halve the channel tile while units stay idle
-            while (L.m_tiles * L.n_tiles < g.hw.sm_count && L.tile_n >= 64) {
+            // (a linked depthwise stage is recomputed per channel tile, so it stops halving earlier)
+            const int min_tile_n = dw ? 128 : 32;
+            while (L.m_tiles * L.n_tiles < g.hw.sm_count && L.tile_n >= 2 * min_tile_n) {
                 int nt = L.n_tiles * 2, tn = round_up(ceil_div(N16, nt), 16);
                 if ((nt - 1) * tn >= N) break;
                 L.n_tiles = nt; L.tile_n = tn;
             }
         }
         L.npad = L.n_tiles * L.tile_n;
+        // two accumulators in tensor memory so the epilogue of one tile overlaps the MMAs of the next
+        L.acc_stride = round_up(L.tile_n, 32);
         L.tmem_cols = 32;
-        while (L.tmem_cols < L.tile_n) L.tmem_cols *= 2;
-        if (L.tmem_cols > g.hw.tmem_columns) return fail(g, XENOS_E_BAD_SPLIT, "split: accumulator tile exceeds tensor memory columns");
+        while (L.tmem_cols < 2 * L.acc_stride) L.tmem_cols *= 2;
+        if (L.tmem_cols > g.hw.tmem_columns) return fail(g, XENOS_E_BAD_SPLIT, "split: accumulator tiles exceed tensor memory columns");
+        // shared memory of the one persistent CTA per SM: [A|B ring][halo ring][epilogue staging][barriers]
         int stage_bytes = 16384 + L.tile_n * 128;
-        int budget = std::min(g.hw.smem_bytes_per_cta, 227 * 1024) / 2 - 4096;   // two CTAs per SM overlap epilogue and main loop
-        L.stages = std::max(2, std::min(6, budget / stage_bytes));
-        L.stages = std::max(1, std::min(L.stages, L.kblocks));
-        // the pool / global-average epilogues stage the tile in the (by then idle) pipeline buffers
-        int staging = L.epi == EPI_POOL ? 128 * (L.tile_n * 2 + 16) : (L.epi == EPI_GAP ? 2 * 128 * 17 * 4 : 0);
-        L.pipe_bytes = (int)align_up((size_t)std::max(L.stages * stage_bytes, staging), 1024);
-        L.smem_bytes = L.pipe_bytes + 128 + 2048 + 1024;     // + barriers, row table, alignment slack
-        if (L.smem_bytes > g.hw.smem_bytes_per_cta) return fail(g, XENOS_E_BAD_SPLIT, "split: pipeline does not fit shared memory");
-        L.grid = L.m_tiles * L.n_tiles;
-        L.block = 320;
+        int stg_bytes = L.epi == EPI_POOL ? 128 * (L.tile_n * 2 + 16) : (L.epi == EPI_GAP ? 128 * 17 * 4 : 0);
+        stg_bytes = (int)align_up((size_t)stg_bytes, 128);
+        int cap = std::min(g.hw.smem_bytes_per_cta, 227 * 1024) - 1024 - 256;
+        L.hstages = dw ? 2 : 0;
+        if (dw && cap - stg_bytes - 3 * L.halo_stride >= 3 * stage_bytes) L.hstages = 3;
+        int room = cap - stg_bytes - L.hstages * L.halo_stride;
+        L.stages = std::min(6, room / stage_bytes);
+        if (L.stages < 1) return fail(g, XENOS_E_BAD_SPLIT, "split: pipeline does not fit shared memory");
+        L.off_halo = L.stages * stage_bytes;
+        L.off_stg = L.off_halo + L.hstages * L.halo_stride;
+        L.off_bar = (int)align_up((size_t)(L.off_stg + stg_bytes), 128);
+        L.pipe_bytes = L.off_bar;
+        L.smem_bytes = L.off_bar + 256 + 1024;     // + barriers, alignment slack
+        L.grid = std::min(L.m_tiles * L.n_tiles, g.hw.sm_count);
+        L.block = 448;
         // --- pack weights + bias
         L.w_off = blob_reserve(g, (size_t)L.npad * L.kpad * 2);
         L.b_off = blob_reserve(g, (size_t)L.npad * 4);
@@ -924,7 +971,10 @@ void emit_plan_json(Graph &g) {
             jint(s, "imgs_per_tile", L.imgs_per_tile);
             jint(s, "patch_th", L.patch_th); jint(s, "patch_tw", L.patch_tw); jint(s, "patch_rh", L.patch_rh);
             jint(s, "patch_rw", L.patch_rw); jint(s, "tiles_y", L.tiles_y); jint(s, "tiles_x", L.tiles_x);
-            jint(s, "stages", L.stages); jint(s, "tmem_cols", L.tmem_cols);
+            jint(s, "stages", L.stages); jint(s, "tmem_cols", L.tmem_cols); jint(s, "acc_stride", L.acc_stride);
+            jint(s, "ni", L.ni); jint(s, "step_y", L.step_y); jint(s, "step_x", L.step_x); jint(s, "off_y", L.off_y); jint(s, "off_x", L.off_x);
+            jint(s, "hstages", L.hstages); jint(s, "halo_h", L.halo_h); jint(s, "halo_w", L.halo_w); jint(s, "halo_cb", L.halo_cb);
+            jint(s, "halo_bytes", L.halo_bytes);
         }
         if (L.kind == LK_F32_CONV_CONV_POOL) {
             jint(s, "parts_outc", L.parts_outc); jint(s, "tile_h", L.tile_h); jint(s, "tile_w", L.tile_w);

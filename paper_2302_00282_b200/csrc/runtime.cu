@@ -22,6 +22,7 @@ struct Runtime {
     int device = -1;
     int sm_count = 0;
     std::vector<CUtensorMap> tmaps;     // one per launch record (used by gemm launches only)
+    std::vector<CUtensorMap> hmaps;     // halo maps of linked depthwise stages
     PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
 };
 
@@ -38,6 +39,23 @@ static uint32_t make_idesc(int tile_n) {
     d |= (uint32_t)(tile_n >> 3) << 17; // N / 8
     d |= (uint32_t)(128 >> 4) << 24;    // M / 16
     return d;
+}
+
+// 4-D map (C, W, H, N) over the NHWC bf16 input of a linked depthwise stage; box = one halo tile.
+// Out-of-range coordinates read zeros, which is the convolution's zero padding.
+static xenos_status_t encode_halo_map(const Graph &g, Runtime *rt, const Launch &L, void *base, CUtensorMap *out) {
+    const ASeg &a = L.seg[0];
+    cuuint64_t dims[4] = {(cuuint64_t)a.C, (cuuint64_t)a.W, (cuuint64_t)a.H, (cuuint64_t)g.max_batch};
+    cuuint64_t strides[3] = {(cuuint64_t)a.C * 2, (cuuint64_t)a.W * a.C * 2, (cuuint64_t)a.H * a.W * a.C * 2};
+    cuuint32_t box[4] = {(cuuint32_t)L.halo_cb, (cuuint32_t)L.halo_w, (cuuint32_t)L.halo_h, (cuuint32_t)L.ni};
+    cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+    if (((uintptr_t)base & 15u) || (strides[0] & 15u) || (box[0] * 2u) % 16u || box[1] > 256u || box[2] > 256u || box[3] > 256u)
+        return fail(g, XENOS_E_CUDA, "depthwise input is not 16-byte aligned or its halo tile exceeds the TMA box limits");
+    CUresult r = rt->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, estr,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(g, XENOS_E_CUDA, "cuTensorMapEncodeTiled (halo) failed with code " + std::to_string((int)r));
+    return XENOS_OK;
 }
 
 void runtime_free(Graph &g) {
@@ -75,6 +93,7 @@ xenos_status_t runtime_bind(Graph &g, void *ws, size_t bytes, void *stream_v) {
         if (L.kind == LK_F32_CONV_CONV_POOL) max_chain_smem = std::max(max_chain_smem, L.smem_bytes);
     }
     rt->tmaps.resize(g.launches.size());
+    rt->hmaps.resize(g.launches.size());
     if (any_gemm) {
         void *fn = nullptr;
         cudaDriverEntryPointQueryResult qres;
@@ -97,6 +116,10 @@ xenos_status_t runtime_bind(Graph &g, void *ws, size_t bytes, void *stream_v) {
                                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
             if (r != CUDA_SUCCESS) return fail(g, XENOS_E_CUDA, "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r));
+            if (L.seg[0].mode == AM_DW && g.tensors[L.seg[0].tensor].input_slot < 0) {
+                xenos_status_t st = encode_halo_map(g, rt, L, static_cast<uint8_t *>(ws) + g.place[L.seg[0].tensor].off, &rt->hmaps[i]);
+                if (st != XENOS_OK) return st;
+            }
         }
     }
     // The opt-in limit is a per-function, per-device setting shared by every graph in the process:
@@ -235,18 +258,38 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
             p.skip_ctot = L.skip >= 0 ? g.tensors[L.skip].c : 0;
             p.out = ptr(L.out); p.status = status;
             p.batch = N; p.P = L.P; p.Q = L.Q; p.rpi = L.rows_per_image;
-            p.map_mode = L.map_mode; p.tile_rows = L.tile_rows; p.imgs_per_tile = L.imgs_per_tile;
-            p.th = L.patch_th; p.tw = L.patch_tw; p.rh = L.patch_rh; p.rw = L.patch_rw; p.tiles_y = L.tiles_y; p.tiles_x = L.tiles_x;
-            p.pool_k = L.pool_k; p.pool_stride = L.pool_stride; p.pool_pad = L.pool_pad; p.PP = L.PP; p.PQ = L.PQ;
-            p.kblocks = L.kblocks; p.stages = L.stages; p.pipe_bytes = L.pipe_bytes; p.tile_n = L.tile_n; p.n_tiles = L.n_tiles; p.N = L.K;
+            p.map_mode = L.map_mode; p.tile_rows = L.tile_rows;
+            p.ni = L.ni; p.rh = L.patch_rh; p.rw = L.patch_rw; p.tiles_y = L.tiles_y; p.tiles_x = L.tiles_x;
+            p.step_y = L.step_y; p.step_x = L.step_x; p.off_y = L.off_y; p.off_x = L.off_x;
+            p.pool_k = L.pool_k; p.pool_stride = L.pool_stride; p.PP = L.PP; p.PQ = L.PQ; p.pth = L.patch_th; p.ptw = L.patch_tw;
+            p.gap_imgs = L.gap_imgs; p.gap_rpi = L.gap_rpi;
+            p.kblocks = L.kblocks; p.stages = L.stages; p.tile_n = L.tile_n; p.n_tiles = L.n_tiles; p.N = L.K;
+            p.acc_stride = L.acc_stride; p.tmem_cols = L.tmem_cols;
+            p.hstages = L.hstages; p.halo_bytes = L.halo_bytes; p.halo_stride = L.halo_stride;
+            p.halo_h = L.halo_h; p.halo_w = L.halo_w; p.halo_cb = L.halo_cb;
+            p.off_halo = L.off_halo; p.off_stg = L.off_stg; p.off_bar = L.off_bar;
             p.act = L.act; p.act2 = L.act2; p.epi = L.epi; p.out_ctot = L.out_ctot; p.out_coff = L.out_coff;
             p.out_f32 = L.out_dtype == XENOS_DTYPE_F32;
             p.idesc = make_idesc(L.tile_n);
-            int m_tiles;
-            if (L.epi == EPI_POOL) m_tiles = N * L.tiles_y * L.tiles_x;
-            else if (L.epi == EPI_GAP) m_tiles = (N + L.imgs_per_tile - 1) / L.imgs_per_tile;
-            else m_tiles = (int)(((long long)N * L.rows_per_image + 127) / 128);
-            xk::gemm_chain_kernel<<<m_tiles * L.n_tiles, xk::kThreads, L.smem_bytes, stream>>>(rt->tmaps[li], p);
+            if (L.map_mode == MAP_PATCH) p.m_tiles = ((N + L.ni - 1) / L.ni) * L.tiles_y * L.tiles_x;
+            else if (L.epi == EPI_GAP) p.m_tiles = (N + L.imgs_per_tile - 1) / L.imgs_per_tile;
+            else p.m_tiles = (int)(((long long)N * L.rows_per_image + 127) / 128);
+            // the halo tensor map of a linked depthwise stage points at the stage's input; when that
+            // is a caller buffer its address is only known now
+            const CUtensorMap *tmh = &rt->tmaps[li];
+            CUtensorMap tmh_now;
+            if (L.seg[0].mode == AM_DW) {
+                const Tensor &hx = g.tensors[L.seg[0].tensor];
+                if (hx.input_slot >= 0) {
+                    xenos_status_t st = encode_halo_map(g, rt, L, ptr(L.seg[0].tensor), &tmh_now);
+                    if (st != XENOS_OK) return st;
+                    tmh = &tmh_now;
+                } else {
+                    tmh = &rt->hmaps[li];
+                }
+            }
+            const int grid = std::min(p.m_tiles * L.n_tiles, sms);
+            xk::gemm_chain_kernel<<<grid, xk::kThreads, L.smem_bytes, stream>>>(rt->tmaps[li], *tmh, p);
             break;
         }
         default:

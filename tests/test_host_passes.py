@@ -265,11 +265,15 @@ def test_gemm_split_prefers_output_channels_until_units_are_busy():
                 continue
             assert L["tile_n"] % 16 == 0 and 16 <= L["tile_n"] <= 256
             assert L["npad"] == L["tile_n"] * L["n_tiles"] and (L["n_tiles"] - 1) * L["tile_n"] < L["K"] <= L["npad"]
-            assert L["grid"] == L["m_tiles"] * L["n_tiles"]
+            assert L["grid"] == min(148, L["m_tiles"] * L["n_tiles"])     # one persistent CTA per unit
             if L["n_tiles"] > -(-L["K"] // 256):               # split finer than the 256-wide maximum
                 assert L["m_tiles"] * (L["n_tiles"] // 2) < 148   # ... only because units would idle otherwise
-            assert L["tmem_cols"] >= L["tile_n"] and 1 <= L["stages"] <= max(1, L["kblocks"])
+                if L["a0"] == "dw":
+                    assert L["tile_n"] >= 128                  # a linked depthwise stage is recomputed per channel tile
+            assert L["tmem_cols"] >= 2 * L["tile_n"] and 1 <= L["stages"] <= 6
             assert L["smem_bytes"] <= 227 * 1024
+            if L["a0"] == "dw":
+                assert L["ni"] * L["patch_rh"] * L["patch_rw"] <= 128 and L["hstages"] >= 2
     g, ids = compiled(spec, 32, splits=[("pw7.relu6", dict(parts_outc=4))])
     L = [l for l in g.plan()["launches"] if l["kind"] == "gemm" and l["K"] == 512][1]
     hw = xb.HwInfo(16, 227 * 1024, 512, 1 << 20)
