@@ -67,11 +67,11 @@ struct GemmParams {
     // PATCH tiles: ni images x rh x rw positions of the conv output, origin (ty*step_y - off_y, tx*step_x - off_x)
     int ni, rh, rw, tiles_y, tiles_x, step_y, step_x, off_y, off_x;
     int pool_k, pool_stride, PP, PQ, pth, ptw;     // max-pool epilogue: pth x ptw pool outputs per tile
-    int gap_imgs, gap_rpi;                         // global-average epilogue: whole images per tile
+    int gap_imgs, gap_area, gap_rpi;               // global-average epilogue: whole images per tile (area rows each, rpi of them real)
     int kblocks, stages, tile_n, n_tiles, m_tiles, N;
     int acc_stride, tmem_cols;                     // two accumulators, acc_stride columns apart
     int hstages, halo_bytes, halo_stride, halo_h, halo_w, halo_cb;   // depthwise halo ring
-    int off_halo, off_stg, off_bar;                // shared-memory offsets from the 1024-aligned base
+    int off_halo, off_stg, off_dww, off_bias, off_bar;   // shared-memory offsets from the 1024-aligned base
     int act, act2, epi, out_ctot, out_coff, out_f32, skip_ctot;
     uint32_t idesc;
 };
@@ -127,6 +127,11 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 __device__ __forceinline__ void st_shared16(uint32_t dst, const uint4 &v) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
+__device__ __forceinline__ float4 ld_shared_f4(uint32_t src) {
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(src));
+    return v;
+}
 __device__ __forceinline__ uint4 ld_shared16(uint32_t src) {
     uint4 v;
     asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(src));
@@ -179,6 +184,21 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float *v) {
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float *v) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 // ---- row <-> pixel -----------------------------------------------------------------------------
@@ -188,10 +208,10 @@ __device__ __forceinline__ RowPos map_row(const GemmParams &g, int mt, int r) {
     RowPos o;
     o.valid = 0; o.n = 0; o.p = 0; o.q = 0;
     if (g.map_mode == GM_FLAT) {
-        long long m = (long long)mt * g.tile_rows + r;
-        if (r < g.tile_rows && m < (long long)g.batch * g.rpi) {
-            o.n = (int)(m / g.rpi);
-            int rem = (int)(m - (long long)o.n * g.rpi);
+        const unsigned m = (unsigned)mt * (unsigned)g.tile_rows + (unsigned)r;     // < 2^31 rows by construction
+        if (r < g.tile_rows && m < (unsigned)g.batch * (unsigned)g.rpi) {
+            o.n = (int)(m / (unsigned)g.rpi);
+            const int rem = (int)(m - (unsigned)o.n * (unsigned)g.rpi);
             o.p = rem / g.Q; o.q = rem - o.p * g.Q;
             o.valid = 1;
         }
@@ -208,6 +228,10 @@ __device__ __forceinline__ RowPos map_row(const GemmParams &g, int mt, int r) {
     }
     return o;
 }
+
+// activation as a clamp: none = (-inf, +inf), ReLU = [0, +inf), ReLU6 = [0, 6]
+__device__ __forceinline__ float act_lo(int act) { return act >= 1 ? 0.0f : -INFINITY; }
+__device__ __forceinline__ float act_hi(int act) { return act == 2 ? 6.0f : INFINITY; }
 
 // ---- A-operand producers ------------------------------------------------------------------------
 // A stage is 128 rows x 128 bytes; 16-byte chunk j of row r sits at r*128 + ((j ^ (r & 7)) << 4),
@@ -250,80 +274,107 @@ __device__ __forceinline__ void produce_gather(const GemmSeg &sg, GatherState st
     }
 }
 
-// stem: K element e = (r * k + s) * C + c of an NCHW image (fp32 or bf16); thread = (row, half)
+// stem: K element e = (r * k + s) * C + c of an NCHW image (fp32 or bf16); thread = (row, half) and
+// takes the chunks j = 2*i + half so that both halves share the real (non-padding) elements.  All
+// loads of a chunk pair are issued before any is used.
 __device__ __forceinline__ void produce_stem(const GemmSeg &sg, int kb_local, const RowPos &rp, uint32_t a_base,
                                              int row, int half) {
-    int e = kb_local * kTileK + half * 32;
-    int tap = e / sg.C, c = e - tap * sg.C;
-    int r = tap / sg.k, s = tap - r * sg.k;
     const int ih0 = rp.p * sg.stride - sg.pad, iw0 = rp.q * sg.stride - sg.pad;
     const size_t img = (size_t)rp.n * sg.C * sg.H * sg.W;
     const float *sf = reinterpret_cast<const float *>(sg.src) + img;
-    const __nv_bfloat16 *sh = reinterpret_cast<const __nv_bfloat16 *>(sg.src) + img;
-#pragma unroll 1
-    for (int j = 0; j < 4; ++j) {
-        f8 v;
+    const unsigned short *sh = reinterpret_cast<const unsigned short *>(sg.src) + img;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            float x = 0.0f;
-            if (rp.valid && r < sg.k) {
-                int ih = ih0 + r, iw = iw0 + s;
-                if (ih >= 0 && ih < sg.H && iw >= 0 && iw < sg.W) {
-                    int off = (c * sg.H + ih) * sg.W + iw;
-                    x = sg.src_f32 ? __ldg(sf + off) : __bfloat162float(sh[off]);
+    for (int pair = 0; pair < 2; ++pair) {
+        float x[16];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int j = 2 * (2 * pair + u) + half;
+            int e = kb_local * kTileK + j * 8;
+            int tap = e / sg.C, c = e - tap * sg.C;
+            int r = tap / sg.k, s = tap - r * sg.k;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                float v = 0.0f;
+                if (rp.valid && r < sg.k) {
+                    const int ih = ih0 + r, iw = iw0 + s;
+                    if (ih >= 0 && ih < sg.H && iw >= 0 && iw < sg.W) {
+                        const int off = (c * sg.H + ih) * sg.W + iw;
+                        v = sg.src_f32 ? __ldg(sf + off) : __uint_as_float((unsigned)__ldg(sh + off) << 16);
+                    }
                 }
+                x[u * 8 + i] = v;
+                if (++c == sg.C) { c = 0; if (++s == sg.k) { s = 0; ++r; } }
             }
-            v.v[i] = x;
-            if (++c == sg.C) { c = 0; if (++s == sg.k) { s = 0; ++r; } }
         }
-        st_shared16(a_chunk_addr(a_base, row, half * 4 + j), pack8(v));
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            f8 v;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v.v[i] = x[u * 8 + i];
+            st_shared16(a_chunk_addr(a_base, row, 2 * (2 * pair + u) + half), pack8(v));
+        }
     }
 }
 
 // depthwise 3x3 + bias + activation from the halo tile in shared memory ([image][y][x][cb channels],
-// dense), rounded to bf16 and stored in the consumer's operand layout.
-// thread = (chunk j of 8 channels, row group); it owns rows rg, rg+32, rg+64, rg+96 so that the nine
-// tap weights of its 8 channels are fetched once per K block.
-__device__ __forceinline__ void produce_dw(const GemmSeg &sg, const GemmParams &g, int kb_local, uint32_t halo,
-                                           const int (&hoff)[4], uint32_t a_base, int j, int rg) {
-    const int c0 = kb_local * kTileK + j * 8;
-    const int cbytes = g.halo_cb * 2;
-    if (c0 >= sg.C || j * 8 >= g.halo_cb) {
+// dense bf16), rounded to bf16 and stored in the consumer's operand layout.
+// A thread owns 8 channels of FOUR horizontally adjacent output pixels (tile rows 4q .. 4q+3; the
+// tile's row pitch is a multiple of 4, so they share an image row).  It walks the 3 x (3S+3) input
+// window once: every input pixel is loaded and widened to fp32 once and feeds up to three outputs.
+struct DwUnit { int quad, j, base, live; };     // base: byte offset of the window origin in the halo tile
+
+template <int S>
+__device__ __forceinline__ void produce_dw(const GemmSeg &sg, const GemmParams &g, int kb_local, uint32_t halo, uint32_t dww,
+                                           const DwUnit &u, uint32_t a_base) {
+    if (u.quad >= 32) return;
+    const int c0 = kb_local * kTileK + u.j * 8;
+    const int r0 = u.quad * 4;
+    if (!u.live || c0 >= sg.C) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) st_shared16(a_chunk_addr(a_base, rg + 32 * i, j), make_uint4(0u, 0u, 0u, 0u));
+        for (int o = 0; o < 4; ++o) st_shared16(a_chunk_addr(a_base, r0 + o, u.j), make_uint4(0u, 0u, 0u, 0u));
         return;
     }
+    const int cbytes = g.halo_cb * 2;
     float acc[4][8];
     {
-        const float4 b0 = __ldg(reinterpret_cast<const float4 *>(sg.dw_b + c0)), b1 = __ldg(reinterpret_cast<const float4 *>(sg.dw_b + c0 + 4));
+        // tap weights [9][C] and the bias [C] were staged in shared memory when the CTA started
+        const float4 b0 = ld_shared_f4(dww + (uint32_t)(9 * sg.C + c0) * 4u), b1 = ld_shared_f4(dww + (uint32_t)(9 * sg.C + c0 + 4) * 4u);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            acc[i][0] = b0.x; acc[i][1] = b0.y; acc[i][2] = b0.z; acc[i][3] = b0.w;
-            acc[i][4] = b1.x; acc[i][5] = b1.y; acc[i][6] = b1.z; acc[i][7] = b1.w;
+        for (int o = 0; o < 4; ++o) {
+            acc[o][0] = b0.x; acc[o][1] = b0.y; acc[o][2] = b0.z; acc[o][3] = b0.w;
+            acc[o][4] = b1.x; acc[o][5] = b1.y; acc[o][6] = b1.z; acc[o][7] = b1.w;
         }
     }
-    const uint32_t hb = halo + j * 16;
+    const uint32_t hb = halo + u.base;
 #pragma unroll
-    for (int t = 0; t < 9; ++t) {
-        const float *wt = sg.dw_w + (size_t)t * sg.C + c0;
-        const float4 w0 = __ldg(reinterpret_cast<const float4 *>(wt)), w1 = __ldg(reinterpret_cast<const float4 *>(wt + 4));
-        const int toff = ((t / 3) * g.halo_w + (t % 3)) * cbytes;
+    for (int ry = 0; ry < 3; ++ry) {
+        float w[3][8];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            if (hoff[i] < 0) continue;
-            const f8 x = unpack8(ld_shared16(hb + hoff[i] + toff));
-            acc[i][0] = fmaf(x.v[0], w0.x, acc[i][0]); acc[i][1] = fmaf(x.v[1], w0.y, acc[i][1]);
-            acc[i][2] = fmaf(x.v[2], w0.z, acc[i][2]); acc[i][3] = fmaf(x.v[3], w0.w, acc[i][3]);
-            acc[i][4] = fmaf(x.v[4], w1.x, acc[i][4]); acc[i][5] = fmaf(x.v[5], w1.y, acc[i][5]);
-            acc[i][6] = fmaf(x.v[6], w1.z, acc[i][6]); acc[i][7] = fmaf(x.v[7], w1.w, acc[i][7]);
+        for (int sx = 0; sx < 3; ++sx) {
+            const uint32_t wa = dww + (uint32_t)((ry * 3 + sx) * sg.C + c0) * 4u;
+            const float4 w0 = ld_shared_f4(wa), w1 = ld_shared_f4(wa + 16);
+            w[sx][0] = w0.x; w[sx][1] = w0.y; w[sx][2] = w0.z; w[sx][3] = w0.w;
+            w[sx][4] = w1.x; w[sx][5] = w1.y; w[sx][6] = w1.z; w[sx][7] = w1.w;
+        }
+#pragma unroll
+        for (int ci = 0; ci < 3 * S + 3; ++ci) {
+            const f8 x = unpack8(ld_shared16(hb + (uint32_t)((ry * g.halo_w + ci) * cbytes)));
+#pragma unroll
+            for (int sx = 0; sx < 3; ++sx) {
+                if ((ci - sx) % S != 0 || ci - sx < 0 || (ci - sx) / S >= 4) continue;     // resolved at compile time
+                const int o = (ci - sx) / S;
+#pragma unroll
+                for (int c = 0; c < 8; ++c) acc[o][c] = fmaf(x.v[c], w[sx][c], acc[o][c]);
+            }
         }
     }
+    const float lo = act_lo(sg.dw_act), hi = act_hi(sg.dw_act);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int o = 0; o < 4; ++o) {
         f8 r;
 #pragma unroll
-        for (int c = 0; c < 8; ++c) r.v[c] = apply_act(acc[i][c], sg.dw_act);
-        st_shared16(a_chunk_addr(a_base, rg + 32 * i, j), hoff[i] < 0 ? make_uint4(0u, 0u, 0u, 0u) : pack8(r));
+        for (int c = 0; c < 8; ++c) r.v[c] = fminf(fmaxf(acc[o][c], lo), hi);
+        st_shared16(a_chunk_addr(a_base, r0 + o, u.j), pack8(r));
     }
 }
 
@@ -348,9 +399,13 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int total_tiles = g.m_tiles * g.n_tiles;
     const bool dw_mode = g.seg[0].mode == GA_DW;
+    // gather stages complete through cp.async arrivals (one per thread); the others through one
+    // arrival per producer warp
+    const bool async_gather = g.seg[0].mode == GA_GATHER;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < g.stages; ++s) { mbar_init(full_bar(s), kProducerThreads / 32 + 1); mbar_init(empty_bar(s), 1); }
+        const uint32_t full_count = (async_gather ? kProducerThreads : kProducerThreads / 32) + 1;
+        for (int s = 0; s < g.stages; ++s) { mbar_init(full_bar(s), full_count); mbar_init(empty_bar(s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), kEpilogueThreads / 32); }
         for (int s = 0; s < g.hstages; ++s) { mbar_init(hfull_bar(s), 1); mbar_init(hempty_bar(s), kProducerThreads / 32); }
         *fail_flag = 0;
@@ -361,6 +416,14 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)g.tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (dw_mode && threadIdx.x >= 64 && threadIdx.x < 64 + kProducerThreads) {
+        // depthwise tap weights [9][C] followed by the bias [C], fp32, once per CTA
+        const int C = g.seg[0].C;
+        float4 *dst = reinterpret_cast<float4 *>(sm + g.off_dww);
+        const float4 *w4 = reinterpret_cast<const float4 *>(g.seg[0].dw_w), *b4 = reinterpret_cast<const float4 *>(g.seg[0].dw_b);
+        for (int i = threadIdx.x - 64; i < 9 * C / 4; i += kProducerThreads) dst[i] = __ldg(w4 + i);
+        for (int i = threadIdx.x - 64; i < C / 4; i += kProducerThreads) dst[9 * C / 4 + i] = __ldg(b4 + i);
     }
     tc_fence_before();
     __syncthreads();
@@ -413,6 +476,9 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                     const int s = it % g.stages;
                     ok = mbar_wait(full_bar(s), (it / g.stages) & 1);
                     if (!ok) break;
+                    // the activation tile was written through the generic proxy (cp.async / st.shared)
+                    // and is read by the tensor core through the async proxy
+                    fence_proxy_async();
                     tc_fence_after();
                     const uint32_t a = sbase + s * stage_bytes, bb = a + kABytes;
 #pragma unroll
@@ -429,25 +495,22 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
         // ---- activation operand ----
         const int pt = threadIdx.x - 64;                 // 0..255
         const int grow = pt & 127, ghalf = pt >> 7;      // gather / stem mapping
-        const int dj = pt & 7, drg = pt >> 3;            // depthwise mapping
-        int hoff[4] = {-1, -1, -1, -1};                  // byte offset of each owned row's window origin in the halo tile
+        DwUnit du;
+        du.quad = 32; du.j = 0; du.base = 0; du.live = 0;
+        int zero_from = 8;                               // chunks >= zero_from of every row are K padding
         if (dw_mode) {
-            const int area = g.rh * g.rw, cbytes = g.halo_cb * 2;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int r = drg + 32 * i;
-                const int img = r / area, rem = r - img * area;
+            const int nj = g.halo_cb >> 3;               // 8-channel chunks per pixel in one K block
+            zero_from = nj;
+            du.quad = pt / nj; du.j = pt - du.quad * nj;
+            if (du.quad < 32) {
+                const int area = g.rh * g.rw, r0 = du.quad * 4;
+                const int img = r0 / area, rem = r0 - img * area;
                 const int dy = rem / g.rw, dx = rem - dy * g.rw;
-                if (img < g.ni) hoff[i] = ((img * g.halo_h + dy * g.seg[0].stride) * g.halo_w + dx * g.seg[0].stride) * cbytes;
+                du.live = img < g.ni;
+                du.base = ((img * g.halo_h + dy * g.seg[0].stride) * g.halo_w + dx * g.seg[0].stride) * g.halo_cb * 2 + du.j * 16;
             }
         }
-        const int lag = g.stages >= 3 ? 2 : (g.stages == 2 ? 1 : 0);
-        int pend = 0, pend_first = 0, it = 0;
-        auto retire_oldest = [&]() {
-            fence_proxy_async();
-            warp_arrive(full_bar(pend_first % g.stages), lane);
-            ++pend_first; --pend;
-        };
+        int it = 0;
         for (int ti = blockIdx.x; ti < total_tiles && ok; ti += gridDim.x) {
             const int mt = ti / g.n_tiles;
             RowPos rp;
@@ -467,34 +530,33 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                 if (sg.mode == GA_GATHER) {
                     if (first) { produce_gather(sg, gs0, rp, a_base, grow, ghalf); gather_advance(gs0, 8, sg.C >> 3, sg.k); }
                     else { produce_gather(sg, gs1, rp, a_base, grow, ghalf); gather_advance(gs1, 8, sg.C >> 3, sg.k); }
-                    cp_async_commit();
-                    ++pend;
-                    if (pend > lag) {
-                        if (lag == 2) cp_async_wait<2>(); else if (lag == 1) cp_async_wait<1>(); else cp_async_wait<0>();
-                        retire_oldest();
+                    // the stage's barrier is signalled when this thread's copies have landed; the
+                    // thread itself moves on to the next stage at once
+                    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(full_bar(s)) : "memory");
+                } else if (sg.mode == GA_DW) {
+                    const int hs = it % g.hstages;
+                    ok = mbar_wait_warp(hfull_bar(hs), (it / g.hstages) & 1, lane);
+                    if (!ok) break;
+                    const uint32_t halo = sbase + g.off_halo + hs * g.halo_stride, dww = sbase + g.off_dww;
+                    if (sg.stride == 1) produce_dw<1>(sg, g, kbl, halo, dww, du, a_base);
+                    else produce_dw<2>(sg, g, kbl, halo, dww, du, a_base);
+                    // K padding: chunks the block's channels do not reach must be zero, not stale
+                    for (int idx = pt; idx < kTileM * (8 - zero_from); idx += kProducerThreads) {
+                        const int row = idx / (8 - zero_from), jj = zero_from + idx - row * (8 - zero_from);
+                        st_shared16(a_chunk_addr(a_base, row, jj), make_uint4(0u, 0u, 0u, 0u));
                     }
+                    fence_proxy_async();
+                    warp_arrive(full_bar(s), lane);
+                    warp_arrive(hempty_bar(hs), lane);     // the halo tile has been read
                 } else {
-                    if (pend) { cp_async_wait<0>(); while (pend) retire_oldest(); }
-                    pend_first = it + 1;
-                    if (sg.mode == GA_DW) {
-                        const int hs = it % g.hstages;
-                        ok = mbar_wait_warp(hfull_bar(hs), (it / g.hstages) & 1, lane);
-                        if (!ok) break;
-                        produce_dw(sg, g, kbl, sbase + g.off_halo + hs * g.halo_stride, hoff, a_base, dj, drg);
-                        fence_proxy_async();
-                        warp_arrive(full_bar(s), lane);
-                        warp_arrive(hempty_bar(hs), lane);     // the halo tile has been read
-                    } else {
-                        produce_stem(sg, kbl, rp, a_base, grow, ghalf);
-                        fence_proxy_async();
-                        warp_arrive(full_bar(s), lane);
-                    }
+                    produce_stem(sg, kbl, rp, a_base, grow, ghalf);
+                    fence_proxy_async();
+                    warp_arrive(full_bar(s), lane);
                 }
             }
         }
-        cp_async_wait<0>();
-        if (ok) { while (pend) retire_oldest(); }
-        else if (lane == 0) atomicCAS(g.status, 0u, kStatusTimeout);
+        if (!ok && lane == 0) atomicCAS(g.status, 0u, kStatusTimeout);
+        cp_async_wait<0>();      // nothing of this thread is in flight when the CTA retires
     } else {
         // ---- epilogue: warp w reads tensor-memory lanes 32*(w%4).. ----
         const int quarter = warp & 3;
@@ -504,88 +566,101 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
         float *stgf = reinterpret_cast<float *>(sm + g.off_stg);
         const int pool_pitch = g.tile_n * 2 + 16;
         const int nchunks = g.tile_n / 16;
+        const float lo1 = act_lo(g.act), hi1 = act_hi(g.act), lo2 = act_lo(g.act2), hi2 = act_hi(g.act2);
         int i = 0;
         for (int ti = blockIdx.x; ti < total_tiles; ti += gridDim.x, ++i) {
             const int mt = ti / g.n_tiles, nt = ti - mt * g.n_tiles;
             const int b = i & 1;
+            // this tile's bias slice goes to shared memory (double-buffered: a warp is at most one tile ahead)
+            const uint32_t sbias = sbase + g.off_bias + b * 1024;
+            if (et * 4 < g.tile_n)
+                *reinterpret_cast<float4 *>(sm + g.off_bias + b * 1024 + et * 16) = __ldg(reinterpret_cast<const float4 *>(g.bias + nt * g.tile_n) + et);
+            const RowPos rq = map_row(g, mt, row);
+            const int n0 = nt * g.tile_n;
+            const size_t pix = ((size_t)rq.n * g.P + rq.p) * g.Q + rq.q;
             // the four epilogue warps share named barriers below, so they must agree on giving up
             if (!mbar_wait_warp(accf_bar(b), (i >> 1) & 1, lane) && lane == 0) *fail_flag = 1;
             epi_bar();
             if (*fail_flag) { ok = false; break; }
             tc_fence_after();
-            const RowPos rq = map_row(g, mt, row);
             const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * g.acc_stride;
-            const int n0 = nt * g.tile_n;
-            const size_t pix = ((size_t)rq.n * g.P + rq.p) * g.Q + rq.q;
-            for (int ch = 0; ch < nchunks; ++ch) {
-                float v[16];
-                tmem_ld16(t_lane + ch * 16, v);
-                if (ch == nchunks - 1) {
+            for (int cbase = 0; cbase < nchunks; cbase += 2) {
+                // two 16-column chunks per tensor-memory load where the tile has them
+                float vv[32];
+                const int nsub = (cbase + 1 < nchunks) ? 2 : 1;
+                if (nsub == 2) tmem_ld32(t_lane + cbase * 16, vv); else tmem_ld16(t_lane + cbase * 16, vv);
+                if (cbase + nsub >= nchunks) {
                     // every column of this accumulator is in registers: hand it back to the MMA warp
                     tc_fence_before();
                     warp_arrive(acce_bar(b), lane);
                 }
-                const int nc = n0 + ch * 16;
 #pragma unroll
-                for (int q4 = 0; q4 < 16; q4 += 4) {
-                    const float4 bz = __ldg(reinterpret_cast<const float4 *>(g.bias + nc + q4));   // bias is padded to npad
-                    v[q4] = apply_act(v[q4] + bz.x, g.act); v[q4 + 1] = apply_act(v[q4 + 1] + bz.y, g.act);
-                    v[q4 + 2] = apply_act(v[q4 + 2] + bz.z, g.act); v[q4 + 3] = apply_act(v[q4 + 3] + bz.w, g.act);
-                }
-                // shortcut connection with an identity branch: the skip tile is read once, here
-                if (g.skip && rq.valid) {
+                for (int sub = 0; sub < 2; ++sub) {
+                    if (sub >= nsub) break;
+                    float *v = vv + 16 * sub;
+                    const int ch = cbase + sub;
+                    const int nc = n0 + ch * 16;
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        if (nc + h * 8 + 8 > g.N) break;
-                        const f8 sv = unpack8(__ldg(reinterpret_cast<const uint4 *>(g.skip + pix * g.skip_ctot + nc + h * 8)));
-#pragma unroll
-                        for (int c = 0; c < 8; ++c) v[h * 8 + c] += sv.v[c];
+                    for (int q4 = 0; q4 < 16; q4 += 4) {
+                        const float4 bz = ld_shared_f4(sbias + (uint32_t)(ch * 16 + q4) * 4u);
+                        v[q4] = fminf(fmaxf(v[q4] + bz.x, lo1), hi1); v[q4 + 1] = fminf(fmaxf(v[q4 + 1] + bz.y, lo1), hi1);
+                        v[q4 + 2] = fminf(fmaxf(v[q4 + 2] + bz.z, lo1), hi1); v[q4 + 3] = fminf(fmaxf(v[q4 + 3] + bz.w, lo1), hi1);
                     }
-                }
-                if (g.act2) {
-#pragma unroll
-                    for (int c = 0; c < 16; ++c) v[c] = apply_act(v[c], g.act2);
-                }
-                if (g.epi == GE_STORE) {
-                    if (!rq.valid) continue;
-                    if (g.out_f32) {
-                        float *o = reinterpret_cast<float *>(g.out) + pix * g.out_ctot + g.out_coff + nc;
-#pragma unroll
-                        for (int c = 0; c < 16; ++c) if (nc + c < g.N) o[c] = v[c];
-                    } else {
-                        __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(g.out) + pix * g.out_ctot + g.out_coff + nc;
+                    // shortcut connection with an identity branch: the skip tile is read once, here
+                    if (g.skip && rq.valid) {
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
                             if (nc + h * 8 + 8 > g.N) break;
-                            f8 pv;
+                            const f8 sv = unpack8(__ldg(reinterpret_cast<const uint4 *>(g.skip + pix * g.skip_ctot + nc + h * 8)));
 #pragma unroll
-                            for (int c = 0; c < 8; ++c) pv.v[c] = v[h * 8 + c];
-                            *reinterpret_cast<uint4 *>(o + h * 8) = pack8(pv);
+                            for (int c = 0; c < 8; ++c) v[h * 8 + c] += sv.v[c];
                         }
                     }
-                } else if (g.epi == GE_POOL) {
-                    // rows outside the conv output never win a max
-                    f8 lo, hi;
+                    if (g.act2) {
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) { lo.v[c] = rq.valid ? v[c] : -INFINITY; hi.v[c] = rq.valid ? v[8 + c] : -INFINITY; }
-                    st_shared16(stg + row * pool_pitch + ch * 32, pack8(lo));
-                    st_shared16(stg + row * pool_pitch + ch * 32 + 16, pack8(hi));
-                } else {
-                    // global average: 16 columns at a time through shared memory, rows summed in ascending order
-                    epi_bar();
+                        for (int c = 0; c < 16; ++c) v[c] = fminf(fmaxf(v[c], lo2), hi2);
+                    }
+                    if (g.epi == GE_STORE) {
+                        if (!rq.valid) continue;
+                        if (g.out_f32) {
+                            float *o = reinterpret_cast<float *>(g.out) + pix * g.out_ctot + g.out_coff + nc;
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) stgf[row * 17 + c] = rq.valid ? v[c] : 0.0f;
-                    epi_bar();
-                    for (int item = et; item < g.gap_imgs * 16; item += kEpilogueThreads) {
-                        const int img = item >> 4, c = item & 15;
-                        const int n = mt * g.gap_imgs + img;
-                        if (n >= g.batch || nc + c >= g.N) continue;
-                        float acc = 0.0f;
-                        for (int r = 0; r < g.gap_rpi; ++r) acc += stgf[(img * g.gap_rpi + r) * 17 + c];
-                        acc /= (float)g.gap_rpi;
-                        const size_t oi = (size_t)n * g.out_ctot + g.out_coff + nc + c;
-                        if (g.out_f32) reinterpret_cast<float *>(g.out)[oi] = acc;
-                        else reinterpret_cast<__nv_bfloat16 *>(g.out)[oi] = __float2bfloat16_rn(acc);
+                            for (int c = 0; c < 16; ++c) if (nc + c < g.N) o[c] = v[c];
+                        } else {
+                            __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(g.out) + pix * g.out_ctot + g.out_coff + nc;
+#pragma unroll
+                            for (int h = 0; h < 2; ++h) {
+                                if (nc + h * 8 + 8 > g.N) break;
+                                f8 pv;
+#pragma unroll
+                                for (int c = 0; c < 8; ++c) pv.v[c] = v[h * 8 + c];
+                                *reinterpret_cast<uint4 *>(o + h * 8) = pack8(pv);
+                            }
+                        }
+                    } else if (g.epi == GE_POOL) {
+                        // rows outside the conv output never win a max
+                        f8 lo, hi;
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) { lo.v[c] = rq.valid ? v[c] : -INFINITY; hi.v[c] = rq.valid ? v[8 + c] : -INFINITY; }
+                        st_shared16(stg + row * pool_pitch + ch * 32, pack8(lo));
+                        st_shared16(stg + row * pool_pitch + ch * 32 + 16, pack8(hi));
+                    } else {
+                        // global average: 16 columns at a time through shared memory, rows summed in ascending order
+                        epi_bar();
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) stgf[row * 17 + c] = rq.valid ? v[c] : 0.0f;
+                        epi_bar();
+                        for (int item = et; item < g.gap_imgs * 16; item += kEpilogueThreads) {
+                            const int img = item >> 4, c = item & 15;
+                            const int n = mt * g.gap_imgs + img;
+                            if (n >= g.batch || nc + c >= g.N) continue;
+                            float acc = 0.0f;
+                            for (int r = 0; r < g.gap_area; ++r) acc += stgf[(img * g.gap_area + r) * 17 + c];
+                            acc /= (float)g.gap_rpi;
+                            const size_t oi = (size_t)n * g.out_ctot + g.out_coff + nc + c;
+                            if (g.out_f32) reinterpret_cast<float *>(g.out)[oi] = acc;
+                            else reinterpret_cast<__nv_bfloat16 *>(g.out)[oi] = __float2bfloat16_rn(acc);
+                        }
                     }
                 }
             }

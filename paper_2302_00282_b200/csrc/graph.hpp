@@ -123,10 +123,10 @@ struct Launch {
     int out_dtype = XENOS_DTYPE_BF16;
     int stages = 0, smem_bytes = 0, tmem_cols = 0, pipe_bytes = 0;
     int ni = 1, step_y = 0, step_x = 0, off_y = 0, off_x = 0;      // PATCH tiles: images, tile pitch, origin offset
-    int gap_imgs = 0, gap_rpi = 0;                                 // global-average epilogue
+    int gap_imgs = 0, gap_area = 0, gap_rpi = 0;                                 // global-average epilogue
     int acc_stride = 0;                                            // columns between the two accumulators
     int hstages = 0, halo_bytes = 0, halo_stride = 0, halo_cb = 0;   // depthwise halo ring (halo_h x halo_w input pixels per image)
-    int off_halo = 0, off_stg = 0, off_bar = 0;                    // shared-memory layout
+    int off_halo = 0, off_stg = 0, off_dww = 0, off_bias = 0, off_bar = 0;                    // shared-memory layout
     // ---- fp32 linked chain (conv kxk -> conv1x1 -> pool)
     int Cmid = 0, K2 = 0, act2 = 0;
     int parts_outc = 1, tile_h = 0, tile_w = 0, tiles_h = 0, tiles_w = 0;   // tile of POOL outputs

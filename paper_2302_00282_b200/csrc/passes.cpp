@@ -172,7 +172,7 @@ static bool try_match(const LinkCtx &cx, int a, Allowed allowed, Chain &out) {
     // ---- bf16 tensor-core chains -----------------------------------------------------------
     if (A.kind == NK_DW) {
         // depthwise -> pointwise: the motivating mismatch of Section 2.2 (ConvX -> ConvY row)
-        if (A.k != 3 || A.cin % 8) return false;
+        if (A.k != 3 || A.cin % 8 || A.stride > 2) return false;
         int b = cx.sole(a);
         if (b < 0 || !allowed(b)) return false;
         const Node &B = g.nodes[b];
@@ -181,7 +181,8 @@ static bool try_match(const LinkCtx &cx, int a, Allowed allowed, Chain &out) {
         out.nodes = {a, b};
         out.pattern = "ConvX -> ConvY (depthwise 3x3 -> pointwise 1x1)";
         int c = cx.sole(b);
-        if (c >= 0 && allowed(c) && g.nodes[c].kind == NK_GAP && cx.rows(b) <= 128) {
+        const Tensor &bo = g.tensors[B.out];
+        if (c >= 0 && allowed(c) && g.nodes[c].kind == NK_GAP && bo.h * ((bo.w + 3) / 4 * 4) <= 128) {
             out.nodes.push_back(c);
             out.pattern = "ConvX -> ConvY -> ZPooling (depthwise -> pointwise -> global average)";
         }
@@ -615,19 +616,21 @@ struct Lower {
             L.epi = EPI_GAP;
             L.imgs_per_tile = 128 / L.rows_per_image;
             L.tile_rows = L.imgs_per_tile * L.rows_per_image;
-            L.gap_imgs = L.imgs_per_tile; L.gap_rpi = L.rows_per_image;
+            L.gap_imgs = L.imgs_per_tile; L.gap_area = L.rows_per_image; L.gap_rpi = L.rows_per_image;
         }
         if (dw) {
             // The depthwise stage reads a halo tile that TMA fetches as one 4-D box, so the tile is a
             // patch: ni whole images when an image fits 128 rows, else th x tw output pixels of one image.
             L.map_mode = MAP_PATCH;
-            if (L.rows_per_image <= 128) {
-                L.ni = 128 / L.rows_per_image; L.patch_rh = L.P; L.patch_rw = L.Q;
+            // the tile's row pitch is a multiple of 4: a producer thread owns 4 adjacent pixels of a row
+            const int Qp = round_up(L.Q, 4);
+            if (L.P * Qp <= 128) {
+                L.ni = 128 / (L.P * Qp); L.patch_rh = L.P; L.patch_rw = Qp;
             } else {
                 if (gapn) return fail(g, XENOS_E_UNSUPPORTED, "internal: global average needs whole images per tile");
                 L.ni = 1;
                 long best = -1;
-                for (int tw = 1; tw <= std::min(L.Q, 128); ++tw) {
+                for (int tw = 4; tw <= std::min(Qp, 128); tw += 4) {
                     int th = std::min(L.P, 128 / tw);
                     long tiles = (long)ceil_div(L.P, th) * ceil_div(L.Q, tw);
                     // fewest tiles first; then the widest tile (longest contiguous rows in memory)
@@ -648,7 +651,7 @@ struct Lower {
             L.halo_bytes = L.ni * L.halo_h * L.halo_w * L.halo_cb * 2;
             L.halo_stride = (int)align_up((size_t)L.halo_bytes, 128);
             if (L.halo_h > 256 || L.halo_w > 256) return fail(g, XENOS_E_UNSUPPORTED, "internal: halo tile exceeds the TMA box limit");
-            if (gapn) { L.gap_imgs = L.ni; L.gap_rpi = L.rows_per_image; }
+            if (gapn) { L.gap_imgs = L.ni; L.gap_area = L.patch_rh * L.patch_rw; L.gap_rpi = L.rows_per_image; }
         }
         L.out = last->out;
         const Tensor &ot = g.tensors[L.out];
@@ -673,7 +676,7 @@ struct Lower {
             L.tile_n = round_up(ceil_div(N16, L.n_tiles), 16);
             // kernels are dealt to idle units first: halve the channel tile while units stay idle
             // (a linked depthwise stage is recomputed per channel tile, so it stops halving earlier)
-            const int min_tile_n = dw ? 128 : 32;
+            const int min_tile_n = dw ? 256 : 32;
             while (L.m_tiles * L.n_tiles < g.hw.sm_count && L.tile_n >= 2 * min_tile_n) {
                 int nt = L.n_tiles * 2, tn = round_up(ceil_div(N16, nt), 16);
                 if ((nt - 1) * tn >= N) break;
@@ -690,7 +693,9 @@ struct Lower {
         int stage_bytes = 16384 + L.tile_n * 128;
         int stg_bytes = L.epi == EPI_POOL ? 128 * (L.tile_n * 2 + 16) : (L.epi == EPI_GAP ? 128 * 17 * 4 : 0);
         stg_bytes = (int)align_up((size_t)stg_bytes, 128);
-        int cap = std::min(g.hw.smem_bytes_per_cta, 227 * 1024) - 1024 - 256;
+        // depthwise tap weights + bias of the linked stage (fp32 [10][C]) and two bias slices of the GEMM
+        int dww_bytes = dw ? (int)align_up((size_t)40 * src.c, 128) : 0;
+        int cap = std::min(g.hw.smem_bytes_per_cta, 227 * 1024) - 1024 - 256 - 2048 - dww_bytes;
         L.hstages = dw ? 2 : 0;
         if (dw && cap - stg_bytes - 3 * L.halo_stride >= 3 * stage_bytes) L.hstages = 3;
         int room = cap - stg_bytes - L.hstages * L.halo_stride;
@@ -698,7 +703,9 @@ struct Lower {
         if (L.stages < 1) return fail(g, XENOS_E_BAD_SPLIT, "split: pipeline does not fit shared memory");
         L.off_halo = L.stages * stage_bytes;
         L.off_stg = L.off_halo + L.hstages * L.halo_stride;
-        L.off_bar = (int)align_up((size_t)(L.off_stg + stg_bytes), 128);
+        L.off_dww = (int)align_up((size_t)(L.off_stg + stg_bytes), 128);
+        L.off_bias = L.off_dww + dww_bytes;
+        L.off_bar = L.off_bias + 2048;
         L.pipe_bytes = L.off_bar;
         L.smem_bytes = L.off_bar + 256 + 1024;     // + barriers, alignment slack
         L.grid = std::min(L.m_tiles * L.n_tiles, g.hw.sm_count);

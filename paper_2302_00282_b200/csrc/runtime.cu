@@ -262,12 +262,12 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
             p.ni = L.ni; p.rh = L.patch_rh; p.rw = L.patch_rw; p.tiles_y = L.tiles_y; p.tiles_x = L.tiles_x;
             p.step_y = L.step_y; p.step_x = L.step_x; p.off_y = L.off_y; p.off_x = L.off_x;
             p.pool_k = L.pool_k; p.pool_stride = L.pool_stride; p.PP = L.PP; p.PQ = L.PQ; p.pth = L.patch_th; p.ptw = L.patch_tw;
-            p.gap_imgs = L.gap_imgs; p.gap_rpi = L.gap_rpi;
+            p.gap_imgs = L.gap_imgs; p.gap_area = L.gap_area; p.gap_rpi = L.gap_rpi;
             p.kblocks = L.kblocks; p.stages = L.stages; p.tile_n = L.tile_n; p.n_tiles = L.n_tiles; p.N = L.K;
             p.acc_stride = L.acc_stride; p.tmem_cols = L.tmem_cols;
             p.hstages = L.hstages; p.halo_bytes = L.halo_bytes; p.halo_stride = L.halo_stride;
             p.halo_h = L.halo_h; p.halo_w = L.halo_w; p.halo_cb = L.halo_cb;
-            p.off_halo = L.off_halo; p.off_stg = L.off_stg; p.off_bar = L.off_bar;
+            p.off_halo = L.off_halo; p.off_stg = L.off_stg; p.off_dww = L.off_dww; p.off_bias = L.off_bias; p.off_bar = L.off_bar;
             p.act = L.act; p.act2 = L.act2; p.epi = L.epi; p.out_ctot = L.out_ctot; p.out_coff = L.out_coff;
             p.out_f32 = L.out_dtype == XENOS_DTYPE_F32;
             p.idesc = make_idesc(L.tile_n);
