@@ -698,6 +698,7 @@ struct Lower {
         int cap = std::min(g.hw.smem_bytes_per_cta, 227 * 1024) - 1024 - 256 - 2048 - dww_bytes;
         L.hstages = dw ? 2 : 0;
         if (dw && cap - stg_bytes - 3 * L.halo_stride >= 3 * stage_bytes) L.hstages = 3;
+        if (dw && cap - stg_bytes - 4 * L.halo_stride >= 4 * stage_bytes) L.hstages = 4;
         int room = cap - stg_bytes - L.hstages * L.halo_stride;
         L.stages = std::min(6, room / stage_bytes);
         if (L.stages < 1) return fail(g, XENOS_E_BAD_SPLIT, "split: pipeline does not fit shared memory");
