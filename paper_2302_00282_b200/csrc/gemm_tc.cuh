@@ -348,8 +348,7 @@ __device__ __forceinline__ void produce_dw(const GemmSeg &sg, const GemmParams &
         }
     }
     const uint32_t hb = halo + u.base;
-    // the row loop stays rolled: its body is the hot code of eight warps and should stay cache-resident
-#pragma unroll 1
+#pragma unroll
     for (int ry = 0; ry < 3; ++ry) {
         float w[3][8];
 #pragma unroll
@@ -382,9 +381,6 @@ __device__ __forceinline__ void produce_dw(const GemmSeg &sg, const GemmParams &
 }
 
 // ---- the kernel --------------------------------------------------------------------------------
-// One instantiation per (activation source, epilogue): a role only ever runs the code of its own
-// mode, and a smaller kernel keeps the instruction caches of the 14 differently-occupied warps warm.
-template <int AMODE, int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmH, const GemmParams g) {
     extern __shared__ uint8_t smem_raw[];
@@ -404,10 +400,10 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int total_tiles = g.m_tiles * g.n_tiles;
-    constexpr bool dw_mode = AMODE == GA_DW;
+    const bool dw_mode = g.seg[0].mode == GA_DW;
     // gather stages complete through cp.async arrivals (one per thread); the others through one
     // arrival per producer warp
-    constexpr bool async_gather = AMODE == GA_GATHER;
+    const bool async_gather = g.seg[0].mode == GA_GATHER;
 
     if (threadIdx.x == 0) {
         const uint32_t full_count = (async_gather ? kProducerThreads : kProducerThreads / 32) + 1;
@@ -523,10 +519,8 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
             rp.valid = 0; rp.n = 0; rp.p = 0; rp.q = 0;
             if (!dw_mode) rp = map_row(g, mt, grow);
             GatherState gs0 = {0, 0, 0}, gs1 = {0, 0, 0};
-            if (AMODE == GA_GATHER && ghalf) {
-                gather_advance(gs0, 4, g.seg[0].C >> 3, g.seg[0].k);
-                if (g.seg[1].mode == GA_GATHER) gather_advance(gs1, 4, g.seg[1].C >> 3, g.seg[1].k);
-            }
+            if (g.seg[0].mode == GA_GATHER && ghalf) gather_advance(gs0, 4, g.seg[0].C >> 3, g.seg[0].k);
+            if (g.seg[1].mode == GA_GATHER && ghalf) gather_advance(gs1, 4, g.seg[1].C >> 3, g.seg[1].k);
             for (int kb = 0; kb < g.kblocks && ok; ++kb, ++it) {
                 const int s = it % g.stages;
                 ok = mbar_wait_warp(empty_bar(s), ((it / g.stages) & 1) ^ 1u, lane);
@@ -535,13 +529,13 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                 const GemmSeg &sg = first ? g.seg[0] : g.seg[1];
                 const int kbl = first ? kb : kb - g.seg[0].kblocks;
                 const uint32_t a_base = sbase + s * stage_bytes;
-                if constexpr (AMODE == GA_GATHER) {
+                if (sg.mode == GA_GATHER) {
                     if (first) { produce_gather(sg, gs0, rp, a_base, grow, ghalf); gather_advance(gs0, 8, sg.C >> 3, sg.k); }
                     else { produce_gather(sg, gs1, rp, a_base, grow, ghalf); gather_advance(gs1, 8, sg.C >> 3, sg.k); }
                     // the stage's barrier is signalled when this thread's copies have landed; the
                     // thread itself moves on to the next stage at once
                     asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(full_bar(s)) : "memory");
-                } else if constexpr (AMODE == GA_DW) {
+                } else if (sg.mode == GA_DW) {
                     const int hs = it % g.hstages;
                     ok = mbar_wait_warp(hfull_bar(hs), (it / g.hstages) & 1, lane);
                     if (!ok) break;
@@ -628,7 +622,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
 #pragma unroll
                         for (int c = 0; c < 16; ++c) v[c] = fminf(fmaxf(v[c], lo2), hi2);
                     }
-                    if constexpr (EPI == GE_STORE) {
+                    if (g.epi == GE_STORE) {
                         if (!rq.valid) continue;
                         if (g.out_f32) {
                             float *o = reinterpret_cast<float *>(g.out) + pix * g.out_ctot + g.out_coff + nc;
@@ -645,7 +639,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                                 *reinterpret_cast<uint4 *>(o + h * 8) = pack8(pv);
                             }
                         }
-                    } else if constexpr (EPI == GE_POOL) {
+                    } else if (g.epi == GE_POOL) {
                         // rows outside the conv output never win a max
                         f8 lo, hi;
 #pragma unroll
@@ -672,7 +666,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                     }
                 }
             }
-            if constexpr (EPI == GE_POOL) {
+            if (g.epi == GE_POOL) {
                 epi_bar();
                 const int per = g.tiles_y * g.tiles_x;
                 const int n = mt / per, tt = mt - n * per;

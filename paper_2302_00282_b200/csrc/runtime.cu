@@ -30,25 +30,6 @@ static xenos_status_t cuda_fail(const Graph &g, const char *what, cudaError_t e)
     return fail(g, XENOS_E_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
 }
 
-typedef void (*gemm_kernel_fn)(const CUtensorMap, const CUtensorMap, const xk::GemmParams);
-
-// the kernel instance for an activation source (gather / stem / depthwise) and an epilogue
-static gemm_kernel_fn gemm_kernel_for(int amode, int epi) {
-    using namespace xk;
-    switch (amode * 3 + epi) {
-    case GA_GATHER * 3 + GE_STORE: return gemm_chain_kernel<GA_GATHER, GE_STORE>;
-    case GA_GATHER * 3 + GE_GAP: return gemm_chain_kernel<GA_GATHER, GE_GAP>;
-    case GA_GATHER * 3 + GE_POOL: return gemm_chain_kernel<GA_GATHER, GE_POOL>;
-    case GA_STEM * 3 + GE_STORE: return gemm_chain_kernel<GA_STEM, GE_STORE>;
-    case GA_STEM * 3 + GE_GAP: return gemm_chain_kernel<GA_STEM, GE_GAP>;
-    case GA_STEM * 3 + GE_POOL: return gemm_chain_kernel<GA_STEM, GE_POOL>;
-    case GA_DW * 3 + GE_STORE: return gemm_chain_kernel<GA_DW, GE_STORE>;
-    case GA_DW * 3 + GE_GAP: return gemm_chain_kernel<GA_DW, GE_GAP>;
-    case GA_DW * 3 + GE_POOL: return gemm_chain_kernel<GA_DW, GE_POOL>;
-    default: return nullptr;
-    }
-}
-
 static uint32_t make_idesc(int tile_n) {
     // kind::f16 instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, M = 128
     uint32_t d = 0;
@@ -147,10 +128,8 @@ xenos_status_t runtime_bind(Graph &g, void *ws, size_t bytes, void *stream_v) {
     if (max_gemm_smem > optin || max_chain_smem > optin)
         return fail(g, XENOS_E_CUDA, "a kernel of this plan needs more shared memory than the device offers");
     if (any_gemm)
-        for (int am = 1; am <= 3; ++am)
-            for (int ep = 0; ep <= 2; ++ep)
-                if ((e = cudaFuncSetAttribute(gemm_kernel_for(am, ep), cudaFuncAttributeMaxDynamicSharedMemorySize, optin)) != cudaSuccess)
-                    return cuda_fail(g, "cudaFuncSetAttribute(gemm)", e);
+        if ((e = cudaFuncSetAttribute(xk::gemm_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin)) != cudaSuccess)
+            return cuda_fail(g, "cudaFuncSetAttribute(gemm)", e);
     if (max_chain_smem > 0)
         if ((e = cudaFuncSetAttribute(xk::f32_conv_conv_pool_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin)) != cudaSuccess)
             return cuda_fail(g, "cudaFuncSetAttribute(f32 chain)", e);
@@ -310,9 +289,7 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
                 }
             }
             const int grid = std::min(p.m_tiles * L.n_tiles, sms);
-            gemm_kernel_fn fn = gemm_kernel_for(L.seg[0].mode, L.epi);
-            if (!fn) return fail(g, XENOS_E_UNSUPPORTED, "internal: no kernel instance for this launch");
-            fn<<<grid, xk::kThreads, L.smem_bytes, stream>>>(rt->tmaps[li], *tmh, p);
+            xk::gemm_chain_kernel<<<grid, xk::kThreads, L.smem_bytes, stream>>>(rt->tmaps[li], *tmh, p);
             break;
         }
         default:
