@@ -337,36 +337,41 @@ __device__ __forceinline__ void produce_dw(const GemmSeg &sg, const GemmParams &
         return;
     }
     const int cbytes = g.halo_cb * 2;
-    float acc[4][8];
+    // accumulators, weights and pixels are kept as fp32 pairs: one packed FMA does two channels
+    float2 acc[4][4];
     {
         // tap weights [9][C] and the bias [C] were staged in shared memory when the CTA started
         const float4 b0 = ld_shared_f4(dww + (uint32_t)(9 * sg.C + c0) * 4u), b1 = ld_shared_f4(dww + (uint32_t)(9 * sg.C + c0 + 4) * 4u);
 #pragma unroll
         for (int o = 0; o < 4; ++o) {
-            acc[o][0] = b0.x; acc[o][1] = b0.y; acc[o][2] = b0.z; acc[o][3] = b0.w;
-            acc[o][4] = b1.x; acc[o][5] = b1.y; acc[o][6] = b1.z; acc[o][7] = b1.w;
+            acc[o][0] = make_float2(b0.x, b0.y); acc[o][1] = make_float2(b0.z, b0.w);
+            acc[o][2] = make_float2(b1.x, b1.y); acc[o][3] = make_float2(b1.z, b1.w);
         }
     }
     const uint32_t hb = halo + u.base;
 #pragma unroll
     for (int ry = 0; ry < 3; ++ry) {
-        float w[3][8];
+        float2 w[3][4];
 #pragma unroll
         for (int sx = 0; sx < 3; ++sx) {
             const uint32_t wa = dww + (uint32_t)((ry * 3 + sx) * sg.C + c0) * 4u;
             const float4 w0 = ld_shared_f4(wa), w1 = ld_shared_f4(wa + 16);
-            w[sx][0] = w0.x; w[sx][1] = w0.y; w[sx][2] = w0.z; w[sx][3] = w0.w;
-            w[sx][4] = w1.x; w[sx][5] = w1.y; w[sx][6] = w1.z; w[sx][7] = w1.w;
+            w[sx][0] = make_float2(w0.x, w0.y); w[sx][1] = make_float2(w0.z, w0.w);
+            w[sx][2] = make_float2(w1.x, w1.y); w[sx][3] = make_float2(w1.z, w1.w);
         }
 #pragma unroll
         for (int ci = 0; ci < 3 * S + 3; ++ci) {
-            const f8 x = unpack8(ld_shared16(hb + (uint32_t)((ry * g.halo_w + ci) * cbytes)));
+            const uint4 raw = ld_shared16(hb + (uint32_t)((ry * g.halo_w + ci) * cbytes));
+            const uint32_t rw4[4] = {raw.x, raw.y, raw.z, raw.w};
+            float2 x[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) x[c] = make_float2(__uint_as_float(rw4[c] << 16), __uint_as_float(rw4[c] & 0xffff0000u));
 #pragma unroll
             for (int sx = 0; sx < 3; ++sx) {
                 if ((ci - sx) % S != 0 || ci - sx < 0 || (ci - sx) / S >= 4) continue;     // resolved at compile time
                 const int o = (ci - sx) / S;
 #pragma unroll
-                for (int c = 0; c < 8; ++c) acc[o][c] = fmaf(x.v[c], w[sx][c], acc[o][c]);
+                for (int c = 0; c < 4; ++c) acc[o][c] = __ffma2_rn(x[c], w[sx][c], acc[o][c]);
             }
         }
     }
@@ -375,7 +380,10 @@ __device__ __forceinline__ void produce_dw(const GemmSeg &sg, const GemmParams &
     for (int o = 0; o < 4; ++o) {
         f8 r;
 #pragma unroll
-        for (int c = 0; c < 8; ++c) r.v[c] = fminf(fmaxf(acc[o][c], lo), hi);
+        for (int c = 0; c < 4; ++c) {
+            r.v[2 * c] = fminf(fmaxf(acc[o][c].x, lo), hi);
+            r.v[2 * c + 1] = fminf(fmaxf(acc[o][c].y, lo), hi);
+        }
         st_shared16(a_chunk_addr(a_base, r0 + o, u.j), pack8(r));
     }
 }
