@@ -696,9 +696,13 @@ struct Lower {
         // depthwise tap weights + bias of the linked stage (fp32 [10][C]) and two bias slices of the GEMM
         int dww_bytes = dw ? (int)align_up((size_t)40 * src.c, 128) : 0;
         int cap = std::min(g.hw.smem_bytes_per_cta, 227 * 1024) - 1024 - 256 - 2048 - dww_bytes;
-        L.hstages = dw ? 2 : 0;
-        if (dw && cap - stg_bytes - 3 * L.halo_stride >= 3 * stage_bytes) L.hstages = 3;
-        if (dw && cap - stg_bytes - 4 * L.halo_stride >= 4 * stage_bytes) L.hstages = 4;
+        // a linked depthwise stage is bound by its own arithmetic, not by the MMA: give the halo ring
+        // (the TMA prefetch distance) up to four stages first, the A|B ring keeps at least two
+        L.hstages = 0;
+        if (dw) {
+            L.hstages = 2;
+            while (L.hstages < 4 && cap - stg_bytes - (L.hstages + 1) * L.halo_stride >= 2 * stage_bytes) ++L.hstages;
+        }
         int room = cap - stg_bytes - L.hstages * L.halo_stride;
         L.stages = std::min(6, room / stage_bytes);
         if (L.stages < 1) return fail(g, XENOS_E_BAD_SPLIT, "split: pipeline does not fit shared memory");
