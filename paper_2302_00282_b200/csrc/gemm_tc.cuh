@@ -72,7 +72,8 @@ struct GemmParams {
     int gap_imgs, gap_area, gap_rpi;               // global-average epilogue: whole images per tile (area rows each, rpi of them real)
     int kblocks, stages, tile_n, n_tiles, m_tiles, N;
     int acc_stride, tmem_cols;                     // two accumulators, acc_stride columns apart
-    int hstages, halo_bytes, halo_stride, halo_h, halo_w, halo_cb;   // depthwise halo ring
+    int hstages, halo_bytes, halo_stride, halo_h, halo_w, halo_cb;   // halo ring (depthwise input tile / stem image patch)
+    int stem_tma, stem_align;                       // stem: patch by TMA; x origin alignment in elements
     int off_halo, off_stg, off_dww, off_bias, off_bar;   // shared-memory offsets from the 1024-aligned base
     int act, act2, epi, out_ctot, out_coff, out_f32, skip_ctot;
     uint32_t idesc;
@@ -260,6 +261,18 @@ __device__ __forceinline__ void produce_gather(const GemmSeg &sg, GatherState st
     const int C8 = sg.C >> 3;
     const int ih0 = rp.p * sg.stride - sg.pad, iw0 = rp.q * sg.stride - sg.pad;
     const __nv_bfloat16 *img = src + (size_t)rp.n * sg.H * sg.W * sg.C;
+    if (sg.k == 1) {
+        // pointwise: the row's channel vector is contiguous, chunk c of the K block is 16 bytes at c*16
+        const bool in = rp.valid && st.tap_r == 0 && ih0 >= 0 && ih0 < sg.H && iw0 >= 0 && iw0 < sg.W;
+        const __nv_bfloat16 *px = img + ((size_t)ih0 * sg.W + iw0) * sg.C;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int c8 = st.cc + i;          // with k == 1 the state's chunk counter runs from the segment start
+            const bool live = in && c8 < C8;
+            cp_async16(a_chunk_addr(a_base, row, half * 4 + i), live ? (const void *)(px + c8 * 8) : (const void *)src, live ? 16u : 0u);
+        }
+        return;
+    }
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const void *ptr = src;
@@ -276,45 +289,70 @@ __device__ __forceinline__ void produce_gather(const GemmSeg &sg, GatherState st
     }
 }
 
-// stem: K element e = (r * k + s) * C + c of an NCHW image (fp32 or bf16); thread = (row, half) and
-// takes the chunks j = 2*i + half so that both halves share the real (non-padding) elements.  All
-// loads of a chunk pair are issued before any is used.
-__device__ __forceinline__ void produce_stem(const GemmSeg &sg, int kb_local, const RowPos &rp, uint32_t a_base,
-                                             int row, int half) {
+// stem (small-channel NCHW image, fp32 or bf16), K element e = (r * k + s) * C + c.
+// Preferred form: TMA brings the tile's input patch [C][ih][iwp] to shared memory (4-D box whose x
+// origin is rounded down to a 16-byte boundary; out-of-range reads are zero = padding), one patch
+// per tile, prefetched through the halo ring; a row's K elements are then shared-memory reads.
+// thread = (row, half); it builds the chunks j = 2*i + half so that both halves share the real elements.
+__device__ __forceinline__ void produce_stem_tile(const GemmSeg &sg, const GemmParams &g, int kb_local, const uint8_t *patch,
+                                                  int xrem, uint32_t a_base, int row, int half) {
+    const int area = g.rh * g.rw;
+    const bool live = row < area;
+    const int dy = row / g.rw, dx = row - dy * g.rw;
+    const int base = (dy * sg.stride) * g.halo_w + xrem + dx * sg.stride;
+    const int plane = g.halo_h * g.halo_w;
+    const float *pf = reinterpret_cast<const float *>(patch);
+    const unsigned short *ph = reinterpret_cast<const unsigned short *>(patch);
+#pragma unroll 1
+    for (int i = 0; i < 4; ++i) {
+        const int j = 2 * i + half;
+        int e = kb_local * kTileK + j * 8;
+        int tap = e / sg.C, c = e - tap * sg.C;
+        int r = tap / sg.k, s = tap - r * sg.k;
+        uint32_t w[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            unsigned v = 0;
+            if (live && r < sg.k) {
+                const int idx = base + c * plane + r * g.halo_w + s;
+                v = sg.src_f32 ? (unsigned)__bfloat16_as_ushort(__float2bfloat16_rn(pf[idx])) : (unsigned)ph[idx];
+            }
+            w[q >> 1] |= v << ((q & 1) * 16);
+            if (++c == sg.C) { c = 0; if (++s == sg.k) { s = 0; ++r; } }
+        }
+        st_shared16(a_chunk_addr(a_base, row, j), make_uint4(w[0], w[1], w[2], w[3]));
+    }
+}
+
+// Fallback when the image's row pitch is not a multiple of 16 bytes (TMA cannot address it): every
+// thread loads its row's elements straight from global memory.
+__device__ __forceinline__ void produce_stem_direct(const GemmSeg &sg, int kb_local, const RowPos &rp, uint32_t a_base,
+                                                    int row, int half) {
     const int ih0 = rp.p * sg.stride - sg.pad, iw0 = rp.q * sg.stride - sg.pad;
     const size_t img = (size_t)rp.n * sg.C * sg.H * sg.W;
     const float *sf = reinterpret_cast<const float *>(sg.src) + img;
     const unsigned short *sh = reinterpret_cast<const unsigned short *>(sg.src) + img;
+#pragma unroll 1
+    for (int i = 0; i < 4; ++i) {
+        const int j = 2 * i + half;
+        int e = kb_local * kTileK + j * 8;
+        int tap = e / sg.C, c = e - tap * sg.C;
+        int r = tap / sg.k, s = tap - r * sg.k;
+        f8 x;
 #pragma unroll
-    for (int pair = 0; pair < 2; ++pair) {
-        float x[16];
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const int j = 2 * (2 * pair + u) + half;
-            int e = kb_local * kTileK + j * 8;
-            int tap = e / sg.C, c = e - tap * sg.C;
-            int r = tap / sg.k, s = tap - r * sg.k;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                float v = 0.0f;
-                if (rp.valid && r < sg.k) {
-                    const int ih = ih0 + r, iw = iw0 + s;
-                    if (ih >= 0 && ih < sg.H && iw >= 0 && iw < sg.W) {
-                        const int off = (c * sg.H + ih) * sg.W + iw;
-                        v = sg.src_f32 ? __ldg(sf + off) : __uint_as_float((unsigned)__ldg(sh + off) << 16);
-                    }
+        for (int q = 0; q < 8; ++q) {
+            float v = 0.0f;
+            if (rp.valid && r < sg.k) {
+                const int ih = ih0 + r, iw = iw0 + s;
+                if (ih >= 0 && ih < sg.H && iw >= 0 && iw < sg.W) {
+                    const int off = (c * sg.H + ih) * sg.W + iw;
+                    v = sg.src_f32 ? __ldg(sf + off) : __uint_as_float((unsigned)__ldg(sh + off) << 16);
                 }
-                x[u * 8 + i] = v;
-                if (++c == sg.C) { c = 0; if (++s == sg.k) { s = 0; ++r; } }
             }
+            x.v[q] = v;
+            if (++c == sg.C) { c = 0; if (++s == sg.k) { s = 0; ++r; } }
         }
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            f8 v;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) v.v[i] = x[u * 8 + i];
-            st_shared16(a_chunk_addr(a_base, row, 2 * (2 * pair + u) + half), pack8(v));
-        }
+        st_shared16(a_chunk_addr(a_base, row, j), pack8(x));
     }
 }
 
@@ -421,7 +459,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
         *fail_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
-        if (dw_mode) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmH) : "memory");
+        if (dw_mode || g.stem_tma) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmH) : "memory");
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)g.tmem_cols) : "memory");
@@ -454,6 +492,19 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                     hn = grp * g.ni;
                     hy = (ty * g.step_y - g.off_y) * g.seg[0].stride - g.seg[0].pad;
                     hx = (tx * g.step_x - g.off_x) * g.seg[0].stride - g.seg[0].pad;
+                }
+                if (g.stem_tma) {
+                    // one image patch per tile: [C][ih][iwp], x origin rounded down to a 16-byte boundary
+                    const int i = (ti - (int)blockIdx.x) / (int)gridDim.x, hs = i % g.hstages;
+                    const int per = g.tiles_y * g.tiles_x, n = mt / per, t = mt - n * per;
+                    const int ty = t / g.tiles_x, tx = t - ty * g.tiles_x;
+                    const int iy0 = (ty * g.step_y - g.off_y) * g.seg[0].stride - g.seg[0].pad;
+                    const int ix0 = (tx * g.step_x - g.off_x) * g.seg[0].stride - g.seg[0].pad;
+                    const int x0 = ix0 - (((ix0 % g.stem_align) + g.stem_align) % g.stem_align);
+                    ok = mbar_wait(hempty_bar(hs), ((i / g.hstages) & 1) ^ 1u);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(hfull_bar(hs), (uint32_t)g.halo_bytes);
+                    tma_load_4d(sbase + g.off_halo + hs * g.halo_stride, &tmH, x0, iy0, 0, n, hfull_bar(hs));
                 }
                 for (int kb = 0; kb < g.kblocks && ok; ++kb, ++it) {
                     if (dw_mode) {
@@ -525,7 +576,17 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
             const int mt = ti / g.n_tiles;
             RowPos rp;
             rp.valid = 0; rp.n = 0; rp.p = 0; rp.q = 0;
-            if (!dw_mode) rp = map_row(g, mt, grow);
+            if (g.seg[0].mode == GA_GATHER || (g.seg[0].mode == GA_STEM && !g.stem_tma)) rp = map_row(g, mt, grow);
+            int xrem = 0, shs = 0;
+            if (g.stem_tma) {
+                const int i = (ti - (int)blockIdx.x) / (int)gridDim.x;
+                shs = i % g.hstages;
+                const int per = g.tiles_y * g.tiles_x, t = mt % per, tx = t % g.tiles_x;
+                const int ix0 = (tx * g.step_x - g.off_x) * g.seg[0].stride - g.seg[0].pad;
+                xrem = ((ix0 % g.stem_align) + g.stem_align) % g.stem_align;
+                ok = mbar_wait_warp(hfull_bar(shs), (i / g.hstages) & 1, lane);
+                if (!ok) break;
+            }
             GatherState gs0 = {0, 0, 0}, gs1 = {0, 0, 0};
             if (g.seg[0].mode == GA_GATHER && ghalf) gather_advance(gs0, 4, g.seg[0].C >> 3, g.seg[0].k);
             if (g.seg[1].mode == GA_GATHER && ghalf) gather_advance(gs1, 4, g.seg[1].C >> 3, g.seg[1].k);
@@ -559,11 +620,13 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                     warp_arrive(full_bar(s), lane);
                     warp_arrive(hempty_bar(hs), lane);     // the halo tile has been read
                 } else {
-                    produce_stem(sg, kbl, rp, a_base, grow, ghalf);
+                    if (g.stem_tma) produce_stem_tile(sg, g, kbl, sm + g.off_halo + shs * g.halo_stride, xrem, a_base, grow, ghalf);
+                    else produce_stem_direct(sg, kbl, rp, a_base, grow, ghalf);
                     fence_proxy_async();
                     warp_arrive(full_bar(s), lane);
                 }
             }
+            if (g.stem_tma && ok) warp_arrive(hempty_bar(shs), lane);      // the image patch has been read
         }
         if (!ok && lane == 0) atomicCAS(g.status, 0u, kStatusTimeout);
         cp_async_wait<0>();      // nothing of this thread is in flight when the CTA retires

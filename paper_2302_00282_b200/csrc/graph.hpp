@@ -126,6 +126,7 @@ struct Launch {
     int gap_imgs = 0, gap_area = 0, gap_rpi = 0;                                 // global-average epilogue
     int acc_stride = 0;                                            // columns between the two accumulators
     int hstages = 0, halo_bytes = 0, halo_stride = 0, halo_cb = 0;   // depthwise halo ring (halo_h x halo_w input pixels per image)
+    int stem_tma = 0, stem_align = 1;                              // stem: image patch by TMA, x alignment in elements
     int off_halo = 0, off_stg = 0, off_dww = 0, off_bias = 0, off_bar = 0;                    // shared-memory layout
     // ---- fp32 linked chain (conv kxk -> conv1x1 -> pool)
     int Cmid = 0, K2 = 0, act2 = 0;

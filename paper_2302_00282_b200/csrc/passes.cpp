@@ -215,12 +215,13 @@ static bool try_match(const LinkCtx &cx, int a, Allowed allowed, Chain &out) {
         return true;
     }
     if (A.kind == NK_CONV) {
-        if (!(g.tensors[A.in[0]].input_slot >= 0 && g.tensors[A.in[0]].io_layout == XENOS_LAYOUT_NCHW) && A.cin % 8)
-            return false;
+        // a convolution that reads the caller's NCHW image stages patches of it: it links with a pool only
+        const bool nchw_in = g.tensors[A.in[0]].input_slot >= 0 && g.tensors[A.in[0]].io_layout == XENOS_LAYOUT_NCHW;
+        if (!nchw_in && A.cin % 8) return false;
         int b = cx.sole(a);
         if (b < 0 || !allowed(b)) return false;
         const Node &B = g.nodes[b];
-        if (B.kind == NK_ADD) {
+        if (B.kind == NK_ADD && !nchw_in) {
             int other = B.in[0] == A.out ? B.in[1] : B.in[0];
             if (other == A.out) return false;
             out.kind = CK_CONV_TAIL;
@@ -251,7 +252,7 @@ static bool try_match(const LinkCtx &cx, int a, Allowed allowed, Chain &out) {
             out.pattern = "ConvX -> ZPooling (CBR-MaxPooling)";
             return true;
         }
-        if (B.kind == NK_GAP && cx.rows(a) <= 128) {
+        if (B.kind == NK_GAP && cx.rows(a) <= 128 && !nchw_in) {
             out.kind = CK_CONV_TAIL;
             out.nodes = {a, b};
             out.pattern = "ConvX -> ZPooling (CBR-AvgPooling, global)";
@@ -618,6 +619,37 @@ struct Lower {
             L.tile_rows = L.imgs_per_tile * L.rows_per_image;
             L.gap_imgs = L.imgs_per_tile; L.gap_area = L.rows_per_image; L.gap_rpi = L.rows_per_image;
         }
+        if (s0.mode == AM_STEM) {
+            // The stem stages the tile's input patch in shared memory, so its tile is a patch too:
+            // the pool patch when a pool is linked, else th x tw output pixels with the fewest tiles.
+            if (gapn) return fail(g, XENOS_E_UNSUPPORTED, "a convolution on an NCHW image cannot be linked with a global average");
+            if (!pooln) {
+                L.map_mode = MAP_PATCH;
+                L.ni = 1;
+                long best = -1;
+                for (int tw = 1; tw <= std::min(L.Q, 128); ++tw) {
+                    int th = std::min(L.P, 128 / tw);
+                    long tiles = (long)ceil_div(L.P, th) * ceil_div(L.Q, tw);
+                    if (best < 0 || tiles < best || (tiles == best && tw > L.patch_rw)) { best = tiles; L.patch_rh = th; L.patch_rw = tw; }
+                }
+                L.tiles_y = ceil_div(L.P, L.patch_rh); L.tiles_x = ceil_div(L.Q, L.patch_rw);
+                L.step_y = L.patch_rh; L.step_x = L.patch_rw; L.off_y = L.off_x = 0;
+                L.tile_rows = L.patch_rh * L.patch_rw;
+            }
+            // TMA fetches the patch when the image rows are 16-byte multiples; the box is widened so
+            // that its x origin can be rounded down to a 16-byte boundary
+            const int es = src.io_dtype == XENOS_DTYPE_F32 ? 4 : 2;
+            L.stem_align = 16 / es;
+            L.stem_tma = (src.w * es) % 16 == 0 ? 1 : 0;
+            L.halo_h = (L.patch_rh - 1) * M.stride + M.k;
+            L.halo_w = round_up((L.patch_rw - 1) * M.stride + M.k + L.stem_align - 1, L.stem_align);
+            L.halo_cb = src.c;
+            if (L.halo_h > 256 || L.halo_w > 256 || src.c > 256) L.stem_tma = 0;
+            if (L.stem_tma) {
+                L.halo_bytes = src.c * L.halo_h * L.halo_w * es;
+                L.halo_stride = (int)align_up((size_t)L.halo_bytes, 128);
+            }
+        }
         if (dw) {
             // The depthwise stage reads a halo tile that TMA fetches as one 4-D box, so the tile is a
             // patch: ni whole images when an image fits 128 rows, else th x tw output pixels of one image.
@@ -699,7 +731,7 @@ struct Lower {
         // a linked depthwise stage is bound by its own arithmetic, not by the MMA: give the halo ring
         // (the TMA prefetch distance) up to four stages first, the A|B ring keeps at least two
         L.hstages = 0;
-        if (dw) {
+        if (dw || L.stem_tma) {
             L.hstages = 2;
             while (L.hstages < 4 && cap - stg_bytes - (L.hstages + 1) * L.halo_stride >= 2 * stage_bytes) ++L.hstages;
         }

@@ -58,6 +58,24 @@ static xenos_status_t encode_halo_map(const Graph &g, Runtime *rt, const Launch 
     return XENOS_OK;
 }
 
+// 4-D map (W, H, C, N) over a small-channel NCHW image; box = one tile's input patch, all channels.
+static xenos_status_t encode_stem_map(const Graph &g, Runtime *rt, const Launch &L, void *base, CUtensorMap *out) {
+    const ASeg &a = L.seg[0];
+    const bool f32 = a.src_dtype == XENOS_DTYPE_F32;
+    const cuuint64_t es = f32 ? 4 : 2;
+    cuuint64_t dims[4] = {(cuuint64_t)a.W, (cuuint64_t)a.H, (cuuint64_t)a.C, (cuuint64_t)g.max_batch};
+    cuuint64_t strides[3] = {(cuuint64_t)a.W * es, (cuuint64_t)a.H * a.W * es, (cuuint64_t)a.C * a.H * a.W * es};
+    cuuint32_t box[4] = {(cuuint32_t)L.halo_w, (cuuint32_t)L.halo_h, (cuuint32_t)a.C, 1u};
+    cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+    if ((strides[0] & 15u) || (strides[1] & 15u) || (strides[2] & 15u) || (box[0] * es) % 16u || box[0] > 256u || box[1] > 256u || box[2] > 256u)
+        return fail(g, XENOS_E_CUDA, "internal: stem image patch violates the TMA limits");
+    CUresult r = rt->encode(out, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, estr,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(g, XENOS_E_CUDA, "cuTensorMapEncodeTiled (stem) failed with code " + std::to_string((int)r));
+    return XENOS_OK;
+}
+
 void runtime_free(Graph &g) {
     delete static_cast<Runtime *>(g.rt);
     g.rt = nullptr;
@@ -267,6 +285,7 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
             p.acc_stride = L.acc_stride; p.tmem_cols = L.tmem_cols;
             p.hstages = L.hstages; p.halo_bytes = L.halo_bytes; p.halo_stride = L.halo_stride;
             p.halo_h = L.halo_h; p.halo_w = L.halo_w; p.halo_cb = L.halo_cb;
+            p.stem_tma = L.stem_tma; p.stem_align = L.stem_align;
             p.off_halo = L.off_halo; p.off_stg = L.off_stg; p.off_dww = L.off_dww; p.off_bias = L.off_bias; p.off_bar = L.off_bar;
             p.act = L.act; p.act2 = L.act2; p.epi = L.epi; p.out_ctot = L.out_ctot; p.out_coff = L.out_coff;
             p.out_f32 = L.out_dtype == XENOS_DTYPE_F32;
@@ -278,6 +297,15 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
             // is a caller buffer its address is only known now
             const CUtensorMap *tmh = &rt->tmaps[li];
             CUtensorMap tmh_now;
+            if (L.stem_tma) {
+                // the image is a caller buffer: encode its patch map now
+                if (((uintptr_t)ptr(L.seg[0].tensor) & 15u) != 0) p.stem_tma = 0;      // unaligned image: direct loads
+                else {
+                    xenos_status_t st = encode_stem_map(g, rt, L, ptr(L.seg[0].tensor), &tmh_now);
+                    if (st != XENOS_OK) return st;
+                    tmh = &tmh_now;
+                }
+            }
             if (L.seg[0].mode == AM_DW) {
                 const Tensor &hx = g.tensors[L.seg[0].tensor];
                 if (hx.input_slot >= 0) {
