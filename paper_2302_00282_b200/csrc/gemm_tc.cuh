@@ -207,11 +207,67 @@ __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: 
 // ---- row <-> pixel -----------------------------------------------------------------------------
 struct RowPos { int valid, n, p, q; };
 
-__device__ __forceinline__ RowPos map_row(const GemmParams &g, int mt, int r) {
+// A ring of n slots with the phase bit of its barriers.
+struct Ring {
+    int s;
+    uint32_t ph;
+    __device__ __forceinline__ void next(int n) { if (++s == n) { s = 0; ph ^= 1u; } }
+};
+
+// Tiles are dealt round-robin: CTA b takes tiles b, b + grid, ...  The walk keeps (mt, nt) and, for
+// patch tiles, (image group, tile row, tile column) current with additions and carries, so that no
+// role divides inside its tile loop.
+struct TileWalk {
+    int ti, mt, nt, grp, ty, tx;
+    int d_mt, d_nt, d_grp, d_ty, d_tx;
+    __device__ __forceinline__ void init(const GemmParams &g) {
+        ti = (int)blockIdx.x; mt = ti / g.n_tiles; nt = ti - mt * g.n_tiles;
+        d_mt = (int)gridDim.x / g.n_tiles; d_nt = (int)gridDim.x - d_mt * g.n_tiles;
+        grp = ty = tx = d_grp = d_ty = d_tx = 0;
+        if (g.map_mode == GM_PATCH) {
+            const int per = g.tiles_y * g.tiles_x;
+            grp = mt / per;
+            int t = mt - grp * per;
+            ty = t / g.tiles_x; tx = t - ty * g.tiles_x;
+            d_grp = d_mt / per;
+            t = d_mt - d_grp * per;
+            d_ty = t / g.tiles_x; d_tx = t - d_ty * g.tiles_x;
+        }
+    }
+    __device__ __forceinline__ void next(const GemmParams &g) {
+        ti += (int)gridDim.x; mt += d_mt; nt += d_nt;
+        int carry = 0;
+        if (nt >= g.n_tiles) { nt -= g.n_tiles; ++mt; carry = 1; }
+        if (g.map_mode == GM_PATCH) {
+            tx += d_tx + carry;
+            if (tx >= g.tiles_x) { tx -= g.tiles_x; ++ty; }
+            ty += d_ty;
+            if (ty >= g.tiles_y) { ty -= g.tiles_y; ++grp; }
+            grp += d_grp;
+        }
+    }
+};
+
+// Position of tile row r inside a patch tile: fixed for a thread over the whole kernel.
+struct RowLocal { int img, dy, dx; };
+
+__device__ __forceinline__ RowLocal row_local(const GemmParams &g, int r) {
+    RowLocal l;
+    l.img = 0; l.dy = 0; l.dx = 0;
+    if (g.map_mode == GM_PATCH) {
+        const int area = g.rh * g.rw;
+        l.img = r / area;
+        const int rem = r - l.img * area;
+        l.dy = rem / g.rw; l.dx = rem - l.dy * g.rw;
+    }
+    return l;
+}
+
+__device__ __forceinline__ RowPos map_row(const GemmParams &g, const TileWalk &w, const RowLocal &l, int r) {
     RowPos o;
     o.valid = 0; o.n = 0; o.p = 0; o.q = 0;
     if (g.map_mode == GM_FLAT) {
-        const unsigned m = (unsigned)mt * (unsigned)g.tile_rows + (unsigned)r;     // < 2^31 rows by construction
+        const unsigned m = (unsigned)w.mt * (unsigned)g.tile_rows + (unsigned)r;     // < 2^31 rows by construction
         if (r < g.tile_rows && m < (unsigned)g.batch * (unsigned)g.rpi) {
             o.n = (int)(m / (unsigned)g.rpi);
             const int rem = (int)(m - (unsigned)o.n * (unsigned)g.rpi);
@@ -219,15 +275,10 @@ __device__ __forceinline__ RowPos map_row(const GemmParams &g, int mt, int r) {
             o.valid = 1;
         }
     } else {
-        const int per = g.tiles_y * g.tiles_x, area = g.rh * g.rw;
-        const int grp = mt / per, t = mt - grp * per;
-        const int ty = t / g.tiles_x, tx = t - ty * g.tiles_x;
-        const int img = r / area, rem = r - img * area;
-        const int dy = rem / g.rw, dx = rem - dy * g.rw;
-        o.n = grp * g.ni + img;
-        o.p = ty * g.step_y - g.off_y + dy;
-        o.q = tx * g.step_x - g.off_x + dx;
-        o.valid = (img < g.ni) && o.n < g.batch && o.p >= 0 && o.p < g.P && o.q >= 0 && o.q < g.Q;
+        o.n = w.grp * g.ni + l.img;
+        o.p = w.ty * g.step_y - g.off_y + l.dy;
+        o.q = w.tx * g.step_x - g.off_x + l.dx;
+        o.valid = (l.img < g.ni) && o.n < g.batch && o.p >= 0 && o.p < g.P && o.q >= 0 && o.q < g.Q;
     }
     return o;
 }
@@ -295,30 +346,30 @@ __device__ __forceinline__ void produce_gather(const GemmSeg &sg, GatherState st
 // per tile, prefetched through the halo ring; a row's K elements are then shared-memory reads.
 // thread = (row, half); it builds the chunks j = 2*i + half so that both halves share the real elements.
 __device__ __forceinline__ void produce_stem_tile(const GemmSeg &sg, const GemmParams &g, int kb_local, const uint8_t *patch,
-                                                  int xrem, uint32_t a_base, int row, int half) {
+                                                  const uint8_t *tab, int xrem, uint32_t a_base, int row, int half) {
+    // tab[e] = offset of K index e (tap-major, channel-minor) inside the patch, 0xFFFF for K padding
     const int area = g.rh * g.rw;
-    const bool live = row < area;
     const int dy = row / g.rw, dx = row - dy * g.rw;
-    const int base = (dy * sg.stride) * g.halo_w + xrem + dx * sg.stride;
-    const int plane = g.halo_h * g.halo_w;
-    const float *pf = reinterpret_cast<const float *>(patch);
-    const unsigned short *ph = reinterpret_cast<const unsigned short *>(patch);
-#pragma unroll 1
+    const int base = row < area ? (dy * sg.stride) * g.halo_w + xrem + dx * sg.stride : 0;   // rows past the tile read pixel 0; never stored
+    const float *pf = reinterpret_cast<const float *>(patch) + base;
+    const unsigned short *ph = reinterpret_cast<const unsigned short *>(patch) + base;
+    const uint4 *t4 = reinterpret_cast<const uint4 *>(tab) + kb_local * 8;
+#pragma unroll
     for (int i = 0; i < 4; ++i) {
         const int j = 2 * i + half;
-        int e = kb_local * kTileK + j * 8;
-        int tap = e / sg.C, c = e - tap * sg.C;
-        int r = tap / sg.k, s = tap - r * sg.k;
-        uint32_t w[4] = {0u, 0u, 0u, 0u};
+        const uint4 o4 = t4[j];
+        const uint32_t ow[4] = {o4.x, o4.y, o4.z, o4.w};
+        uint32_t w[4];
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            unsigned v = 0;
-            if (live && r < sg.k) {
-                const int idx = base + c * plane + r * g.halo_w + s;
-                v = sg.src_f32 ? (unsigned)__bfloat16_as_ushort(__float2bfloat16_rn(pf[idx])) : (unsigned)ph[idx];
+        for (int q = 0; q < 4; ++q) {
+            const uint32_t o0 = ow[q] & 0xFFFFu, o1 = ow[q] >> 16;
+            if (sg.src_f32) {
+                const float v0 = o0 != 0xFFFFu ? pf[o0] : 0.f, v1 = o1 != 0xFFFFu ? pf[o1] : 0.f;
+                w[q] = pack2(v0, v1);
+            } else {
+                const uint32_t v0 = o0 != 0xFFFFu ? (uint32_t)ph[o0] : 0u, v1 = o1 != 0xFFFFu ? (uint32_t)ph[o1] : 0u;
+                w[q] = v0 | (v1 << 16);
             }
-            w[q >> 1] |= v << ((q & 1) * 16);
-            if (++c == sg.C) { c = 0; if (++s == sg.k) { s = 0; ++r; } }
         }
         st_shared16(a_chunk_addr(a_base, row, j), make_uint4(w[0], w[1], w[2], w[3]));
     }
@@ -358,30 +409,32 @@ __device__ __forceinline__ void produce_stem_direct(const GemmSeg &sg, int kb_lo
 
 // depthwise 3x3 + bias + activation from the halo tile in shared memory ([image][y][x][cb channels],
 // dense bf16), rounded to bf16 and stored in the consumer's operand layout.
-// A thread owns 8 channels of FOUR horizontally adjacent output pixels (tile rows 4q .. 4q+3; the
-// tile's row pitch is a multiple of 4, so they share an image row).  It walks the 3 x (3S+3) input
-// window once: every input pixel is loaded and widened to fp32 once and feeds up to three outputs.
-struct DwUnit { int quad, j, base, live; };     // base: byte offset of the window origin in the halo tile
+// A thread owns 8 channels of PX horizontally adjacent output pixels (tile rows PX*u .. PX*u+PX-1;
+// the tile's row pitch is a multiple of 4, so they share an image row).  It walks the
+// 3 x ((PX-1)S+3) input window once: every input pixel is loaded and widened to fp32 once and feeds
+// up to three outputs.  PX = 4 when a K block has 64 channels, 2 when it has 32 (so that all
+// producer threads have a unit).
+struct DwUnit { int unit, j, base, live; };     // base: byte offset of the window origin in the halo tile
 
-template <int S>
+template <int S, int PX>
 __device__ __forceinline__ void produce_dw(const GemmSeg &sg, const GemmParams &g, int kb_local, uint32_t halo, uint32_t dww,
                                            const DwUnit &u, uint32_t a_base) {
-    if (u.quad >= 32) return;
+    if (u.unit >= kTileM / PX) return;
     const int c0 = kb_local * kTileK + u.j * 8;
-    const int r0 = u.quad * 4;
+    const int r0 = u.unit * PX;
     if (!u.live || c0 >= sg.C) {
 #pragma unroll
-        for (int o = 0; o < 4; ++o) st_shared16(a_chunk_addr(a_base, r0 + o, u.j), make_uint4(0u, 0u, 0u, 0u));
+        for (int o = 0; o < PX; ++o) st_shared16(a_chunk_addr(a_base, r0 + o, u.j), make_uint4(0u, 0u, 0u, 0u));
         return;
     }
     const int cbytes = g.halo_cb * 2;
     // accumulators, weights and pixels are kept as fp32 pairs: one packed FMA does two channels
-    float2 acc[4][4];
+    float2 acc[PX][4];
     {
         // tap weights [9][C] and the bias [C] were staged in shared memory when the CTA started
         const float4 b0 = ld_shared_f4(dww + (uint32_t)(9 * sg.C + c0) * 4u), b1 = ld_shared_f4(dww + (uint32_t)(9 * sg.C + c0 + 4) * 4u);
 #pragma unroll
-        for (int o = 0; o < 4; ++o) {
+        for (int o = 0; o < PX; ++o) {
             acc[o][0] = make_float2(b0.x, b0.y); acc[o][1] = make_float2(b0.z, b0.w);
             acc[o][2] = make_float2(b1.x, b1.y); acc[o][3] = make_float2(b1.z, b1.w);
         }
@@ -398,7 +451,7 @@ __device__ __forceinline__ void produce_dw(const GemmSeg &sg, const GemmParams &
             w[sx][2] = make_float2(w1.x, w1.y); w[sx][3] = make_float2(w1.z, w1.w);
         }
 #pragma unroll
-        for (int ci = 0; ci < 3 * S + 3; ++ci) {
+        for (int ci = 0; ci < (PX - 1) * S + 3; ++ci) {
             const uint4 raw = ld_shared16(hb + (uint32_t)((ry * g.halo_w + ci) * cbytes));
             const uint32_t rw4[4] = {raw.x, raw.y, raw.z, raw.w};
             float2 x[4];
@@ -406,7 +459,7 @@ __device__ __forceinline__ void produce_dw(const GemmSeg &sg, const GemmParams &
             for (int c = 0; c < 4; ++c) x[c] = make_float2(__uint_as_float(rw4[c] << 16), __uint_as_float(rw4[c] & 0xffff0000u));
 #pragma unroll
             for (int sx = 0; sx < 3; ++sx) {
-                if ((ci - sx) % S != 0 || ci - sx < 0 || (ci - sx) / S >= 4) continue;     // resolved at compile time
+                if ((ci - sx) % S != 0 || ci - sx < 0 || (ci - sx) / S >= PX) continue;     // resolved at compile time
                 const int o = (ci - sx) / S;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) acc[o][c] = __ffma2_rn(x[c], w[sx][c], acc[o][c]);
@@ -415,7 +468,7 @@ __device__ __forceinline__ void produce_dw(const GemmSeg &sg, const GemmParams &
     }
     const float lo = act_lo(sg.dw_act), hi = act_hi(sg.dw_act);
 #pragma unroll
-    for (int o = 0; o < 4; ++o) {
+    for (int o = 0; o < PX; ++o) {
         f8 r;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
@@ -473,6 +526,15 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
         for (int i = threadIdx.x - 64; i < 9 * C / 4; i += kProducerThreads) dst[i] = __ldg(w4 + i);
         for (int i = threadIdx.x - 64; i < C / 4; i += kProducerThreads) dst[9 * C / 4 + i] = __ldg(b4 + i);
     }
+    if (g.stem_tma && threadIdx.x >= 64 && threadIdx.x < 64 + kProducerThreads) {
+        // K index -> offset inside the image patch [C][halo_h][halo_w]
+        unsigned short *tab = reinterpret_cast<unsigned short *>(sm + g.off_dww);
+        const int C = g.seg[0].C, k = g.seg[0].k, kreal = C * k * k;
+        for (int e = threadIdx.x - 64; e < g.kblocks * kTileK; e += kProducerThreads) {
+            const int tap = e / C, c = e - tap * C, r = tap / k, s2 = tap - r * k;
+            tab[e] = e < kreal ? (unsigned short)(c * g.halo_h * g.halo_w + r * g.halo_w + s2) : (unsigned short)0xFFFFu;
+        }
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -482,43 +544,36 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
     if (warp == 0) {
         // ---- TMA: weight tiles, and the depthwise halo tiles ----
         if (lane == 0) {
-            int it = 0;
-            for (int ti = blockIdx.x; ti < total_tiles && ok; ti += gridDim.x) {
-                const int mt = ti / g.n_tiles, nt = ti - mt * g.n_tiles;
-                int hx = 0, hy = 0, hn = 0;
-                if (dw_mode) {
-                    const int per = g.tiles_y * g.tiles_x, grp = mt / per, t = mt - grp * per;
-                    const int ty = t / g.tiles_x, tx = t - ty * g.tiles_x;
-                    hn = grp * g.ni;
-                    hy = (ty * g.step_y - g.off_y) * g.seg[0].stride - g.seg[0].pad;
-                    hx = (tx * g.step_x - g.off_x) * g.seg[0].stride - g.seg[0].pad;
-                }
+            TileWalk w;
+            w.init(g);
+            Ring st = {0, 0u}, hr = {0, 0u};
+            for (; w.ti < total_tiles && ok; w.next(g)) {
+                // input origin of the tile's patch (depthwise halo / stem image patch)
+                const int hn = w.grp * g.ni;
+                const int hy = (w.ty * g.step_y - g.off_y) * g.seg[0].stride - g.seg[0].pad;
+                const int hx = (w.tx * g.step_x - g.off_x) * g.seg[0].stride - g.seg[0].pad;
                 if (g.stem_tma) {
                     // one image patch per tile: [C][ih][iwp], x origin rounded down to a 16-byte boundary
-                    const int i = (ti - (int)blockIdx.x) / (int)gridDim.x, hs = i % g.hstages;
-                    const int per = g.tiles_y * g.tiles_x, n = mt / per, t = mt - n * per;
-                    const int ty = t / g.tiles_x, tx = t - ty * g.tiles_x;
-                    const int iy0 = (ty * g.step_y - g.off_y) * g.seg[0].stride - g.seg[0].pad;
-                    const int ix0 = (tx * g.step_x - g.off_x) * g.seg[0].stride - g.seg[0].pad;
-                    const int x0 = ix0 - (((ix0 % g.stem_align) + g.stem_align) % g.stem_align);
-                    ok = mbar_wait(hempty_bar(hs), ((i / g.hstages) & 1) ^ 1u);
+                    // (stem_align is a power of two)
+                    ok = mbar_wait(hempty_bar(hr.s), hr.ph ^ 1u);
                     if (!ok) break;
-                    mbar_arrive_expect_tx(hfull_bar(hs), (uint32_t)g.halo_bytes);
-                    tma_load_4d(sbase + g.off_halo + hs * g.halo_stride, &tmH, x0, iy0, 0, n, hfull_bar(hs));
+                    mbar_arrive_expect_tx(hfull_bar(hr.s), (uint32_t)g.halo_bytes);
+                    tma_load_4d(sbase + g.off_halo + hr.s * g.halo_stride, &tmH, hx & ~(g.stem_align - 1), hy, 0, hn, hfull_bar(hr.s));
+                    hr.next(g.hstages);
                 }
-                for (int kb = 0; kb < g.kblocks && ok; ++kb, ++it) {
+                for (int kb = 0; kb < g.kblocks && ok; ++kb) {
                     if (dw_mode) {
-                        const int hs = it % g.hstages;
-                        ok = mbar_wait(hempty_bar(hs), ((it / g.hstages) & 1) ^ 1u);
+                        ok = mbar_wait(hempty_bar(hr.s), hr.ph ^ 1u);
                         if (!ok) break;
-                        mbar_arrive_expect_tx(hfull_bar(hs), (uint32_t)g.halo_bytes);
-                        tma_load_4d(sbase + g.off_halo + hs * g.halo_stride, &tmH, kb * kTileK, hx, hy, hn, hfull_bar(hs));
+                        mbar_arrive_expect_tx(hfull_bar(hr.s), (uint32_t)g.halo_bytes);
+                        tma_load_4d(sbase + g.off_halo + hr.s * g.halo_stride, &tmH, kb * kTileK, hx, hy, hn, hfull_bar(hr.s));
+                        hr.next(g.hstages);
                     }
-                    const int s = it % g.stages;
-                    ok = mbar_wait(empty_bar(s), ((it / g.stages) & 1) ^ 1u);
+                    ok = mbar_wait(empty_bar(st.s), st.ph ^ 1u);
                     if (!ok) break;
-                    mbar_arrive_expect_tx(full_bar(s), (uint32_t)g.tile_n * 128u);
-                    tma_load_2d(sbase + s * stage_bytes + kABytes, &tmB, kb * kTileK, nt * g.tile_n, full_bar(s));
+                    mbar_arrive_expect_tx(full_bar(st.s), (uint32_t)g.tile_n * 128u);
+                    tma_load_2d(sbase + st.s * stage_bytes + kABytes, &tmB, kb * kTileK, w.nt * g.tile_n, full_bar(st.s));
+                    st.next(g.stages);
                 }
             }
             if (!ok) atomicCAS(g.status, 0u, kStatusTimeout);
@@ -526,17 +581,19 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
     } else if (warp == 1) {
         // ---- MMA issue ----
         if (lane == 0) {
-            int it = 0, i = 0;
+            int i = 0;
+            Ring st = {0, 0u};
             for (int ti = blockIdx.x; ti < total_tiles && ok; ti += gridDim.x, ++i) {
                 const int b = i & 1;
                 ok = mbar_wait(acce_bar(b), ((i >> 1) & 1) ^ 1u);      // the epilogue has drained this accumulator
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + b * g.acc_stride;
-                for (int kb = 0; kb < g.kblocks && ok; ++kb, ++it) {
-                    const int s = it % g.stages;
-                    ok = mbar_wait(full_bar(s), (it / g.stages) & 1);
+                for (int kb = 0; kb < g.kblocks && ok; ++kb) {
+                    const int s = st.s;
+                    ok = mbar_wait(full_bar(s), st.ph);
                     if (!ok) break;
+                    st.next(g.stages);
                     // the activation tile was written through the generic proxy (cp.async / st.shared)
                     // and is read by the tensor core through the async proxy
                     fence_proxy_async();
@@ -557,43 +614,56 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
         const int pt = threadIdx.x - 64;                 // 0..255
         const int grow = pt & 127, ghalf = pt >> 7;      // gather / stem mapping
         DwUnit du;
-        du.quad = 32; du.j = 0; du.base = 0; du.live = 0;
+        du.unit = kTileM; du.j = 0; du.base = 0; du.live = 0;
         int zero_from = 8;                               // chunks >= zero_from of every row are K padding
+        const int dw_px = g.halo_cb > 32 ? 4 : 2;        // pixels per depthwise unit: every unit needs a thread
         if (dw_mode) {
             const int nj = g.halo_cb >> 3;               // 8-channel chunks per pixel in one K block
             zero_from = nj;
-            du.quad = pt / nj; du.j = pt - du.quad * nj;
-            if (du.quad < 32) {
-                const int area = g.rh * g.rw, r0 = du.quad * 4;
+            du.unit = pt / nj; du.j = pt - du.unit * nj;
+            if (du.unit < kTileM / dw_px) {
+                const int area = g.rh * g.rw, r0 = du.unit * dw_px;
                 const int img = r0 / area, rem = r0 - img * area;
                 const int dy = rem / g.rw, dx = rem - dy * g.rw;
                 du.live = img < g.ni;
                 du.base = ((img * g.halo_h + dy * g.seg[0].stride) * g.halo_w + dx * g.seg[0].stride) * g.halo_cb * 2 + du.j * 16;
             }
         }
-        int it = 0;
-        for (int ti = blockIdx.x; ti < total_tiles && ok; ti += gridDim.x) {
-            const int mt = ti / g.n_tiles;
+        // K-padding chunks of a depthwise stage are only ever written with zeros: when no other
+        // producer shares the ring they are cleared once, here, instead of with every K block
+        const bool zero_once = dw_mode && g.seg[1].mode == GA_NONE;
+        if (zero_once && zero_from < 8) {
+            const int nz = 8 - zero_from;
+            for (int idx = pt; idx < g.stages * kTileM * nz; idx += kProducerThreads) {
+                const int sr = idx / nz, jj = zero_from + idx - sr * nz, s = sr / kTileM, row = sr - s * kTileM;
+                st_shared16(a_chunk_addr(sbase + s * stage_bytes, row, jj), make_uint4(0u, 0u, 0u, 0u));
+            }
+            fence_proxy_async();      // ordered before every later arrival of this thread
+        }
+        const RowLocal rl = row_local(g, grow);
+        TileWalk w;
+        w.init(g);
+        Ring st = {0, 0u}, hr = {0, 0u};
+        for (; w.ti < total_tiles && ok; w.next(g)) {
             RowPos rp;
             rp.valid = 0; rp.n = 0; rp.p = 0; rp.q = 0;
-            if (g.seg[0].mode == GA_GATHER || (g.seg[0].mode == GA_STEM && !g.stem_tma)) rp = map_row(g, mt, grow);
+            if (g.seg[0].mode == GA_GATHER || (g.seg[0].mode == GA_STEM && !g.stem_tma)) rp = map_row(g, w, rl, grow);
             int xrem = 0, shs = 0;
             if (g.stem_tma) {
-                const int i = (ti - (int)blockIdx.x) / (int)gridDim.x;
-                shs = i % g.hstages;
-                const int per = g.tiles_y * g.tiles_x, t = mt % per, tx = t % g.tiles_x;
-                const int ix0 = (tx * g.step_x - g.off_x) * g.seg[0].stride - g.seg[0].pad;
-                xrem = ((ix0 % g.stem_align) + g.stem_align) % g.stem_align;
-                ok = mbar_wait_warp(hfull_bar(shs), (i / g.hstages) & 1, lane);
+                shs = hr.s;
+                xrem = ((w.tx * g.step_x - g.off_x) * g.seg[0].stride - g.seg[0].pad) & (g.stem_align - 1);
+                ok = mbar_wait_warp(hfull_bar(shs), hr.ph, lane);
                 if (!ok) break;
+                hr.next(g.hstages);
             }
             GatherState gs0 = {0, 0, 0}, gs1 = {0, 0, 0};
             if (g.seg[0].mode == GA_GATHER && ghalf) gather_advance(gs0, 4, g.seg[0].C >> 3, g.seg[0].k);
             if (g.seg[1].mode == GA_GATHER && ghalf) gather_advance(gs1, 4, g.seg[1].C >> 3, g.seg[1].k);
-            for (int kb = 0; kb < g.kblocks && ok; ++kb, ++it) {
-                const int s = it % g.stages;
-                ok = mbar_wait_warp(empty_bar(s), ((it / g.stages) & 1) ^ 1u, lane);
+            for (int kb = 0; kb < g.kblocks && ok; ++kb) {
+                const int s = st.s;
+                ok = mbar_wait_warp(empty_bar(s), st.ph ^ 1u, lane);
                 if (!ok) break;
+                st.next(g.stages);
                 const bool first = kb < g.seg[0].kblocks;
                 const GemmSeg &sg = first ? g.seg[0] : g.seg[1];
                 const int kbl = first ? kb : kb - g.seg[0].kblocks;
@@ -605,22 +675,29 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                     // thread itself moves on to the next stage at once
                     asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(full_bar(s)) : "memory");
                 } else if (sg.mode == GA_DW) {
-                    const int hs = it % g.hstages;
-                    ok = mbar_wait_warp(hfull_bar(hs), (it / g.hstages) & 1, lane);
+                    const int hs = hr.s;
+                    ok = mbar_wait_warp(hfull_bar(hs), hr.ph, lane);
                     if (!ok) break;
+                    hr.next(g.hstages);
                     const uint32_t halo = sbase + g.off_halo + hs * g.halo_stride, dww = sbase + g.off_dww;
-                    if (sg.stride == 1) produce_dw<1>(sg, g, kbl, halo, dww, du, a_base);
-                    else produce_dw<2>(sg, g, kbl, halo, dww, du, a_base);
-                    // K padding: chunks the block's channels do not reach must be zero, not stale
-                    for (int idx = pt; idx < kTileM * (8 - zero_from); idx += kProducerThreads) {
-                        const int row = idx / (8 - zero_from), jj = zero_from + idx - row * (8 - zero_from);
-                        st_shared16(a_chunk_addr(a_base, row, jj), make_uint4(0u, 0u, 0u, 0u));
+                    if (dw_px == 4) {
+                        if (sg.stride == 1) produce_dw<1, 4>(sg, g, kbl, halo, dww, du, a_base);
+                        else produce_dw<2, 4>(sg, g, kbl, halo, dww, du, a_base);
+                    } else {
+                        if (sg.stride == 1) produce_dw<1, 2>(sg, g, kbl, halo, dww, du, a_base);
+                        else produce_dw<2, 2>(sg, g, kbl, halo, dww, du, a_base);
                     }
+                    // K padding: chunks the block's channels do not reach must be zero, not stale
+                    if (!zero_once)
+                        for (int idx = pt; idx < kTileM * (8 - zero_from); idx += kProducerThreads) {
+                            const int row = idx / (8 - zero_from), jj = zero_from + idx - row * (8 - zero_from);
+                            st_shared16(a_chunk_addr(a_base, row, jj), make_uint4(0u, 0u, 0u, 0u));
+                        }
                     fence_proxy_async();
                     warp_arrive(full_bar(s), lane);
                     warp_arrive(hempty_bar(hs), lane);     // the halo tile has been read
                 } else {
-                    if (g.stem_tma) produce_stem_tile(sg, g, kbl, sm + g.off_halo + shs * g.halo_stride, xrem, a_base, grow, ghalf);
+                    if (g.stem_tma) produce_stem_tile(sg, g, kbl, sm + g.off_halo + shs * g.halo_stride, sm + g.off_dww, xrem, a_base, grow, ghalf);
                     else produce_stem_direct(sg, kbl, rp, a_base, grow, ghalf);
                     fence_proxy_async();
                     warp_arrive(full_bar(s), lane);
@@ -640,15 +717,18 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
         const int pool_pitch = g.tile_n * 2 + 16;
         const int nchunks = g.tile_n / 16;
         const float lo1 = act_lo(g.act), hi1 = act_hi(g.act), lo2 = act_lo(g.act2), hi2 = act_hi(g.act2);
+        const RowLocal rl = row_local(g, row);
+        TileWalk w;
+        w.init(g);
         int i = 0;
-        for (int ti = blockIdx.x; ti < total_tiles; ti += gridDim.x, ++i) {
-            const int mt = ti / g.n_tiles, nt = ti - mt * g.n_tiles;
+        for (; w.ti < total_tiles; w.next(g), ++i) {
+            const int mt = w.mt, nt = w.nt;
             const int b = i & 1;
             // this tile's bias slice goes to shared memory (double-buffered: a warp is at most one tile ahead)
             const uint32_t sbias = sbase + g.off_bias + b * 1024;
             if (et * 4 < g.tile_n)
                 *reinterpret_cast<float4 *>(sm + g.off_bias + b * 1024 + et * 16) = __ldg(reinterpret_cast<const float4 *>(g.bias + nt * g.tile_n) + et);
-            const RowPos rq = map_row(g, mt, row);
+            const RowPos rq = map_row(g, w, rl, row);
             const int n0 = nt * g.tile_n;
             const size_t pix = ((size_t)rq.n * g.P + rq.p) * g.Q + rq.q;
             // the four epilogue warps share named barriers below, so they must agree on giving up
@@ -739,9 +819,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
             }
             if (g.epi == GE_POOL) {
                 epi_bar();
-                const int per = g.tiles_y * g.tiles_x;
-                const int n = mt / per, tt = mt - n * per;
-                const int ty = tt / g.tiles_x, tx = tt - ty * g.tiles_x;
+                const int n = w.grp, ty = w.ty, tx = w.tx;      // pool tiles hold one image
                 const int c8n = g.tile_n / 8;
                 for (int item = et; item < g.pth * g.ptw * c8n; item += kEpilogueThreads) {
                     const int c8 = item % c8n, o = item / c8n;

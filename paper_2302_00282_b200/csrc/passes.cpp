@@ -644,7 +644,8 @@ struct Lower {
             L.halo_h = (L.patch_rh - 1) * M.stride + M.k;
             L.halo_w = round_up((L.patch_rw - 1) * M.stride + M.k + L.stem_align - 1, L.stem_align);
             L.halo_cb = src.c;
-            if (L.halo_h > 256 || L.halo_w > 256 || src.c > 256) L.stem_tma = 0;
+            // (patch offsets are kept as 16-bit table entries)
+            if (L.halo_h > 256 || L.halo_w > 256 || src.c > 256 || (long)src.c * L.halo_h * L.halo_w >= 65535) L.stem_tma = 0;
             if (L.stem_tma) {
                 L.halo_bytes = src.c * L.halo_h * L.halo_w * es;
                 L.halo_stride = (int)align_up((size_t)L.halo_bytes, 128);
@@ -726,7 +727,8 @@ struct Lower {
         int stg_bytes = L.epi == EPI_POOL ? 128 * (L.tile_n * 2 + 16) : (L.epi == EPI_GAP ? 128 * 17 * 4 : 0);
         stg_bytes = (int)align_up((size_t)stg_bytes, 128);
         // depthwise tap weights + bias of the linked stage (fp32 [10][C]) and two bias slices of the GEMM
-        int dww_bytes = dw ? (int)align_up((size_t)40 * src.c, 128) : 0;
+        // (a TMA-fed stem keeps its K-index -> patch-offset table there instead)
+        int dww_bytes = dw ? (int)align_up((size_t)40 * src.c, 128) : (L.stem_tma ? (int)align_up((size_t)L.kpad * 2, 128) : 0);
         int cap = std::min(g.hw.smem_bytes_per_cta, 227 * 1024) - 1024 - 256 - 2048 - dww_bytes;
         // a linked depthwise stage is bound by its own arithmetic, not by the MMA: give the halo ring
         // (the TMA prefetch distance) up to four stages first, the A|B ring keeps at least two
