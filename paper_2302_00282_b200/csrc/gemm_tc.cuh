@@ -44,7 +44,9 @@ constexpr int kABytes = kTileM * kTileK * 2;    // 16 KB per stage
 constexpr int kMaxStages = 6;
 constexpr int kMaxHaloStages = 4;
 constexpr int kProducerThreads = 256;           // warps 2..9
-constexpr int kEpilogueThreads = 128;           // warps 10..13
+constexpr int kParts = kProducerThreads / kTileM;      // gather / stem: threads per tile row
+constexpr int kChunksPerThread = 8 / kParts;    // 16-byte chunks of a row's K block per thread
+constexpr int kEpilogueThreads = 128;           // the last four warps
 constexpr int kThreads = 64 + kProducerThreads + kEpilogueThreads;
 constexpr unsigned kStatusTimeout = 0x80000000u | 9u;
 constexpr unsigned kStatusBounds = 0x80000000u | 10u;
@@ -305,9 +307,9 @@ __device__ __forceinline__ void gather_advance(GatherState &st, int n, int C8, i
     }
 }
 
-// gather: thread = (row, half); it copies chunks 4*half .. 4*half+3 of its row with 16-byte cp.async
+// gather: thread = (row, part); it copies kChunksPerThread adjacent chunks of its row with 16-byte cp.async
 __device__ __forceinline__ void produce_gather(const GemmSeg &sg, GatherState st, const RowPos &rp, uint32_t a_base,
-                                               int row, int half) {
+                                               int row, int part) {
     const __nv_bfloat16 *src = reinterpret_cast<const __nv_bfloat16 *>(sg.src);
     const int C8 = sg.C >> 3;
     const int ih0 = rp.p * sg.stride - sg.pad, iw0 = rp.q * sg.stride - sg.pad;
@@ -317,15 +319,15 @@ __device__ __forceinline__ void produce_gather(const GemmSeg &sg, GatherState st
         const bool in = rp.valid && st.tap_r == 0 && ih0 >= 0 && ih0 < sg.H && iw0 >= 0 && iw0 < sg.W;
         const __nv_bfloat16 *px = img + ((size_t)ih0 * sg.W + iw0) * sg.C;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < kChunksPerThread; ++i) {
             const int c8 = st.cc + i;          // with k == 1 the state's chunk counter runs from the segment start
             const bool live = in && c8 < C8;
-            cp_async16(a_chunk_addr(a_base, row, half * 4 + i), live ? (const void *)(px + c8 * 8) : (const void *)src, live ? 16u : 0u);
+            cp_async16(a_chunk_addr(a_base, row, part * kChunksPerThread + i), live ? (const void *)(px + c8 * 8) : (const void *)src, live ? 16u : 0u);
         }
         return;
     }
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < kChunksPerThread; ++i) {
         const void *ptr = src;
         uint32_t bytes = 0;
         if (rp.valid && st.tap_r < sg.k) {
@@ -335,7 +337,7 @@ __device__ __forceinline__ void produce_gather(const GemmSeg &sg, GatherState st
                 bytes = 16;
             }
         }
-        cp_async16(a_chunk_addr(a_base, row, half * 4 + i), ptr, bytes);
+        cp_async16(a_chunk_addr(a_base, row, part * kChunksPerThread + i), ptr, bytes);
         gather_advance(st, 1, C8, sg.k);
     }
 }
@@ -344,9 +346,9 @@ __device__ __forceinline__ void produce_gather(const GemmSeg &sg, GatherState st
 // Preferred form: TMA brings the tile's input patch [C][ih][iwp] to shared memory (4-D box whose x
 // origin is rounded down to a 16-byte boundary; out-of-range reads are zero = padding), one patch
 // per tile, prefetched through the halo ring; a row's K elements are then shared-memory reads.
-// thread = (row, half); it builds the chunks j = 2*i + half so that both halves share the real elements.
+// thread = (row, part); it builds the chunks j = kParts*i + part so that all parts share the real elements.
 __device__ __forceinline__ void produce_stem_tile(const GemmSeg &sg, const GemmParams &g, int kb_local, const uint8_t *patch,
-                                                  const uint8_t *tab, int xrem, uint32_t a_base, int row, int half) {
+                                                  const uint8_t *tab, int xrem, uint32_t a_base, int row, int part) {
     // tab[e] = offset of K index e (tap-major, channel-minor) inside the patch, 0xFFFF for K padding
     const int area = g.rh * g.rw;
     const int dy = row / g.rw, dx = row - dy * g.rw;
@@ -355,8 +357,8 @@ __device__ __forceinline__ void produce_stem_tile(const GemmSeg &sg, const GemmP
     const unsigned short *ph = reinterpret_cast<const unsigned short *>(patch) + base;
     const uint4 *t4 = reinterpret_cast<const uint4 *>(tab) + kb_local * 8;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int j = 2 * i + half;
+    for (int i = 0; i < kChunksPerThread; ++i) {
+        const int j = kParts * i + part;
         const uint4 o4 = t4[j];
         const uint32_t ow[4] = {o4.x, o4.y, o4.z, o4.w};
         uint32_t w[4];
@@ -378,14 +380,14 @@ __device__ __forceinline__ void produce_stem_tile(const GemmSeg &sg, const GemmP
 // Fallback when the image's row pitch is not a multiple of 16 bytes (TMA cannot address it): every
 // thread loads its row's elements straight from global memory.
 __device__ __forceinline__ void produce_stem_direct(const GemmSeg &sg, int kb_local, const RowPos &rp, uint32_t a_base,
-                                                    int row, int half) {
+                                                    int row, int part) {
     const int ih0 = rp.p * sg.stride - sg.pad, iw0 = rp.q * sg.stride - sg.pad;
     const size_t img = (size_t)rp.n * sg.C * sg.H * sg.W;
     const float *sf = reinterpret_cast<const float *>(sg.src) + img;
     const unsigned short *sh = reinterpret_cast<const unsigned short *>(sg.src) + img;
 #pragma unroll 1
-    for (int i = 0; i < 4; ++i) {
-        const int j = 2 * i + half;
+    for (int i = 0; i < kChunksPerThread; ++i) {
+        const int j = kParts * i + part;
         int e = kb_local * kTileK + j * 8;
         int tap = e / sg.C, c = e - tap * sg.C;
         int r = tap / sg.k, s = tap - r * sg.k;
@@ -409,73 +411,95 @@ __device__ __forceinline__ void produce_stem_direct(const GemmSeg &sg, int kb_lo
 
 // depthwise 3x3 + bias + activation from the halo tile in shared memory ([image][y][x][cb channels],
 // dense bf16), rounded to bf16 and stored in the consumer's operand layout.
-// A thread owns 8 channels of PX horizontally adjacent output pixels (tile rows PX*u .. PX*u+PX-1;
-// the tile's row pitch is a multiple of 4, so they share an image row).  It walks the
-// 3 x ((PX-1)S+3) input window once: every input pixel is loaded and widened to fp32 once and feeds
-// up to three outputs.  PX = 4 when a K block has 64 channels, 2 when it has 32 (so that all
-// producer threads have a unit).
-struct DwUnit { int unit, j, base, live; };     // base: byte offset of the window origin in the halo tile
+// A thread owns a BR x 4 block of output pixels for FOUR channels: it walks the block's input window
+// once with 8-byte loads (every input value is read once per block and feeds up to 3 * BR outputs)
+// and keeps the 36 tap weights in registers.  A 64-channel K block has 16 channel quads, so the 256
+// producer threads cover 16 blocks of 2 x 4 pixels; with 32 or fewer channels per K block they
+// cover 32 blocks of 1 x 4.
+struct DwUnit {
+    int q;          // channel quad inside the K block
+    int base;       // byte offset of the window origin in the halo tile (channel offset included)
+    int row0;       // tile row of the block's top-left output pixel
+    int nrows;      // live output rows of the block (the tile may end inside it)
+    int live;
+};
 
-template <int S, int PX>
+__device__ __forceinline__ uint32_t clamp_bf16x2(uint32_t v, uint32_t lo, uint32_t hi) {
+    __nv_bfloat162 x = *reinterpret_cast<__nv_bfloat162 *>(&v);
+    x = __hmin2(__hmax2(x, *reinterpret_cast<__nv_bfloat162 *>(&lo)), *reinterpret_cast<__nv_bfloat162 *>(&hi));
+    return *reinterpret_cast<uint32_t *>(&x);
+}
+
+template <int S, int BR>
 __device__ __forceinline__ void produce_dw(const GemmSeg &sg, const GemmParams &g, int kb_local, uint32_t halo, uint32_t dww,
                                            const DwUnit &u, uint32_t a_base) {
-    if (u.unit >= kTileM / PX) return;
-    const int c0 = kb_local * kTileK + u.j * 8;
-    const int r0 = u.unit * PX;
-    if (!u.live || c0 >= sg.C) {
+    if (!u.live) return;
+    const int c0 = kb_local * kTileK + u.q * 4;
+    const uint32_t half = (uint32_t)(u.q & 1) * 8u;      // which 8 bytes of the 16-byte chunk
+    const int j = u.q >> 1;
+    if (c0 >= sg.C) {
+        // K padding inside the block: zeros, so that the zero weights there never meet a NaN
+        for (int a = 0; a < u.nrows; ++a)
 #pragma unroll
-        for (int o = 0; o < PX; ++o) st_shared16(a_chunk_addr(a_base, r0 + o, u.j), make_uint4(0u, 0u, 0u, 0u));
+            for (int b = 0; b < 4; ++b) {
+                const int r = u.row0 + a * g.rw + b;
+                asm volatile("st.shared.v2.b32 [%0], {%1, %1};" ::"r"(a_chunk_addr(a_base, r, j) + half), "r"(0u) : "memory");
+            }
         return;
     }
-    const int cbytes = g.halo_cb * 2;
-    // accumulators, weights and pixels are kept as fp32 pairs: one packed FMA does two channels
-    float2 acc[PX][4];
-    {
-        // tap weights [9][C] and the bias [C] were staged in shared memory when the CTA started
-        const float4 b0 = ld_shared_f4(dww + (uint32_t)(9 * sg.C + c0) * 4u), b1 = ld_shared_f4(dww + (uint32_t)(9 * sg.C + c0 + 4) * 4u);
+    // tap weights [9][C] and the bias [C] were staged in shared memory when the CTA started
+    float2 w[9][2];
 #pragma unroll
-        for (int o = 0; o < PX; ++o) {
-            acc[o][0] = make_float2(b0.x, b0.y); acc[o][1] = make_float2(b0.z, b0.w);
-            acc[o][2] = make_float2(b1.x, b1.y); acc[o][3] = make_float2(b1.z, b1.w);
-        }
+    for (int t = 0; t < 9; ++t) {
+        const float4 wv = ld_shared_f4(dww + (uint32_t)(t * sg.C + c0) * 4u);
+        w[t][0] = make_float2(wv.x, wv.y); w[t][1] = make_float2(wv.z, wv.w);
+    }
+    float2 acc[BR][4][2];
+    {
+        const float4 bv = ld_shared_f4(dww + (uint32_t)(9 * sg.C + c0) * 4u);
+#pragma unroll
+        for (int a = 0; a < BR; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) { acc[a][b][0] = make_float2(bv.x, bv.y); acc[a][b][1] = make_float2(bv.z, bv.w); }
     }
     const uint32_t hb = halo + u.base;
+    const int cbytes = g.halo_cb * 2;
 #pragma unroll
-    for (int ry = 0; ry < 3; ++ry) {
-        float2 w[3][4];
+    for (int iy = 0; iy < (BR - 1) * S + 3; ++iy) {
 #pragma unroll
-        for (int sx = 0; sx < 3; ++sx) {
-            const uint32_t wa = dww + (uint32_t)((ry * 3 + sx) * sg.C + c0) * 4u;
-            const float4 w0 = ld_shared_f4(wa), w1 = ld_shared_f4(wa + 16);
-            w[sx][0] = make_float2(w0.x, w0.y); w[sx][1] = make_float2(w0.z, w0.w);
-            w[sx][2] = make_float2(w1.x, w1.y); w[sx][3] = make_float2(w1.z, w1.w);
-        }
+        for (int ci = 0; ci < 3 * S + 3; ++ci) {
+            uint32_t r0, r1;
+            asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(hb + (uint32_t)((iy * g.halo_w + ci) * cbytes)));
+            const float2 x0 = make_float2(__uint_as_float(r0 << 16), __uint_as_float(r0 & 0xffff0000u));
+            const float2 x1 = make_float2(__uint_as_float(r1 << 16), __uint_as_float(r1 & 0xffff0000u));
 #pragma unroll
-        for (int ci = 0; ci < (PX - 1) * S + 3; ++ci) {
-            const uint4 raw = ld_shared16(hb + (uint32_t)((ry * g.halo_w + ci) * cbytes));
-            const uint32_t rw4[4] = {raw.x, raw.y, raw.z, raw.w};
-            float2 x[4];
+            for (int ry = 0; ry < 3; ++ry) {
+                if ((iy - ry) % S != 0 || iy - ry < 0 || (iy - ry) / S >= BR) continue;      // resolved at compile time
+                const int a = (iy - ry) / S;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) x[c] = make_float2(__uint_as_float(rw4[c] << 16), __uint_as_float(rw4[c] & 0xffff0000u));
-#pragma unroll
-            for (int sx = 0; sx < 3; ++sx) {
-                if ((ci - sx) % S != 0 || ci - sx < 0 || (ci - sx) / S >= PX) continue;     // resolved at compile time
-                const int o = (ci - sx) / S;
-#pragma unroll
-                for (int c = 0; c < 4; ++c) acc[o][c] = __ffma2_rn(x[c], w[sx][c], acc[o][c]);
+                for (int sx = 0; sx < 3; ++sx) {
+                    if ((ci - sx) % S != 0 || ci - sx < 0 || (ci - sx) / S >= 4) continue;
+                    const int b = (ci - sx) / S;
+                    acc[a][b][0] = __ffma2_rn(x0, w[ry * 3 + sx][0], acc[a][b][0]);
+                    acc[a][b][1] = __ffma2_rn(x1, w[ry * 3 + sx][1], acc[a][b][1]);
+                }
             }
         }
     }
-    const float lo = act_lo(sg.dw_act), hi = act_hi(sg.dw_act);
+    // round to bf16, then clamp: the bounds 0 and 6 are bf16 values and rounding is monotonic, so
+    // this equals clamping first
+    const uint32_t lo = sg.dw_act >= 1 ? 0u : 0xff80ff80u;              // 0 | -inf, as bf16 pairs
+    const uint32_t hi = sg.dw_act == 2 ? 0x40c040c0u : 0x7f807f80u;     // 6 | +inf
 #pragma unroll
-    for (int o = 0; o < PX; ++o) {
-        f8 r;
+    for (int a = 0; a < BR; ++a) {
+        if (a >= u.nrows) break;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            r.v[2 * c] = fminf(fmaxf(acc[o][c].x, lo), hi);
-            r.v[2 * c + 1] = fminf(fmaxf(acc[o][c].y, lo), hi);
+        for (int b = 0; b < 4; ++b) {
+            const int r = u.row0 + a * g.rw + b;
+            const uint32_t p0 = clamp_bf16x2(pack2(acc[a][b][0].x, acc[a][b][0].y), lo, hi);
+            const uint32_t p1 = clamp_bf16x2(pack2(acc[a][b][1].x, acc[a][b][1].y), lo, hi);
+            asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(a_chunk_addr(a_base, r, j) + half), "r"(p0), "r"(p1) : "memory");
         }
-        st_shared16(a_chunk_addr(a_base, r0 + o, u.j), pack8(r));
     }
 }
 
@@ -503,12 +527,18 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
     // gather stages complete through cp.async arrivals (one per thread); the others through one
     // arrival per producer warp
     const bool async_gather = g.seg[0].mode == GA_GATHER;
+    // depthwise: the producer threads are (pixel block, channel quad of the K block) pairs
+    const int dw_quads = g.halo_cb > 32 ? 16 : 8;
+    const int dw_br = g.halo_cb > 32 ? 2 : 1;       // block rows
 
     if (threadIdx.x == 0) {
-        const uint32_t full_count = (async_gather ? kProducerThreads : kProducerThreads / 32) + 1;
+        // arrivals on a stage's "full" barrier: the TMA lane plus the producers of that stage (every
+        // thread for cp.async gathers, every warp otherwise)
+        const uint32_t prod_warps = kProducerThreads / 32;
+        const uint32_t full_count = (async_gather ? kProducerThreads : prod_warps) + 1;
         for (int s = 0; s < g.stages; ++s) { mbar_init(full_bar(s), full_count); mbar_init(empty_bar(s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), kEpilogueThreads / 32); }
-        for (int s = 0; s < g.hstages; ++s) { mbar_init(hfull_bar(s), 1); mbar_init(hempty_bar(s), kProducerThreads / 32); }
+        for (int s = 0; s < g.hstages; ++s) { mbar_init(hfull_bar(s), 1); mbar_init(hempty_bar(s), prod_warps); }
         *fail_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
@@ -612,22 +642,22 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
     } else if (warp < 2 + kProducerThreads / 32) {
         // ---- activation operand ----
         const int pt = threadIdx.x - 64;                 // 0..255
-        const int grow = pt & 127, ghalf = pt >> 7;      // gather / stem mapping
+        const int grow = pt & 127, gpart = pt >> 7;      // gather / stem mapping
         DwUnit du;
-        du.unit = kTileM; du.j = 0; du.base = 0; du.live = 0;
+        du.q = 0; du.base = 0; du.row0 = 0; du.nrows = 0; du.live = 0;
         int zero_from = 8;                               // chunks >= zero_from of every row are K padding
-        const int dw_px = g.halo_cb > 32 ? 4 : 2;        // pixels per depthwise unit: every unit needs a thread
         if (dw_mode) {
-            const int nj = g.halo_cb >> 3;               // 8-channel chunks per pixel in one K block
-            zero_from = nj;
-            du.unit = pt / nj; du.j = pt - du.unit * nj;
-            if (du.unit < kTileM / dw_px) {
-                const int area = g.rh * g.rw, r0 = du.unit * dw_px;
-                const int img = r0 / area, rem = r0 - img * area;
-                const int dy = rem / g.rw, dx = rem - dy * g.rw;
-                du.live = img < g.ni;
-                du.base = ((img * g.halo_h + dy * g.seg[0].stride) * g.halo_w + dx * g.seg[0].stride) * g.halo_cb * 2 + du.j * 16;
-            }
+            zero_from = g.halo_cb >> 3;
+            du.q = pt & (dw_quads - 1);
+            const int blk = pt / dw_quads;               // (image, block row, block column)
+            const int upr = g.rw >> 2, upi = ((g.rh + dw_br - 1) / dw_br) * upr;
+            const int img = blk / upi, rem = blk - img * upi;
+            const int uy = rem / upr, ux = rem - uy * upr;
+            const int S = g.seg[0].stride;
+            du.live = img < g.ni && du.q * 4 < g.halo_cb;
+            du.base = ((img * g.halo_h + dw_br * uy * S) * g.halo_w + 4 * ux * S) * g.halo_cb * 2 + du.q * 8;
+            du.row0 = img * g.rh * g.rw + dw_br * uy * g.rw + 4 * ux;
+            du.nrows = min(dw_br, max(0, g.rh - dw_br * uy));
         }
         // K-padding chunks of a depthwise stage are only ever written with zeros: when no other
         // producer shares the ring they are cleared once, here, instead of with every K block
@@ -657,35 +687,35 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                 hr.next(g.hstages);
             }
             GatherState gs0 = {0, 0, 0}, gs1 = {0, 0, 0};
-            if (g.seg[0].mode == GA_GATHER && ghalf) gather_advance(gs0, 4, g.seg[0].C >> 3, g.seg[0].k);
-            if (g.seg[1].mode == GA_GATHER && ghalf) gather_advance(gs1, 4, g.seg[1].C >> 3, g.seg[1].k);
+            if (g.seg[0].mode == GA_GATHER && gpart) gather_advance(gs0, gpart * kChunksPerThread, g.seg[0].C >> 3, g.seg[0].k);
+            if (g.seg[1].mode == GA_GATHER && gpart) gather_advance(gs1, gpart * kChunksPerThread, g.seg[1].C >> 3, g.seg[1].k);
             for (int kb = 0; kb < g.kblocks && ok; ++kb) {
-                const int s = st.s;
-                ok = mbar_wait_warp(empty_bar(s), st.ph ^ 1u, lane);
-                if (!ok) break;
+                const int s = st.s, hs = hr.s;
+                const uint32_t sph = st.ph, hph = hr.ph;
                 st.next(g.stages);
                 const bool first = kb < g.seg[0].kblocks;
                 const GemmSeg &sg = first ? g.seg[0] : g.seg[1];
                 const int kbl = first ? kb : kb - g.seg[0].kblocks;
+                if (sg.mode == GA_DW) hr.next(g.hstages);
+                ok = mbar_wait_warp(empty_bar(s), sph ^ 1u, lane);
+                if (!ok) break;
                 const uint32_t a_base = sbase + s * stage_bytes;
                 if (sg.mode == GA_GATHER) {
-                    if (first) { produce_gather(sg, gs0, rp, a_base, grow, ghalf); gather_advance(gs0, 8, sg.C >> 3, sg.k); }
-                    else { produce_gather(sg, gs1, rp, a_base, grow, ghalf); gather_advance(gs1, 8, sg.C >> 3, sg.k); }
+                    if (first) { produce_gather(sg, gs0, rp, a_base, grow, gpart); gather_advance(gs0, 8, sg.C >> 3, sg.k); }
+                    else { produce_gather(sg, gs1, rp, a_base, grow, gpart); gather_advance(gs1, 8, sg.C >> 3, sg.k); }
                     // the stage's barrier is signalled when this thread's copies have landed; the
                     // thread itself moves on to the next stage at once
                     asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(full_bar(s)) : "memory");
                 } else if (sg.mode == GA_DW) {
-                    const int hs = hr.s;
-                    ok = mbar_wait_warp(hfull_bar(hs), hr.ph, lane);
+                    ok = mbar_wait_warp(hfull_bar(hs), hph, lane);
                     if (!ok) break;
-                    hr.next(g.hstages);
                     const uint32_t halo = sbase + g.off_halo + hs * g.halo_stride, dww = sbase + g.off_dww;
-                    if (dw_px == 4) {
-                        if (sg.stride == 1) produce_dw<1, 4>(sg, g, kbl, halo, dww, du, a_base);
-                        else produce_dw<2, 4>(sg, g, kbl, halo, dww, du, a_base);
-                    } else {
+                    if (dw_br == 2) {
                         if (sg.stride == 1) produce_dw<1, 2>(sg, g, kbl, halo, dww, du, a_base);
                         else produce_dw<2, 2>(sg, g, kbl, halo, dww, du, a_base);
+                    } else {
+                        if (sg.stride == 1) produce_dw<1, 1>(sg, g, kbl, halo, dww, du, a_base);
+                        else produce_dw<2, 1>(sg, g, kbl, halo, dww, du, a_base);
                     }
                     // K padding: chunks the block's channels do not reach must be zero, not stale
                     if (!zero_once)
@@ -697,8 +727,8 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                     warp_arrive(full_bar(s), lane);
                     warp_arrive(hempty_bar(hs), lane);     // the halo tile has been read
                 } else {
-                    if (g.stem_tma) produce_stem_tile(sg, g, kbl, sm + g.off_halo + shs * g.halo_stride, sm + g.off_dww, xrem, a_base, grow, ghalf);
-                    else produce_stem_direct(sg, kbl, rp, a_base, grow, ghalf);
+                    if (g.stem_tma) produce_stem_tile(sg, g, kbl, sm + g.off_halo + shs * g.halo_stride, sm + g.off_dww, xrem, a_base, grow, gpart);
+                    else produce_stem_direct(sg, kbl, rp, a_base, grow, gpart);
                     fence_proxy_async();
                     warp_arrive(full_bar(s), lane);
                 }

@@ -182,7 +182,8 @@ static bool try_match(const LinkCtx &cx, int a, Allowed allowed, Chain &out) {
         out.pattern = "ConvX -> ConvY (depthwise 3x3 -> pointwise 1x1)";
         int c = cx.sole(b);
         const Tensor &bo = g.tensors[B.out];
-        if (c >= 0 && allowed(c) && g.nodes[c].kind == NK_GAP && bo.h * ((bo.w + 3) / 4 * 4) <= 128) {
+        if (c >= 0 && allowed(c) && g.nodes[c].kind == NK_GAP && bo.h * ((bo.w + 3) / 4 * 4) <= 128 &&
+            ((bo.h + 1) / 2) * ((bo.w + 3) / 4) <= 16) {     // whole images per tile, in 2 x 4 pixel blocks
             out.nodes.push_back(c);
             out.pattern = "ConvX -> ConvY -> ZPooling (depthwise -> pointwise -> global average)";
         }
@@ -656,15 +657,19 @@ struct Lower {
             // patch: ni whole images when an image fits 128 rows, else th x tw output pixels of one image.
             L.map_mode = MAP_PATCH;
             // the tile's row pitch is a multiple of 4: a producer thread owns 4 adjacent pixels of a row
+            // ... made of br x 4 pixel blocks, the unit of work of a depthwise producer thread: 16 blocks of
+            // 2 x 4 when a K block has 64 channels, 32 blocks of 1 x 4 otherwise
             const int Qp = round_up(L.Q, 4);
-            if (L.P * Qp <= 128) {
-                L.ni = 128 / (L.P * Qp); L.patch_rh = L.P; L.patch_rw = Qp;
+            const int br = std::min(64, src.c) > 32 ? 2 : 1, nblk = br == 2 ? 16 : 32;
+            auto blocks_of = [&](int th, int tw) { return ceil_div(th, br) * (tw / 4); };
+            if (L.P * Qp <= 128 && blocks_of(L.P, Qp) <= nblk) {
+                L.ni = std::min(128 / (L.P * Qp), nblk / blocks_of(L.P, Qp)); L.patch_rh = L.P; L.patch_rw = Qp;
             } else {
                 if (gapn) return fail(g, XENOS_E_UNSUPPORTED, "internal: global average needs whole images per tile");
                 L.ni = 1;
                 long best = -1;
-                for (int tw = 4; tw <= std::min(Qp, 128); tw += 4) {
-                    int th = std::min(L.P, 128 / tw);
+                for (int tw = 4; tw <= std::min(Qp, 64); tw += 4) {
+                    int th = std::min(L.P, br * (nblk / (tw / 4)));
                     long tiles = (long)ceil_div(L.P, th) * ceil_div(L.Q, tw);
                     // fewest tiles first; then the widest tile (longest contiguous rows in memory)
                     if (best < 0 || tiles < best || (tiles == best && tw > L.patch_rw)) { best = tiles; L.patch_rh = th; L.patch_rw = tw; }
@@ -672,14 +677,15 @@ struct Lower {
             }
             // keep one halo tile (64 channels of the input window) small enough for a 2-3 deep ring
             auto halo_of = [&](int ni, int th, int tw) {
-                return (long)ni * ((th - 1) * dw->stride + 3) * ((tw - 1) * dw->stride + 3) * std::min(64, src.c) * 2;
+                return (long)ni * ((round_up(th, br) - 1) * dw->stride + 3) * ((tw - 1) * dw->stride + 3) * std::min(64, src.c) * 2;
             };
             while (L.ni > 1 && halo_of(L.ni, L.patch_rh, L.patch_rw) > 40 * 1024) --L.ni;
             while (!gapn && L.patch_rh > 1 && halo_of(L.ni, L.patch_rh, L.patch_rw) > 76 * 1024) --L.patch_rh;
             L.tiles_y = ceil_div(L.P, L.patch_rh); L.tiles_x = ceil_div(L.Q, L.patch_rw);
             L.step_y = L.patch_rh; L.step_x = L.patch_rw; L.off_y = L.off_x = 0;
             L.tile_rows = L.ni * L.patch_rh * L.patch_rw;
-            L.halo_h = (L.patch_rh - 1) * dw->stride + 3; L.halo_w = (L.patch_rw - 1) * dw->stride + 3;
+            // (the box covers whole blocks: a producer thread reads its block's full window)
+            L.halo_h = (round_up(L.patch_rh, br) - 1) * dw->stride + 3; L.halo_w = (L.patch_rw - 1) * dw->stride + 3;
             L.halo_cb = std::min(64, src.c);
             L.halo_bytes = L.ni * L.halo_h * L.halo_w * L.halo_cb * 2;
             L.halo_stride = (int)align_up((size_t)L.halo_bytes, 128);
