@@ -204,6 +204,11 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float *v) {
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// Programmatic dependent launch: let the next kernel of the stream be scheduled early / wait until
+// the previous kernel's memory is complete and visible (no-ops without the launch attribute).
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 // ---- row <-> pixel -----------------------------------------------------------------------------
@@ -507,6 +512,9 @@ __device__ __forceinline__ void produce_dw(const GemmSeg &sg, const GemmParams &
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmH, const GemmParams g) {
     extern __shared__ uint8_t smem_raw[];
+    // every CTA of this grid is resident (one per SM at most), so the next kernel can be scheduled
+    // as soon as they have all started: it fills SMs as they drain and waits before touching data
+    pdl_launch_dependents();
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t sbase = (raw + 1023u) & ~1023u;
     uint8_t *sm = smem_raw + (sbase - raw);
@@ -570,6 +578,8 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     bool ok = true;
+    // set-up touched constants only (weights, bias, tables); activations are the previous kernel's
+    if (warp != 1) pdl_wait();
 
     if (warp == 0) {
         // ---- TMA: weight tiles, and the depthwise halo tiles ----

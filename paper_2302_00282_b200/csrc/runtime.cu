@@ -317,7 +317,18 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
                 }
             }
             const int grid = std::min(p.m_tiles * L.n_tiles, sms);
-            xk::gemm_chain_kernel<<<grid, xk::kThreads, L.smem_bytes, stream>>>(rt->tmaps[li], *tmh, p);
+            // Programmatic dependent launch: the kernel may be scheduled while its predecessor in the
+            // stream drains, runs its set-up (barriers, tensor memory, constant staging) and then
+            // waits (griddepcontrol.wait) before it touches any activation.
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3((unsigned)xk::kThreads);
+            cfg.dynamicSmemBytes = (size_t)L.smem_bytes; cfg.stream = stream;
+            cudaLaunchAttribute at[1];
+            at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            at[0].val.programmaticStreamSerializationAllowed = 1;
+            cfg.attrs = at; cfg.numAttrs = 1;
+            cudaError_t le = cudaLaunchKernelEx(&cfg, xk::gemm_chain_kernel, rt->tmaps[li], *tmh, p);
+            if (le != cudaSuccess) return cuda_fail(g, "kernel launch", le);
             break;
         }
         default:
