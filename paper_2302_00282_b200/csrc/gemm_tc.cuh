@@ -757,24 +757,39 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
         const int pool_pitch = g.tile_n * 2 + 16;
         const int nchunks = g.tile_n / 16;
         const float lo1 = act_lo(g.act), hi1 = act_hi(g.act), lo2 = act_lo(g.act2), hi2 = act_hi(g.act2);
+        // the common epilogue (bias, one activation, bf16 store or pool) runs on packed pairs
+        const bool fast = !g.skip && !g.act2 && !g.out_f32 && g.epi != GE_GAP;
+        const uint32_t plo = g.act >= 1 ? 0u : 0xff80ff80u, phi = g.act == 2 ? 0x40c040c0u : 0x7f807f80u;
+        // 32-byte stores need a 32-byte aligned row start and column offset
+        const bool wide_ok = ((reinterpret_cast<uintptr_t>(g.out) | (uintptr_t)(g.out_ctot * 2) | (uintptr_t)(g.out_coff * 2)) & 31u) == 0;
         const RowLocal rl = row_local(g, row);
         TileWalk w;
         w.init(g);
-        int i = 0;
+        int i = 0, bias_nt = -1, bias_buf = 0;
         for (; w.ti < total_tiles; w.next(g), ++i) {
             const int mt = w.mt, nt = w.nt;
             const int b = i & 1;
-            // this tile's bias slice goes to shared memory (double-buffered: a warp is at most one tile ahead)
-            const uint32_t sbias = sbase + g.off_bias + b * 1024;
-            if (et * 4 < g.tile_n)
-                *reinterpret_cast<float4 *>(sm + g.off_bias + b * 1024 + et * 16) = __ldg(reinterpret_cast<const float4 *>(g.bias + nt * g.tile_n) + et);
+            // the bias slice of this channel tile goes to shared memory when the channel tile changes
+            // (two buffers: a warp is at most one tile ahead of the others)
+            const bool new_bias = nt != bias_nt;
+            if (new_bias) {
+                bias_nt = nt; bias_buf ^= 1;
+                if (et * 4 < g.tile_n)
+                    *reinterpret_cast<float4 *>(sm + g.off_bias + bias_buf * 1024 + et * 16) = __ldg(reinterpret_cast<const float4 *>(g.bias + nt * g.tile_n) + et);
+            }
+            const uint32_t sbias = sbase + g.off_bias + bias_buf * 1024;
             const RowPos rq = map_row(g, w, rl, row);
             const int n0 = nt * g.tile_n;
             const size_t pix = ((size_t)rq.n * g.P + rq.p) * g.Q + rq.q;
-            // the four epilogue warps share named barriers below, so they must agree on giving up
-            if (!mbar_wait_warp(accf_bar(b), (i >> 1) & 1, lane) && lane == 0) *fail_flag = 1;
-            epi_bar();
-            if (*fail_flag) { ok = false; break; }
+            if (g.epi == GE_STORE && !new_bias) {
+                // plain stores share nothing between the warps: each waits for the accumulator by itself
+                if (!mbar_wait_warp(accf_bar(b), (i >> 1) & 1, lane)) { ok = false; break; }
+            } else {
+                // the four epilogue warps share named barriers below, so they must agree on giving up
+                if (!mbar_wait_warp(accf_bar(b), (i >> 1) & 1, lane) && lane == 0) *fail_flag = 1;
+                epi_bar();
+                if (*fail_flag) { ok = false; break; }
+            }
             tc_fence_after();
             const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * g.acc_stride;
             for (int cbase = 0; cbase < nchunks; cbase += 2) {
@@ -793,6 +808,39 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                     float *v = vv + 16 * sub;
                     const int ch = cbase + sub;
                     const int nc = n0 + ch * 16;
+                    if (fast) {
+                        // bias as packed fp32 adds, rounding to bf16 pairs, activation as a clamp on the pairs
+                        // (0 and 6 are bf16 values and rounding is monotonic: same result as clamping first)
+                        uint32_t pk[8];
+#pragma unroll
+                        for (int q4 = 0; q4 < 16; q4 += 4) {
+                            const float4 bz = ld_shared_f4(sbias + (uint32_t)(ch * 16 + q4) * 4u);
+                            const float2 t0 = __fadd2_rn(make_float2(v[q4], v[q4 + 1]), make_float2(bz.x, bz.y));
+                            const float2 t1 = __fadd2_rn(make_float2(v[q4 + 2], v[q4 + 3]), make_float2(bz.z, bz.w));
+                            pk[q4 / 2] = clamp_bf16x2(pack2(t0.x, t0.y), plo, phi);
+                            pk[q4 / 2 + 1] = clamp_bf16x2(pack2(t1.x, t1.y), plo, phi);
+                        }
+                        if (g.epi == GE_STORE) {
+                            if (!rq.valid) continue;
+                            __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(g.out) + pix * g.out_ctot + g.out_coff + nc;
+                            if (nc + 16 <= g.N && wide_ok) {
+                                asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(o), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]),
+                                             "r"(pk[3]), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7]) : "memory");
+                            } else {
+                                if (nc + 8 <= g.N) *reinterpret_cast<uint4 *>(o) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                                if (nc + 16 <= g.N) *reinterpret_cast<uint4 *>(o + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                            }
+                        } else {
+                            // rows outside the conv output never win a max
+                            if (!rq.valid) {
+#pragma unroll
+                                for (int q = 0; q < 8; ++q) pk[q] = 0xff80ff80u;
+                            }
+                            st_shared16(stg + row * pool_pitch + ch * 32, make_uint4(pk[0], pk[1], pk[2], pk[3]));
+                            st_shared16(stg + row * pool_pitch + ch * 32 + 16, make_uint4(pk[4], pk[5], pk[6], pk[7]));
+                        }
+                        continue;
+                    }
 #pragma unroll
                     for (int q4 = 0; q4 < 16; q4 += 4) {
                         const float4 bz = ld_shared_f4(sbias + (uint32_t)(ch * 16 + q4) * 4u);
