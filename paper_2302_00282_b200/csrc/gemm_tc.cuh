@@ -885,20 +885,46 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                         for (int c = 0; c < 8; ++c) { lo.v[c] = rq.valid ? v[c] : -INFINITY; hi.v[c] = rq.valid ? v[8 + c] : -INFINITY; }
                         st_shared16(stg + row * pool_pitch + ch * 32, pack8(lo));
                         st_shared16(stg + row * pool_pitch + ch * 32 + 16, pack8(hi));
-                    } else {
-                        // global average: 16 columns at a time through shared memory, rows summed in ascending order
-                        epi_bar();
+                    }
+                    // (global average: the activated values stay in vv for the reduction below)
+                }
+                if (g.epi == GE_GAP) {
+                    // global average of up to 32 columns through shared memory: every thread parks its
+                    // row, then (image, column, part) items sum the rows r = part, part + parts, ... in
+                    // ascending order and the parts are added in ascending order: a fixed order
+                    const int ncols = nsub * 16, nc0 = n0 + cbase * 16;
+                    const int per = g.gap_imgs * 32;
+                    const int parts = per >= 128 ? 1 : (per >= 64 ? 2 : 4);
+                    float *part = stgf + kTileM * 33;
+                    epi_bar();          // the previous slab's readers are done
 #pragma unroll
-                        for (int c = 0; c < 16; ++c) stgf[row * 17 + c] = rq.valid ? v[c] : 0.0f;
+                    for (int c = 0; c < 32; ++c)
+                        if (c < ncols) stgf[row * 33 + c] = rq.valid ? vv[c] : 0.0f;
+                    epi_bar();
+                    for (int item = et; item < per * parts; item += kEpilogueThreads) {
+                        const int c = item & 31, rest = item >> 5;
+                        const int img = rest / parts, pa = rest - img * parts;
+                        float acc = 0.0f;
+                        if (c < ncols)
+                            for (int r = pa; r < g.gap_area; r += parts) acc += stgf[(img * g.gap_area + r) * 33 + c];
+                        if (parts > 1) { part[item] = acc; continue; }
+                        const int n = mt * g.gap_imgs + img;
+                        if (c >= ncols || n >= g.batch || nc0 + c >= g.N) continue;
+                        acc /= (float)g.gap_rpi;
+                        const size_t oi = (size_t)n * g.out_ctot + g.out_coff + nc0 + c;
+                        if (g.out_f32) reinterpret_cast<float *>(g.out)[oi] = acc;
+                        else reinterpret_cast<__nv_bfloat16 *>(g.out)[oi] = __float2bfloat16_rn(acc);
+                    }
+                    if (parts > 1) {
                         epi_bar();
-                        for (int item = et; item < g.gap_imgs * 16; item += kEpilogueThreads) {
-                            const int img = item >> 4, c = item & 15;
+                        for (int item = et; item < per; item += kEpilogueThreads) {
+                            const int c = item & 31, img = item >> 5;
                             const int n = mt * g.gap_imgs + img;
-                            if (n >= g.batch || nc + c >= g.N) continue;
+                            if (c >= ncols || n >= g.batch || nc0 + c >= g.N) continue;
                             float acc = 0.0f;
-                            for (int r = 0; r < g.gap_area; ++r) acc += stgf[(img * g.gap_area + r) * 17 + c];
+                            for (int pa = 0; pa < parts; ++pa) acc += part[((img * parts + pa) << 5) + c];
                             acc /= (float)g.gap_rpi;
-                            const size_t oi = (size_t)n * g.out_ctot + g.out_coff + nc + c;
+                            const size_t oi = (size_t)n * g.out_ctot + g.out_coff + nc0 + c;
                             if (g.out_f32) reinterpret_cast<float *>(g.out)[oi] = acc;
                             else reinterpret_cast<__nv_bfloat16 *>(g.out)[oi] = __float2bfloat16_rn(acc);
                         }

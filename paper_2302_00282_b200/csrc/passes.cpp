@@ -730,7 +730,7 @@ struct Lower {
         if (L.tmem_cols > g.hw.tmem_columns) return fail(g, XENOS_E_BAD_SPLIT, "split: accumulator tiles exceed tensor memory columns");
         // shared memory of the one persistent CTA per SM: [A|B ring][halo ring][epilogue staging][barriers]
         int stage_bytes = 16384 + L.tile_n * 128;
-        int stg_bytes = L.epi == EPI_POOL ? 128 * (L.tile_n * 2 + 16) : (L.epi == EPI_GAP ? 128 * 17 * 4 : 0);
+        int stg_bytes = L.epi == EPI_POOL ? 128 * (L.tile_n * 2 + 16) : (L.epi == EPI_GAP ? 128 * 33 * 4 + 512 : 0);
         stg_bytes = (int)align_up((size_t)stg_bytes, 128);
         // depthwise tap weights + bias of the linked stage (fp32 [10][C]) and two bias slices of the GEMM
         // (a TMA-fed stem keeps its K-index -> patch-offset table there instead)
