@@ -353,17 +353,18 @@ __device__ __forceinline__ void produce_gather(const GemmSeg &sg, GatherState st
 // per tile, prefetched through the halo ring; a row's K elements are then shared-memory reads.
 // thread = (row, part); it builds the chunks j = kParts*i + part so that all parts share the real elements.
 __device__ __forceinline__ void produce_stem_tile(const GemmSeg &sg, const GemmParams &g, int kb_local, const uint8_t *patch,
-                                                  const uint8_t *tab, int xrem, uint32_t a_base, int row, int part) {
-    // tab[e] = offset of K index e (tap-major, channel-minor) inside the patch, 0xFFFF for K padding
-    const int area = g.rh * g.rw;
-    const int dy = row / g.rw, dx = row - dy * g.rw;
-    const int base = row < area ? (dy * sg.stride) * g.halo_w + xrem + dx * sg.stride : 0;   // rows past the tile read pixel 0; never stored
+                                                  const uint8_t *tab, int xrem, uint32_t a_base, int row, int part,
+                                                  const RowLocal &rl, int jlimit) {
+    // tab[e] = offset of K index e (tap-major, channel-minor) inside the patch, 0xFFFF for K padding;
+    // chunks >= jlimit are K padding that the caller has cleared already
+    const int base = rl.img == 0 ? (rl.dy * sg.stride) * g.halo_w + xrem + rl.dx * sg.stride : 0;   // rows past the tile read pixel 0; never stored
     const float *pf = reinterpret_cast<const float *>(patch) + base;
     const unsigned short *ph = reinterpret_cast<const unsigned short *>(patch) + base;
     const uint4 *t4 = reinterpret_cast<const uint4 *>(tab) + kb_local * 8;
 #pragma unroll
     for (int i = 0; i < kChunksPerThread; ++i) {
         const int j = kParts * i + part;
+        if (j >= jlimit) break;
         const uint4 o4 = t4[j];
         const uint32_t ow[4] = {o4.x, o4.y, o4.z, o4.w};
         uint32_t w[4];
@@ -684,18 +685,43 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
         TileWalk w;
         w.init(g);
         Ring st = {0, 0u}, hr = {0, 0u};
-        for (; w.ti < total_tiles && ok; w.next(g)) {
-            RowPos rp;
-            rp.valid = 0; rp.n = 0; rp.p = 0; rp.q = 0;
-            if (g.seg[0].mode == GA_GATHER || (g.seg[0].mode == GA_STEM && !g.stem_tma)) rp = map_row(g, w, rl, grow);
-            int xrem = 0, shs = 0;
-            if (g.stem_tma) {
-                shs = hr.s;
-                xrem = ((w.tx * g.step_x - g.off_x) * g.seg[0].stride - g.seg[0].pad) & (g.stem_align - 1);
+        if (g.stem_tma) {
+            // ---- stem: one image patch per tile, its K blocks gathered from the patch ----
+            const GemmSeg &sg = g.seg[0];
+            // with a single K block its padding chunks never change: cleared once, then skipped
+            int jlimit = 8;
+            if (g.kblocks == 1) {
+                jlimit = (sg.C * sg.k * sg.k + 7) >> 3;
+                const int nz = 8 - jlimit;
+                for (int idx = pt; idx < g.stages * kTileM * nz; idx += kProducerThreads) {
+                    const int sr = idx / nz, jj = jlimit + idx - sr * nz, s = sr / kTileM, row = sr - s * kTileM;
+                    st_shared16(a_chunk_addr(sbase + s * stage_bytes, row, jj), make_uint4(0u, 0u, 0u, 0u));
+                }
+                fence_proxy_async();      // ordered before every later arrival of this thread
+            }
+            for (; w.ti < total_tiles && ok; w.next(g)) {
+                const int shs = hr.s;
+                const int xrem = ((w.tx * g.step_x - g.off_x) * sg.stride - sg.pad) & (g.stem_align - 1);
                 ok = mbar_wait_warp(hfull_bar(shs), hr.ph, lane);
                 if (!ok) break;
                 hr.next(g.hstages);
+                for (int kb = 0; kb < g.kblocks && ok; ++kb) {
+                    const int s = st.s;
+                    ok = mbar_wait_warp(empty_bar(s), st.ph ^ 1u, lane);
+                    if (!ok) break;
+                    st.next(g.stages);
+                    produce_stem_tile(sg, g, kb, sm + g.off_halo + shs * g.halo_stride, sm + g.off_dww, xrem, sbase + s * stage_bytes, grow, gpart, rl, jlimit);
+                    fence_proxy_async();
+                    warp_arrive(full_bar(s), lane);
+                }
+                if (ok) warp_arrive(hempty_bar(shs), lane);      // the image patch has been read
             }
+        }
+        // ---- general form: gathers (one or two K segments), depthwise stages, direct stem loads ----
+        for (; !g.stem_tma && w.ti < total_tiles && ok; w.next(g)) {
+            RowPos rp;
+            rp.valid = 0; rp.n = 0; rp.p = 0; rp.q = 0;
+            if (g.seg[0].mode == GA_GATHER || g.seg[0].mode == GA_STEM) rp = map_row(g, w, rl, grow);
             GatherState gs0 = {0, 0, 0}, gs1 = {0, 0, 0};
             if (g.seg[0].mode == GA_GATHER && gpart) gather_advance(gs0, gpart * kChunksPerThread, g.seg[0].C >> 3, g.seg[0].k);
             if (g.seg[1].mode == GA_GATHER && gpart) gather_advance(gs1, gpart * kChunksPerThread, g.seg[1].C >> 3, g.seg[1].k);
@@ -737,13 +763,11 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                     warp_arrive(full_bar(s), lane);
                     warp_arrive(hempty_bar(hs), lane);     // the halo tile has been read
                 } else {
-                    if (g.stem_tma) produce_stem_tile(sg, g, kbl, sm + g.off_halo + shs * g.halo_stride, sm + g.off_dww, xrem, a_base, grow, gpart);
-                    else produce_stem_direct(sg, kbl, rp, a_base, grow, gpart);
+                    produce_stem_direct(sg, kbl, rp, a_base, grow, gpart);
                     fence_proxy_async();
                     warp_arrive(full_bar(s), lane);
                 }
             }
-            if (g.stem_tma && ok) warp_arrive(hempty_bar(shs), lane);      // the image patch has been read
         }
         if (!ok && lane == 0) atomicCAS(g.status, 0u, kStatusTimeout);
         cp_async_wait<0>();      // nothing of this thread is in flight when the CTA retires
