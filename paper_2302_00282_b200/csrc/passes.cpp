@@ -680,6 +680,9 @@ struct Lower {
                 return (long)ni * ((round_up(th, br) - 1) * dw->stride + 3) * ((tw - 1) * dw->stride + 3) * std::min(64, src.c) * 2;
             };
             while (L.ni > 1 && halo_of(L.ni, L.patch_rh, L.patch_rw) > 40 * 1024) --L.ni;
+            // the depthwise stage is recomputed per channel tile and its time grows with the tile's pixels:
+            // while SMs would stay idle, fewer images per tile spread it over more of them
+            while (L.ni > 1 && (long)ceil_div(g.max_batch, L.ni) * ceil_div(round_up(N, 16), 256) * 2 <= g.hw.sm_count) --L.ni;
             while (!gapn && L.patch_rh > 1 && halo_of(L.ni, L.patch_rh, L.patch_rw) > 76 * 1024) --L.patch_rh;
             L.tiles_y = ceil_div(L.P, L.patch_rh); L.tiles_x = ceil_div(L.Q, L.patch_rw);
             L.step_y = L.patch_rh; L.step_x = L.patch_rw; L.off_y = L.off_x = 0;
