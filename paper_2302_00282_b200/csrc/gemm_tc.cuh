@@ -553,6 +553,12 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
         if (dw_mode || g.stem_tma) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmH) : "memory");
     }
+    if (warp == 0) {
+        // The TMA lane needs the barriers only: warp 0 signals that they exist and goes straight to its
+        // loads, while the other warps allocate tensor memory and stage constants before they wait.
+        __syncwarp();
+        asm volatile("bar.arrive 3, %0;" ::"r"(kThreads) : "memory");
+    }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)g.tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -575,9 +581,9 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
         }
     }
     tc_fence_before();
-    __syncthreads();
+    if (warp != 0) asm volatile("bar.sync 3, %0;" ::"r"(kThreads) : "memory");
     tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_base = warp != 0 ? *tmem_slot : 0u;
     bool ok = true;
     // set-up touched constants only (weights, bias, tables); activations are the previous kernel's
     if (warp != 1) pdl_wait();
