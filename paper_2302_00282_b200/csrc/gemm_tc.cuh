@@ -331,6 +331,17 @@ __device__ __forceinline__ void produce_gather(const GemmSeg &sg, GatherState st
         }
         return;
     }
+    if ((sg.C & 63) == 0) {
+        // a K block lies inside one tap and the thread's chunks are adjacent channels of one input pixel:
+        // one bounds check and one address for all of them
+        const int ih = ih0 + st.tap_r, iw = iw0 + st.tap_s;
+        const bool live = rp.valid && st.tap_r < sg.k && ih >= 0 && ih < sg.H && iw >= 0 && iw < sg.W;
+        const __nv_bfloat16 *px = live ? img + ((size_t)ih * sg.W + iw) * sg.C + st.cc * 8 : src;
+#pragma unroll
+        for (int i = 0; i < kChunksPerThread; ++i)
+            cp_async16(a_chunk_addr(a_base, row, part * kChunksPerThread + i), live ? (const void *)(px + i * 8) : (const void *)src, live ? 16u : 0u);
+        return;
+    }
 #pragma unroll
     for (int i = 0; i < kChunksPerThread; ++i) {
         const void *ptr = src;
