@@ -113,6 +113,13 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, in
     ok = __shfl_sync(0xffffffffu, ok, 0);
     return ok != 0;
 }
+// Two barriers, one poller, one broadcast.
+__device__ __forceinline__ bool mbar_wait2_warp(uint32_t bar_a, uint32_t par_a, uint32_t bar_b, uint32_t par_b, int lane) {
+    int ok = 1;
+    if (lane == 0) ok = (mbar_wait(bar_a, par_a) && mbar_wait(bar_b, par_b)) ? 1 : 0;
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    return ok != 0;
+}
 // Every lane has finished (and fenced) its own accesses; one arrival per warp.
 __device__ __forceinline__ void warp_arrive(uint32_t bar, int lane) {
     __syncwarp();
@@ -312,49 +319,30 @@ __device__ __forceinline__ void gather_advance(GatherState &st, int n, int C8, i
     }
 }
 
-// gather: thread = (row, part); it copies kChunksPerThread adjacent chunks of its row with 16-byte cp.async
-__device__ __forceinline__ void produce_gather(const GemmSeg &sg, GatherState st, const RowPos &rp, uint32_t a_base,
-                                               int row, int part) {
+// gather: a thread copies ONE 16-byte chunk j of FOUR tile rows (row0, row0 + 32, ...) per K block, so
+// that the eight lanes that share a row read its 128 contiguous bytes: whole lines leave L2, not a
+// 16-byte piece of 32 different lines per instruction.
+struct GatherRow { int pb, ih0, iw0; };      // element index and coordinates of the row's window origin
+
+__device__ __forceinline__ GatherRow gather_row(const GemmSeg &sg, const RowPos &rp) {
+    GatherRow r;
+    r.ih0 = rp.p * sg.stride - sg.pad; r.iw0 = rp.q * sg.stride - sg.pad;
+    r.pb = (rp.n * sg.H + r.ih0) * sg.W + r.iw0;
+    if (!rp.valid) r.ih0 = -(1 << 20);       // every tap of a row outside the tile is out of range
+    return r;
+}
+
+__device__ __forceinline__ void produce_gather(const GemmSeg &sg, const GatherState &st, const GatherRow (&gr)[4], uint32_t a_base,
+                                               int row0, int j) {
     const __nv_bfloat16 *src = reinterpret_cast<const __nv_bfloat16 *>(sg.src);
-    const int C8 = sg.C >> 3;
-    const int ih0 = rp.p * sg.stride - sg.pad, iw0 = rp.q * sg.stride - sg.pad;
-    const __nv_bfloat16 *img = src + (size_t)rp.n * sg.H * sg.W * sg.C;
-    if (sg.k == 1) {
-        // pointwise: the row's channel vector is contiguous, chunk c of the K block is 16 bytes at c*16
-        const bool in = rp.valid && st.tap_r == 0 && ih0 >= 0 && ih0 < sg.H && iw0 >= 0 && iw0 < sg.W;
-        const __nv_bfloat16 *px = img + ((size_t)ih0 * sg.W + iw0) * sg.C;
+    const bool live_tap = st.tap_r < sg.k;                 // false: K padding behind the last tap
+    const int tapoff = st.tap_r * sg.W + st.tap_s;
 #pragma unroll
-        for (int i = 0; i < kChunksPerThread; ++i) {
-            const int c8 = st.cc + i;          // with k == 1 the state's chunk counter runs from the segment start
-            const bool live = in && c8 < C8;
-            cp_async16(a_chunk_addr(a_base, row, part * kChunksPerThread + i), live ? (const void *)(px + c8 * 8) : (const void *)src, live ? 16u : 0u);
-        }
-        return;
-    }
-    if ((sg.C & 63) == 0) {
-        // a K block lies inside one tap and the thread's chunks are adjacent channels of one input pixel:
-        // one bounds check and one address for all of them
-        const int ih = ih0 + st.tap_r, iw = iw0 + st.tap_s;
-        const bool live = rp.valid && st.tap_r < sg.k && ih >= 0 && ih < sg.H && iw >= 0 && iw < sg.W;
-        const __nv_bfloat16 *px = live ? img + ((size_t)ih * sg.W + iw) * sg.C + st.cc * 8 : src;
-#pragma unroll
-        for (int i = 0; i < kChunksPerThread; ++i)
-            cp_async16(a_chunk_addr(a_base, row, part * kChunksPerThread + i), live ? (const void *)(px + i * 8) : (const void *)src, live ? 16u : 0u);
-        return;
-    }
-#pragma unroll
-    for (int i = 0; i < kChunksPerThread; ++i) {
-        const void *ptr = src;
-        uint32_t bytes = 0;
-        if (rp.valid && st.tap_r < sg.k) {
-            int ih = ih0 + st.tap_r, iw = iw0 + st.tap_s;
-            if (ih >= 0 && ih < sg.H && iw >= 0 && iw < sg.W) {
-                ptr = img + ((size_t)ih * sg.W + iw) * sg.C + st.cc * 8;
-                bytes = 16;
-            }
-        }
-        cp_async16(a_chunk_addr(a_base, row, part * kChunksPerThread + i), ptr, bytes);
-        gather_advance(st, 1, C8, sg.k);
+    for (int i = 0; i < 4; ++i) {
+        const int ih = gr[i].ih0 + st.tap_r, iw = gr[i].iw0 + st.tap_s;
+        const bool live = live_tap && (unsigned)ih < (unsigned)sg.H && (unsigned)iw < (unsigned)sg.W;
+        const __nv_bfloat16 *ptr = src + ((size_t)(gr[i].pb + tapoff) * sg.C + st.cc * 8);
+        cp_async16(a_chunk_addr(a_base, row0 + 32 * i, j), live ? (const void *)ptr : (const void *)src, live ? 16u : 0u);
     }
 }
 
@@ -734,41 +722,23 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                 if (ok) warp_arrive(hempty_bar(shs), lane);      // the image patch has been read
             }
         }
-        // ---- general form: gathers (one or two K segments), depthwise stages, direct stem loads ----
-        for (; !g.stem_tma && w.ti < total_tiles && ok; w.next(g)) {
-            RowPos rp;
-            rp.valid = 0; rp.n = 0; rp.p = 0; rp.q = 0;
-            if (g.seg[0].mode == GA_GATHER || g.seg[0].mode == GA_STEM) rp = map_row(g, w, rl, grow);
-            GatherState gs0 = {0, 0, 0}, gs1 = {0, 0, 0};
-            if (g.seg[0].mode == GA_GATHER && gpart) gather_advance(gs0, gpart * kChunksPerThread, g.seg[0].C >> 3, g.seg[0].k);
-            if (g.seg[1].mode == GA_GATHER && gpart) gather_advance(gs1, gpart * kChunksPerThread, g.seg[1].C >> 3, g.seg[1].k);
-            for (int kb = 0; kb < g.kblocks && ok; ++kb) {
-                const int s = st.s, hs = hr.s;
-                const uint32_t sph = st.ph, hph = hr.ph;
-                st.next(g.stages);
-                const bool first = kb < g.seg[0].kblocks;
-                const GemmSeg &sg = first ? g.seg[0] : g.seg[1];
-                const int kbl = first ? kb : kb - g.seg[0].kblocks;
-                if (sg.mode == GA_DW) hr.next(g.hstages);
-                ok = mbar_wait_warp(empty_bar(s), sph ^ 1u, lane);
-                if (!ok) break;
-                const uint32_t a_base = sbase + s * stage_bytes;
-                if (sg.mode == GA_GATHER) {
-                    if (first) { produce_gather(sg, gs0, rp, a_base, grow, gpart); gather_advance(gs0, 8, sg.C >> 3, sg.k); }
-                    else { produce_gather(sg, gs1, rp, a_base, grow, gpart); gather_advance(gs1, 8, sg.C >> 3, sg.k); }
-                    // the stage's barrier is signalled when this thread's copies have landed; the
-                    // thread itself moves on to the next stage at once
-                    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(full_bar(s)) : "memory");
-                } else if (sg.mode == GA_DW) {
-                    ok = mbar_wait_warp(hfull_bar(hs), hph, lane);
+        if (dw_mode) {
+            // ---- depthwise stage of a linked chain: every K block comes from a halo tile ----
+            const uint32_t dww = sbase + g.off_dww;
+            const GemmSeg &sg = g.seg[0];
+            for (; w.ti < total_tiles && ok; w.next(g)) {
+                for (int kb = 0; kb < g.kblocks && ok; ++kb) {
+                    const int s = st.s, hs = hr.s;
+                    ok = mbar_wait2_warp(empty_bar(s), st.ph ^ 1u, hfull_bar(hs), hr.ph, lane);
                     if (!ok) break;
-                    const uint32_t halo = sbase + g.off_halo + hs * g.halo_stride, dww = sbase + g.off_dww;
+                    st.next(g.stages); hr.next(g.hstages);
+                    const uint32_t a_base = sbase + s * stage_bytes, halo = sbase + g.off_halo + hs * g.halo_stride;
                     if (dw_br == 2) {
-                        if (sg.stride == 1) produce_dw<1, 2>(sg, g, kbl, halo, dww, du, a_base);
-                        else produce_dw<2, 2>(sg, g, kbl, halo, dww, du, a_base);
+                        if (sg.stride == 1) produce_dw<1, 2>(sg, g, kb, halo, dww, du, a_base);
+                        else produce_dw<2, 2>(sg, g, kb, halo, dww, du, a_base);
                     } else {
-                        if (sg.stride == 1) produce_dw<1, 1>(sg, g, kbl, halo, dww, du, a_base);
-                        else produce_dw<2, 1>(sg, g, kbl, halo, dww, du, a_base);
+                        if (sg.stride == 1) produce_dw<1, 1>(sg, g, kb, halo, dww, du, a_base);
+                        else produce_dw<2, 1>(sg, g, kb, halo, dww, du, a_base);
                     }
                     // K padding: chunks the block's channels do not reach must be zero, not stale
                     if (!zero_once)
@@ -777,8 +747,48 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                             st_shared16(a_chunk_addr(a_base, row, jj), make_uint4(0u, 0u, 0u, 0u));
                         }
                     fence_proxy_async();
-                    warp_arrive(full_bar(s), lane);
-                    warp_arrive(hempty_bar(hs), lane);     // the halo tile has been read
+                    __syncwarp();
+                    if (lane == 0) { mbar_arrive(full_bar(s)); mbar_arrive(hempty_bar(hs)); }     // stage filled, halo tile read
+                }
+            }
+        }
+        // ---- general form: gathers (one or two K segments), direct stem loads ----
+        const int grow0 = pt >> 3, gj = pt & 7;          // gather mapping: rows grow0 + 32 i, chunk gj
+        RowLocal grl[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) grl[i] = row_local(g, grow0 + 32 * i);
+        for (; !g.stem_tma && !dw_mode && w.ti < total_tiles && ok; w.next(g)) {
+            RowPos rp;
+            rp.valid = 0; rp.n = 0; rp.p = 0; rp.q = 0;
+            if (g.seg[0].mode == GA_STEM) rp = map_row(g, w, rl, grow);
+            GatherRow gr0[4], gr1[4];
+            GatherState gs0 = {0, 0, 0}, gs1 = {0, 0, 0};
+            if (g.seg[0].mode == GA_GATHER) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const RowPos r4 = map_row(g, w, grl[i], grow0 + 32 * i);
+                    gr0[i] = gather_row(g.seg[0], r4);
+                    gr1[i] = gather_row(g.seg[1], r4);       // (unused without a second segment)
+                }
+                if (gj) gather_advance(gs0, gj, g.seg[0].C >> 3, g.seg[0].k);
+                if (g.seg[1].mode == GA_GATHER && gj) gather_advance(gs1, gj, g.seg[1].C >> 3, g.seg[1].k);
+            }
+            for (int kb = 0; kb < g.kblocks && ok; ++kb) {
+                const int s = st.s;
+                const uint32_t sph = st.ph;
+                st.next(g.stages);
+                const bool first = kb < g.seg[0].kblocks;
+                const GemmSeg &sg = first ? g.seg[0] : g.seg[1];
+                const int kbl = first ? kb : kb - g.seg[0].kblocks;
+                ok = mbar_wait_warp(empty_bar(s), sph ^ 1u, lane);
+                if (!ok) break;
+                const uint32_t a_base = sbase + s * stage_bytes;
+                if (sg.mode == GA_GATHER) {
+                    if (first) { produce_gather(sg, gs0, gr0, a_base, grow0, gj); gather_advance(gs0, 8, sg.C >> 3, sg.k); }
+                    else { produce_gather(sg, gs1, gr1, a_base, grow0, gj); gather_advance(gs1, 8, sg.C >> 3, sg.k); }
+                    // the stage's barrier is signalled when this thread's copies have landed; the
+                    // thread itself moves on to the next stage at once
+                    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(full_bar(s)) : "memory");
                 } else {
                     produce_stem_direct(sg, kbl, rp, a_base, grow, gpart);
                     fence_proxy_async();
