@@ -346,12 +346,17 @@ __device__ __forceinline__ void produce_gather(const GemmSeg &sg, const GatherSt
     }
 }
 
-// stem (small-channel NCHW image, fp32 or bf16), K element e = (r * k + s) * C + c.
+// stem (small-channel NCHW image, fp32 or bf16).  For k > 4, K is made of (channel c, tap row r) segments of
+// kp = 8 elements, K index = (c * k + r) * kp + s: the taps s of one window row,
+// which are adjacent in the image, so a 16-byte operand chunk is one or two short copies and not
+// eight gathered elements.  Elements s >= k of a segment meet zero weights; they read real pixels.
 // Preferred form: TMA brings the tile's input patch [C][ih][iwp] to shared memory (4-D box whose x
 // origin is rounded down to a 16-byte boundary; out-of-range reads are zero = padding), one patch
-// per tile, prefetched through the halo ring; a row's K elements are then shared-memory reads.
+// per tile, prefetched through the halo ring.
 // thread = (row, part); it builds the chunks j = kParts*i + part so that all parts share the real elements.
-__device__ __forceinline__ void produce_stem_tile(const GemmSeg &sg, const GemmParams &g, int kb_local, const uint8_t *patch,
+// Small kernels (k <= 4) keep the K order (tap, channel) without padding inside K, K index e = (r * k + s) * C + c,
+// and gather element by element through a table of patch offsets.
+__device__ __forceinline__ void produce_stem_tile_elems(const GemmSeg &sg, const GemmParams &g, int kb_local, const uint8_t *patch,
                                                   const uint8_t *tab, int xrem, uint32_t a_base, int row, int part,
                                                   const RowLocal &rl, int jlimit) {
     // tab[e] = offset of K index e (tap-major, channel-minor) inside the patch, 0xFFFF for K padding;
@@ -382,9 +387,8 @@ __device__ __forceinline__ void produce_stem_tile(const GemmSeg &sg, const GemmP
     }
 }
 
-// Fallback when the image's row pitch is not a multiple of 16 bytes (TMA cannot address it): every
-// thread loads its row's elements straight from global memory.
-__device__ __forceinline__ void produce_stem_direct(const GemmSeg &sg, int kb_local, const RowPos &rp, uint32_t a_base,
+
+__device__ __forceinline__ void produce_stem_direct_elems(const GemmSeg &sg, int kb_local, const RowPos &rp, uint32_t a_base,
                                                     int row, int part) {
     const int ih0 = rp.p * sg.stride - sg.pad, iw0 = rp.q * sg.stride - sg.pad;
     const size_t img = (size_t)rp.n * sg.C * sg.H * sg.W;
@@ -409,6 +413,80 @@ __device__ __forceinline__ void produce_stem_direct(const GemmSeg &sg, int kb_lo
             }
             x.v[q] = v;
             if (++c == sg.C) { c = 0; if (++s == sg.k) { s = 0; ++r; } }
+        }
+        st_shared16(a_chunk_addr(a_base, row, j), pack8(x));
+    }
+}
+
+
+// Larger kernels (k = 5..8): segments of 8.
+__device__ __forceinline__ int stem_kp(int k) { return 8; }
+
+// n = 4 or 8 consecutive patch elements starting at element offset off, as bf16 pairs
+__device__ __forceinline__ void stem_copy(const uint8_t *patch, bool f32, uint32_t off, int n, uint32_t *out) {
+    if (f32) {
+        const float *pf = reinterpret_cast<const float *>(patch) + off;
+        for (int q = 0; q < n / 2; ++q) out[q] = pack2(pf[2 * q], pf[2 * q + 1]);
+    } else {
+        // 16-bit elements: read the covering 32-bit words and shift by the odd element
+        const uint32_t *pw = reinterpret_cast<const uint32_t *>(patch) + (off >> 1);
+        const uint32_t sh = (off & 1u) * 16u;
+        uint32_t w0 = pw[0];
+        for (int q = 0; q < n / 2; ++q) {
+            const uint32_t w1 = pw[q + 1];
+            out[q] = __funnelshift_r(w0, w1, sh);
+            w0 = w1;
+        }
+    }
+}
+
+__device__ __forceinline__ void produce_stem_tile(const GemmSeg &sg, const GemmParams &g, int kb_local, const uint8_t *patch,
+                                                  const uint8_t *tab, int xrem, uint32_t a_base, int row, int part,
+                                                  const RowLocal &rl, int jlimit) {
+    // tab[segment] = offset of the segment's first element for the tile's pixel (0, 0), ~0 for K padding;
+    // chunks >= jlimit are K padding that the caller has cleared already
+    const uint32_t base = rl.img == 0 ? (uint32_t)((rl.dy * sg.stride) * g.halo_w + xrem + rl.dx * sg.stride) : 0u;   // rows past the tile read pixel 0; never stored
+    const uint32_t *t32 = reinterpret_cast<const uint32_t *>(tab);
+    const bool f32 = sg.src_f32 != 0;
+#pragma unroll
+    for (int i = 0; i < kChunksPerThread; ++i) {
+        const int j = kParts * i + part;
+        if (j >= jlimit) break;
+        uint32_t w[4] = {0u, 0u, 0u, 0u};
+        const uint32_t o = t32[kb_local * 8 + j];
+        if (o != 0xFFFFFFFFu) stem_copy(patch, f32, base + o, 8, w);
+        st_shared16(a_chunk_addr(a_base, row, j), make_uint4(w[0], w[1], w[2], w[3]));
+    }
+}
+
+// Fallback when the image's row pitch is not a multiple of 16 bytes (TMA cannot address it): every
+// thread loads its row's elements straight from global memory.
+__device__ __forceinline__ void produce_stem_direct(const GemmSeg &sg, int kb_local, const RowPos &rp, uint32_t a_base,
+                                                    int row, int part) {
+    const int ih0 = rp.p * sg.stride - sg.pad, iw0 = rp.q * sg.stride - sg.pad;
+    const size_t img = (size_t)rp.n * sg.C * sg.H * sg.W;
+    const float *sf = reinterpret_cast<const float *>(sg.src) + img;
+    const unsigned short *sh = reinterpret_cast<const unsigned short *>(sg.src) + img;
+    const int kp = stem_kp(sg.k);
+#pragma unroll 1
+    for (int i = 0; i < kChunksPerThread; ++i) {
+        const int j = kParts * i + part;
+        const int e = kb_local * kTileK + j * 8;
+        int seg = e / kp, s = e - seg * kp;
+        int c = seg / sg.k, r = seg - c * sg.k;
+        f8 x;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            float v = 0.0f;
+            if (rp.valid && c < sg.C && s < sg.k) {
+                const int ih = ih0 + r, iw = iw0 + s;
+                if (ih >= 0 && ih < sg.H && iw >= 0 && iw < sg.W) {
+                    const int off = (c * sg.H + ih) * sg.W + iw;
+                    v = sg.src_f32 ? __ldg(sf + off) : __uint_as_float((unsigned)__ldg(sh + off) << 16);
+                }
+            }
+            x.v[q] = v;
+            if (++s == kp) { s = 0; if (++r == sg.k) { r = 0; ++c; } }
         }
         st_shared16(a_chunk_addr(a_base, row, j), pack8(x));
     }
@@ -571,12 +649,23 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
         for (int i = threadIdx.x - 64; i < C / 4; i += kProducerThreads) dst[9 * C / 4 + i] = __ldg(b4 + i);
     }
     if (g.stem_tma && threadIdx.x >= 64 && threadIdx.x < 64 + kProducerThreads) {
-        // K index -> offset inside the image patch [C][halo_h][halo_w]
-        unsigned short *tab = reinterpret_cast<unsigned short *>(sm + g.off_dww);
-        const int C = g.seg[0].C, k = g.seg[0].k, kreal = C * k * k;
-        for (int e = threadIdx.x - 64; e < g.kblocks * kTileK; e += kProducerThreads) {
-            const int tap = e / C, c = e - tap * C, r = tap / k, s2 = tap - r * k;
-            tab[e] = e < kreal ? (unsigned short)(c * g.halo_h * g.halo_w + r * g.halo_w + s2) : (unsigned short)0xFFFFu;
+        const int C = g.seg[0].C, k = g.seg[0].k;
+        if (k > 4) {
+            // K segment (channel, tap row) -> offset of its first element inside the image patch [C][halo_h][halo_w]
+            uint32_t *tab = reinterpret_cast<uint32_t *>(sm + g.off_dww);
+            const int nseg = g.kblocks * kTileK / stem_kp(k);
+            for (int sgm = threadIdx.x - 64; sgm < nseg; sgm += kProducerThreads) {
+                const int c = sgm / k, r = sgm - c * k;
+                tab[sgm] = c < C ? (uint32_t)(c * g.halo_h * g.halo_w + r * g.halo_w) : 0xFFFFFFFFu;
+            }
+        } else {
+            // K index -> offset inside the image patch
+            unsigned short *tab = reinterpret_cast<unsigned short *>(sm + g.off_dww);
+            const int kreal = C * k * k;
+            for (int e = threadIdx.x - 64; e < g.kblocks * kTileK; e += kProducerThreads) {
+                const int tap = e / C, c = e - tap * C, r = tap / k, s2 = tap - r * k;
+                tab[e] = e < kreal ? (unsigned short)(c * g.halo_h * g.halo_w + r * g.halo_w + s2) : (unsigned short)0xFFFFu;
+            }
         }
     }
     tc_fence_before();
@@ -696,7 +785,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
             // with a single K block its padding chunks never change: cleared once, then skipped
             int jlimit = 8;
             if (g.kblocks == 1) {
-                jlimit = (sg.C * sg.k * sg.k + 7) >> 3;
+                jlimit = (sg.C * sg.k * (sg.k > 4 ? stem_kp(sg.k) : sg.k) + 7) >> 3;
                 const int nz = 8 - jlimit;
                 for (int idx = pt; idx < g.stages * kTileM * nz; idx += kProducerThreads) {
                     const int sr = idx / nz, jj = jlimit + idx - sr * nz, s = sr / kTileM, row = sr - s * kTileM;
@@ -715,7 +804,8 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                     ok = mbar_wait_warp(empty_bar(s), st.ph ^ 1u, lane);
                     if (!ok) break;
                     st.next(g.stages);
-                    produce_stem_tile(sg, g, kb, sm + g.off_halo + shs * g.halo_stride, sm + g.off_dww, xrem, sbase + s * stage_bytes, grow, gpart, rl, jlimit);
+                    if (sg.k > 4) produce_stem_tile(sg, g, kb, sm + g.off_halo + shs * g.halo_stride, sm + g.off_dww, xrem, sbase + s * stage_bytes, grow, gpart, rl, jlimit);
+                    else produce_stem_tile_elems(sg, g, kb, sm + g.off_halo + shs * g.halo_stride, sm + g.off_dww, xrem, sbase + s * stage_bytes, grow, gpart, rl, jlimit);
                     fence_proxy_async();
                     warp_arrive(full_bar(s), lane);
                 }
@@ -790,7 +880,8 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                     // thread itself moves on to the next stage at once
                     asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(full_bar(s)) : "memory");
                 } else {
-                    produce_stem_direct(sg, kbl, rp, a_base, grow, gpart);
+                    if (sg.k > 4) produce_stem_direct(sg, kbl, rp, a_base, grow, gpart);
+                    else produce_stem_direct_elems(sg, kbl, rp, a_base, grow, gpart);
                     fence_proxy_async();
                     warp_arrive(full_bar(s), lane);
                 }

@@ -574,8 +574,12 @@ struct Lower {
             s0.dw_b_off = put_f32(dw->b);
         } else if (src.input_slot >= 0 && src.io_layout == XENOS_LAYOUT_NCHW) {
             if (expand2) return fail(g, XENOS_E_UNSUPPORTED, "internal: expand on an NCHW input");
+            // K order of a stem with k > 4: (channel, tap row) segments of 8 elements, the taps of one window row,
+            // which are adjacent in the image: a producer thread copies a segment instead of gathering elements.
+            // Small kernels keep (tap, channel) order without padding inside K.
+            if (M.k > 8) return fail(g, XENOS_E_UNSUPPORTED, "a convolution on an NCHW image supports kernels up to 8 x 8");
             s0.mode = AM_STEM; s0.k = M.k; s0.stride = M.stride; s0.pad = M.pad;
-            s0.kelems = M.k * M.k * src.c; s0.src_dtype = src.io_dtype;
+            s0.kelems = M.k > 4 ? src.c * M.k * 8 : M.k * M.k * src.c; s0.src_dtype = src.io_dtype;
         } else {
             if (src.c % 8) return fail(g, XENOS_E_UNSUPPORTED, "bf16 NHWC tensors need a channel count that is a multiple of 8");
             s0.mode = AM_GATHER; s0.k = kk; s0.stride = M.stride; s0.pad = expand2 ? kpadg : M.pad;
@@ -643,10 +647,11 @@ struct Lower {
             L.stem_align = 16 / es;
             L.stem_tma = (src.w * es) % 16 == 0 ? 1 : 0;
             L.halo_h = (L.patch_rh - 1) * M.stride + M.k;
-            L.halo_w = round_up((L.patch_rw - 1) * M.stride + M.k + L.stem_align - 1, L.stem_align);
+            // (a segment is read whole, kp elements plus up to two for the alignment of 16-bit images)
+            L.halo_w = round_up((L.patch_rw - 1) * M.stride + (M.k > 4 ? 8 + 2 : M.k) + L.stem_align - 1, L.stem_align);
             L.halo_cb = src.c;
-            // (patch offsets are kept as 16-bit table entries)
-            if (L.halo_h > 256 || L.halo_w > 256 || src.c > 256 || (long)src.c * L.halo_h * L.halo_w >= 65535) L.stem_tma = 0;
+            // (small kernels keep patch offsets as 16-bit table entries)
+            if (L.halo_h > 256 || L.halo_w > 256 || src.c > 256 || (M.k <= 4 && (long)src.c * L.halo_h * L.halo_w >= 65535)) L.stem_tma = 0;
             if (L.stem_tma) {
                 L.halo_bytes = src.c * L.halo_h * L.halo_w * es;
                 L.halo_stride = (int)align_up((size_t)L.halo_bytes, 128);
@@ -785,6 +790,16 @@ struct Lower {
             // concat order decides the row offsets; both read the same kk x kk window
             pack_conv(M, 0, 0, kk, src.c);
             pack_conv(*expand2, M.cout, 0, kk, src.c);
+        } else if (s0.mode == AM_STEM && M.k > 4) {
+            const int kp = 8;
+            for (int o = 0; o < M.cout; ++o) {
+                for (int c = 0; c < src.c; ++c)
+                    for (int r = 0; r < M.k; ++r)
+                        for (int sx = 0; sx < M.k; ++sx)
+                            wp[(size_t)o * L.kpad + (c * M.k + r) * kp + sx] =
+                                f32_to_bf16_rne(M.w[(((size_t)o * src.c + c) * M.k + r) * M.k + sx]);
+                bp[o] += M.b[o];
+            }
         } else {
             pack_conv(M, 0, 0, M.k, src.c);
         }
