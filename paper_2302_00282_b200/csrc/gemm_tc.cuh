@@ -513,6 +513,11 @@ __device__ __forceinline__ uint32_t clamp_bf16x2(uint32_t v, uint32_t lo, uint32
     return *reinterpret_cast<uint32_t *>(&x);
 }
 
+__device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b) {
+    __nv_bfloat162 x = __hmax2(*reinterpret_cast<__nv_bfloat162 *>(&a), *reinterpret_cast<__nv_bfloat162 *>(&b));
+    return *reinterpret_cast<uint32_t *>(&x);
+}
+
 template <int S, int BR>
 __device__ __forceinline__ void produce_dw(const GemmSeg &sg, const GemmParams &g, int kb_local, uint32_t halo, uint32_t dww,
                                            const DwUnit &u, uint32_t a_base) {
@@ -1083,19 +1088,18 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                     const int gy = ty * g.pth + oy, gx = tx * g.ptw + ox;
                     const int col = n0 + c8 * 8;
                     if (gy >= g.PP || gx >= g.PQ || col + 8 > g.N || n >= g.batch) continue;
-                    f8 m;
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) m.v[c] = -INFINITY;
+                    // the maximum of bf16 values is taken on the packed pairs (comparisons only: exact)
+                    uint4 m = make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);      // -inf
+                    const uint32_t win = stg + (uint32_t)((oy * g.pool_stride) * g.rw + ox * g.pool_stride) * pool_pitch + c8 * 16;
                     for (int dy = 0; dy < g.pool_k; ++dy)
                         for (int dx = 0; dx < g.pool_k; ++dx) {
-                            const int r = (oy * g.pool_stride + dy) * g.rw + ox * g.pool_stride + dx;
-                            const f8 xv = unpack8(ld_shared16(stg + r * pool_pitch + c8 * 16));
-#pragma unroll
-                            for (int c = 0; c < 8; ++c) m.v[c] = fmaxf(m.v[c], xv.v[c]);
+                            const uint4 xv = ld_shared16(win + (uint32_t)(dy * g.rw + dx) * pool_pitch);
+                            m.x = max_bf16x2(m.x, xv.x); m.y = max_bf16x2(m.y, xv.y);
+                            m.z = max_bf16x2(m.z, xv.z); m.w = max_bf16x2(m.w, xv.w);
                         }
                     __nv_bfloat16 *o2 = reinterpret_cast<__nv_bfloat16 *>(g.out) +
                                         (((size_t)n * g.PP + gy) * g.PQ + gx) * g.out_ctot + g.out_coff + col;
-                    *reinterpret_cast<uint4 *>(o2) = pack8(m);
+                    *reinterpret_cast<uint4 *>(o2) = m;
                 }
                 epi_bar();          // the staging tile is free for the next tile
             }
