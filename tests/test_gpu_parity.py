@@ -110,7 +110,10 @@ def test_bf16_conv1x1_equals_matmul():
     assert np.abs(y - ref).max() <= 2 ** -8 * np.abs(ref).max() + 1e-6
 
 
-@pytest.mark.parametrize("stem", [(3, 2, 1, 32, 33), (7, 2, 3, 64, 40), (3, 2, 0, 64, 31)])
+# (k, stride, pad, cout, hw): k <= 4 gathers by element, k = 5..8 copies (channel, tap row) segments; widths whose row
+# pitch is not a multiple of 16 bytes take the direct-load form of either
+@pytest.mark.parametrize("stem", [(3, 2, 1, 32, 33), (7, 2, 3, 64, 40), (3, 2, 0, 64, 31), (7, 2, 3, 64, 37), (5, 1, 2, 32, 24),
+                                  (8, 4, 2, 16, 32)])
 @pytest.mark.parametrize("in_mode", ["f32_nchw", "bf16_nchw"])
 def test_bf16_stem(stem, in_mode):
     k, st, pad, cout, hw = stem
@@ -192,6 +195,17 @@ def test_bf16_conv_gap_linked():
         g.gap("gap", x)
     spec = _one(build, 64, 7)
     _, _, gg = check_bf16("conv_gap", spec, 5, linked=True, in_mode="bf16_nhwc")
+    assert gg.g.launch_count() == 1
+
+
+@pytest.mark.parametrize("hw,batch", [(4, 9), (2, 40), (1, 7)])
+def test_bf16_conv_gap_many_images_per_tile(hw, batch):
+    """Small images: a 128-row tile holds several whole images and the average runs without partial sums."""
+    def build(g):
+        x = g.cbr("c", "input", 48, 3, 1, 1, act="relu")
+        g.gap("gap", x)
+    spec = _one(build, 16, hw)
+    _, _, gg = check_bf16(f"conv_gap_small{hw}", spec, batch, linked=True, in_mode="bf16_nhwc")
     assert gg.g.launch_count() == 1
 
 
