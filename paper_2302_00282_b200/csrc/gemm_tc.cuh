@@ -591,6 +591,43 @@ __device__ __forceinline__ void produce_dw(const GemmSeg &sg, const GemmParams &
     }
 }
 
+// The common store epilogue (bias, one activation as a clamp, bf16) for the 16-column chunks
+// [ch0, ch1) of one tile row, bias read from global memory.  The producer warps run it on the last
+// tile of their CTA, when they have nothing left to produce: three warps then share each quarter
+// of the accumulator's lanes.
+__device__ __forceinline__ void store_chunks(const GemmParams &g, uint32_t t_lane, const float *bias_tile, int n0, int ch0, int ch1,
+                                             const RowPos &rq, size_t pix, uint32_t plo, uint32_t phi, bool wide_ok) {
+    for (int cbase = ch0; cbase < ch1; cbase += 2) {
+        float vv[32];
+        const int nsub = (cbase + 1 < ch1) ? 2 : 1;
+        if (nsub == 2) tmem_ld32(t_lane + cbase * 16, vv); else tmem_ld16(t_lane + cbase * 16, vv);
+#pragma unroll
+        for (int sub = 0; sub < 2; ++sub) {
+            if (sub >= nsub) break;
+            const float *v = vv + 16 * sub;
+            const int ch = cbase + sub, nc = n0 + ch * 16;
+            uint32_t pk[8];
+#pragma unroll
+            for (int q4 = 0; q4 < 16; q4 += 4) {
+                const float4 bz = __ldg(reinterpret_cast<const float4 *>(bias_tile + ch * 16 + q4));
+                const float2 t0 = __fadd2_rn(make_float2(v[q4], v[q4 + 1]), make_float2(bz.x, bz.y));
+                const float2 t1 = __fadd2_rn(make_float2(v[q4 + 2], v[q4 + 3]), make_float2(bz.z, bz.w));
+                pk[q4 / 2] = clamp_bf16x2(pack2(t0.x, t0.y), plo, phi);
+                pk[q4 / 2 + 1] = clamp_bf16x2(pack2(t1.x, t1.y), plo, phi);
+            }
+            if (!rq.valid) continue;
+            __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(g.out) + pix * g.out_ctot + g.out_coff + nc;
+            if (nc + 16 <= g.N && wide_ok) {
+                asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(o), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]),
+                             "r"(pk[3]), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7]) : "memory");
+            } else {
+                if (nc + 8 <= g.N) *reinterpret_cast<uint4 *>(o) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                if (nc + 16 <= g.N) *reinterpret_cast<uint4 *>(o + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+            }
+        }
+    }
+}
+
 // ---- the kernel --------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmH, const GemmParams g) {
@@ -621,6 +658,9 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
     // depthwise: the producer threads are (pixel block, channel quad of the K block) pairs
     const int dw_quads = g.halo_cb > 32 ? 16 : 8;
     const int dw_br = g.halo_cb > 32 ? 2 : 1;       // block rows
+    // On a CTA's last tile the producer warps take two thirds of the columns of a plain store epilogue.
+    const bool help_last = g.epi == GE_STORE && !g.skip && !g.act2 && !g.out_f32 && g.tile_n >= 96;
+    const int help_per = (((g.tile_n / 16) + 2) / 3 + 1) & ~1;      // 16-column chunks per sharing warp, even
 
     if (threadIdx.x == 0) {
         // arrivals on a stage's "full" barrier: the TMA lane plus the producers of that stage (every
@@ -894,6 +934,30 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
         }
         if (!ok && lane == 0) atomicCAS(g.status, 0u, kStatusTimeout);
         cp_async_wait<0>();      // nothing of this thread is in flight when the CTA retires
+        if (help_last && ok) {
+            // this CTA's last tile: which one it is, which accumulator it sits in
+            TileWalk wl, last;
+            wl.init(g);
+            last = wl;
+            int cnt = 0;
+            for (; wl.ti < total_tiles; wl.next(g)) { last = wl; ++cnt; }
+            if (cnt > 0) {
+                const int b = (cnt - 1) & 1, quarter = warp & 3, row = quarter * 32 + lane, helper = (warp - 2) >> 2;
+                const RowLocal hl = row_local(g, row);
+                const RowPos rq = map_row(g, last, hl, row);
+                const size_t pix = ((size_t)rq.n * g.P + rq.p) * g.Q + rq.q;
+                const uint32_t plo = g.act >= 1 ? 0u : 0xff80ff80u, phi = g.act == 2 ? 0x40c040c0u : 0x7f807f80u;
+                const bool wide_ok = ((reinterpret_cast<uintptr_t>(g.out) | (uintptr_t)(g.out_ctot * 2) | (uintptr_t)(g.out_coff * 2)) & 31u) == 0;
+                if (mbar_wait_warp(accf_bar(b), ((cnt - 1) >> 1) & 1, lane)) {
+                    tc_fence_after();
+                    const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * g.acc_stride;
+                    const int nch = g.tile_n / 16;
+                    const int ch0 = min(nch, help_per * (1 + helper)), ch1 = min(nch, help_per * (2 + helper));
+                    store_chunks(g, t_lane, g.bias + last.nt * g.tile_n, last.nt * g.tile_n, ch0, ch1, rq, pix, plo, phi, wide_ok);
+                    tc_fence_before();
+                } else if (lane == 0) atomicCAS(g.status, 0u, kStatusTimeout);
+            }
+        }
     } else {
         // ---- epilogue: warp w reads tensor-memory lanes 32*(w%4).. ----
         const int quarter = warp & 3;
@@ -939,12 +1003,14 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
             }
             tc_fence_after();
             const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * g.acc_stride;
-            for (int cbase = 0; cbase < nchunks; cbase += 2) {
+            // (on the CTA's last tile the producer warps store the columns behind help_per)
+            const int nchunks_own = (help_last && w.ti + (int)gridDim.x >= total_tiles) ? min(nchunks, help_per) : nchunks;
+            for (int cbase = 0; cbase < nchunks_own; cbase += 2) {
                 // two 16-column chunks per tensor-memory load where the tile has them
                 float vv[32];
-                const int nsub = (cbase + 1 < nchunks) ? 2 : 1;
+                const int nsub = (cbase + 1 < nchunks_own) ? 2 : 1;
                 if (nsub == 2) tmem_ld32(t_lane + cbase * 16, vv); else tmem_ld16(t_lane + cbase * 16, vv);
-                if (cbase + nsub >= nchunks) {
+                if (cbase + nsub >= nchunks_own) {
                     // every column of this accumulator is in registers: hand it back to the MMA warp
                     tc_fence_before();
                     warp_arrive(acce_bar(b), lane);
