@@ -37,6 +37,20 @@ L2_FLUSH_BYTES = 256 << 20
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {("mobilenet_v1_b32", "linked", "gemm"): 217.24e6 / 15}
 
 
+def max_over_ranks(value: float, device: str) -> float:
+    """The slowest rank decides: replicas run independently, the job is as fast as its last replica."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_throughput(world: int, batch: int, steps: int, total_ms: float) -> float:
+    """Images per second of all replicas together: every rank processes `batch` images per step."""
+    return world * batch * steps / (total_ms * 1e-3)
+
+
 def measured_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -195,9 +209,7 @@ def main():
         g.status(stream)
         total_ms = sum(s.elapsed_time(e) for s, e in zip(starts, ends))
         if world > 1:
-            t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            total_ms = float(t.item())
+            total_ms = max_over_ranks(total_ms, "cuda")
             dist.barrier()
         torch.cuda.synchronize()
         return total_ms
@@ -238,9 +250,7 @@ def main():
         g.status(stream)
         total_ms = t0.elapsed_time(t1)
         if world > 1:
-            t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            total_ms = float(t.item())
+            total_ms = max_over_ranks(total_ms, "cuda")
             dist.barrier()
         torch.cuda.synchronize()
         return total_ms
@@ -250,7 +260,7 @@ def main():
     sampler.start()
     total_ms = time_steps(g_main, args.steps, args.warmup)
     clocks = sampler.stop()
-    value = world * batch * args.steps / (total_ms * 1e-3)
+    value = whole_job_throughput(world, batch, args.steps, total_ms)
     e2e_steps = max(8, args.steps // 2)
     e2e_ms = time_e2e(g_main, e2e_steps, 3)
     e2e_val = world * batch * e2e_steps / (e2e_ms * 1e-3)
