@@ -50,8 +50,8 @@ constexpr int kEpilogueThreads = 128;           // the last four warps
 constexpr int kThreads = 64 + kProducerThreads + kEpilogueThreads;
 constexpr unsigned kStatusTimeout = 0x80000000u | 9u;
 constexpr unsigned kStatusBounds = 0x80000000u | 10u;
-constexpr int kSpinLimit = 1 << 20;             // try_wait polls before a wait gives up (about a second)
-constexpr unsigned kSuspendHintNs = 1000;       // a waiting thread sleeps in hardware up to this long per poll,
+constexpr int kSpinLimit = 1 << 16;             // try_wait polls before a wait gives up (about a second)
+constexpr unsigned kSuspendHintNs = 16000;       // a waiting thread sleeps in hardware up to this long per poll,
                                                 // so pollers do not take issue slots from the working warps
 
 struct GemmSeg {

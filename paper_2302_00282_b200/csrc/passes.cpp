@@ -745,11 +745,11 @@ struct Lower {
         int dww_bytes = dw ? (int)align_up((size_t)40 * src.c, 128) : (L.stem_tma ? (int)align_up((size_t)L.kpad * 2, 128) : 0);
         int cap = std::min(g.hw.smem_bytes_per_cta, 227 * 1024) - 1024 - 256 - 2048 - dww_bytes;
         // a linked depthwise stage is bound by its own arithmetic, not by the MMA: give the halo ring
-        // (the TMA prefetch distance) up to four stages first, the A|B ring keeps at least two
+        // (the TMA prefetch distance) up to four stages first, the A|B ring keeps three when it can
         L.hstages = 0;
         if (dw || L.stem_tma) {
             L.hstages = 2;
-            while (L.hstages < 4 && cap - stg_bytes - (L.hstages + 1) * L.halo_stride >= 2 * stage_bytes) ++L.hstages;
+            while (L.hstages < 4 && cap - stg_bytes - (L.hstages + 1) * L.halo_stride >= 3 * stage_bytes) ++L.hstages;
         }
         int room = cap - stg_bytes - L.hstages * L.halo_stride;
         L.stages = std::min(6, room / stage_bytes);
