@@ -34,7 +34,7 @@ L2_FLUSH_BYTES = 256 << 20
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel (average over the launches of one
 # step), from the ncu capture summarised in profiles/<workload>_gemm_chain_dram.txt.  Only for the workload and
 # arm that capture covers; set back to None whenever the kernel changes after the capture.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {("mobilenet_v1_b32", "linked", "gemm"): 217.54e6 / 15}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {("mobilenet_v1_b32", "linked", "gemm"): 217.23e6 / 15}
 
 
 def max_over_ranks(value: float, device: str) -> float:
