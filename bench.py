@@ -23,6 +23,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 from xenos_workloads import graphs  # noqa: E402
+from xenos_workloads.feed import graph_from_spec  # noqa: E402
 
 WORKLOADS = {
     "mobilenet_v1_b32": (1, 32), "mobilenet_v1_b1": (1, 1),
@@ -165,7 +166,7 @@ def main():
     x = graphs.make_input(spec, batch)
 
     def make(linked):
-        g, ids = xb.graph_from_spec(spec, P, in_dtype=xb.DTYPE_F32 if fp32 else xb.DTYPE_BF16, in_layout=xb.LAYOUT_NCHW)
+        g, ids = graph_from_spec(spec, P, in_dtype=xb.DTYPE_F32 if fp32 else xb.DTYPE_BF16, in_layout=xb.LAYOUT_NCHW)
         if linked:
             g.link()
         nbytes = g.compile(batch, xb.PRECISION_FP32_CUDA_CORE if fp32 else xb.PRECISION_BF16_TENSOR)

@@ -2,8 +2,8 @@
  * xenos.h - C ABI of the linked-chain CNN inference library for NVIDIA B200 (sm_100a).
  *
  * The calls follow the paper's statement of the problem (Xenos, arXiv 2302.00282): the user
- * supplies "a computation graph for the inference model, along with the hardware-specific
- * information" (Section 6) built from the operators of Table 3; the library fuses
+ * hands over the model as a graph of Table 3 operators together with a description of the
+ * hardware (Section 6); the library fuses
  * Conv+Bn+Bias+Relu (Section 4.3), links adjacent operators so a producer hands its tile to
  * the consumer in the order the consumer reads it (Section 4.1, Table 1), splits operators
  * across the parallel units (Section 4.2, Eq. 1), and runs the optimised model, which is
@@ -84,8 +84,8 @@ enum { XENOS_LAYOUT_NCHW = 0, XENOS_LAYOUT_NHWC = 1 };
  *                  cores; tensors between kernels are NHWC bf16. */
 enum { XENOS_PRECISION_FP32_CUDA_CORE = 0, XENOS_PRECISION_BF16_TENSOR = 1 };
 
-/* "Hardware-specific information ... memory hierarchy, number of DSP units" (Section 6),
- * in this device's terms.  Pass NULL to xenos_graph_create for the B200 defaults
+/* The hardware description the optimiser needs - sizes of the memory levels and the number
+ * of parallel units (Section 6) - in this device's terms.  Pass NULL to xenos_graph_create for the B200 defaults
  * (148 SMs, 227 KB shared memory per block, 512 tensor-memory columns, 126 MB L2). */
 typedef struct {
     int32_t sm_count;             /* parallel units the split pass deals tiles to       */
@@ -169,8 +169,9 @@ XENOS_API xenos_status_t xenos_graph_bind(xenos_graph_t *g, void *workspace_dev,
                                           void *cuda_stream);
 
 /* Enqueue one inference of `batch` (<= max_batch) images on `cuda_stream`.
- * inputs_dev / outputs_dev: HOST arrays of DEVICE pointers in declaration order.
- * Asynchronous; does not synchronise.  Launch errors are returned, device-side status is
+ * inputs_dev / outputs_dev: HOST arrays of DEVICE pointers in declaration order; every
+ * pointer must be 16-byte aligned (XENOS_E_INVALID otherwise: the kernels use 16-byte
+ * vector accesses and TMA).  Asynchronous; does not synchronise.  Launch errors are returned, device-side status is
  * read with xenos_graph_status. */
 XENOS_API xenos_status_t xenos_graph_run(xenos_graph_t *g, int32_t batch,
                                          const void *const *inputs_dev, void *const *outputs_dev,
@@ -216,6 +217,14 @@ XENOS_API xenos_status_t xenos_graph_run_builtin_scratch(xenos_graph_t *g, int32
  * XENOS_E_TIMEOUT / XENOS_E_BOUNDS if a kernel gave up a bounded wait or failed an index
  * check since the last call (the word is then cleared). */
 XENOS_API xenos_status_t xenos_graph_status(xenos_graph_t *g, void *cuda_stream);
+
+/* Diagnostic.  Every device-side wait of the chain kernels is bounded; when one runs out the
+ * kernel records XENOS_E_TIMEOUT in the graph's status word and returns.  This call enqueues
+ * a one-thread kernel on `cuda_stream` that waits for four short polls on a barrier nothing
+ * signals and then reports exactly that way, so that the report path can be checked on a
+ * healthy device: the next xenos_graph_status returns XENOS_E_TIMEOUT once, later runs are
+ * unaffected.  Valid on a bound graph.  (No counterpart in the paper.) */
+XENOS_API xenos_status_t xenos_graph_selftest_wait_expiry(xenos_graph_t *g, void *cuda_stream);
 
 /* Write the compiled plan as JSON into `json` (capacity `cap`, always NUL-terminated when
  * cap > 0); *needed receives the length including the NUL.  Contents: fused operators,

@@ -9,7 +9,7 @@ from __future__ import annotations
 import ctypes
 import json
 import os
-from typing import Dict, List, Optional, Sequence
+from typing import List, Optional, Sequence
 
 import numpy as np
 
@@ -42,7 +42,7 @@ class OpDesc(ctypes.Structure):
 
 EXPORTS = ["xenos_graph_create", "xenos_graph_add_input", "xenos_graph_add_op", "xenos_graph_mark_output",
            "xenos_graph_link", "xenos_graph_split", "xenos_graph_compile", "xenos_graph_bind", "xenos_graph_run",
-           "xenos_graph_profile", "xenos_graph_run_builtin_scratch", "xenos_graph_status", "xenos_graph_get_plan", "xenos_graph_launch_count", "xenos_graph_destroy",
+           "xenos_graph_profile", "xenos_graph_run_builtin_scratch", "xenos_graph_status", "xenos_graph_selftest_wait_expiry", "xenos_graph_get_plan", "xenos_graph_launch_count", "xenos_graph_destroy",
            "xenos_last_error"]
 
 _lib = None
@@ -67,6 +67,7 @@ def lib() -> ctypes.CDLL:
         L.xenos_graph_profile.argtypes = [vp, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), vp, _f32p, i32]
         L.xenos_graph_run_builtin_scratch.argtypes = [vp, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), vp]
         L.xenos_graph_status.argtypes = [vp, vp]
+        L.xenos_graph_selftest_wait_expiry.argtypes = [vp, vp]
         L.xenos_graph_get_plan.argtypes = [vp, ctypes.c_char_p, sz, ctypes.POINTER(sz)]
         L.xenos_graph_launch_count.argtypes = [vp, ctypes.POINTER(i32)]
         L.xenos_graph_destroy.argtypes = [vp]
@@ -167,6 +168,9 @@ class Graph:
     def status(self, stream: int = 0):
         self._check(lib().xenos_graph_status(self._h, ctypes.c_void_p(stream)))
 
+    def selftest_wait_expiry(self, stream: int = 0):
+        self._check(lib().xenos_graph_selftest_wait_expiry(self._h, ctypes.c_void_p(stream)))
+
     def plan(self) -> dict:
         n = ctypes.c_size_t()
         self._check(lib().xenos_graph_get_plan(self._h, None, 0, ctypes.byref(n)))
@@ -196,36 +200,3 @@ class Graph:
             self.destroy()
         except Exception:
             pass
-
-
-_KIND = {"maxpool": OP_POOL_MAX, "avgpool": OP_POOL_AVG, "gap": OP_POOL_GLOBAL_AVG, "add": OP_ADD,
-         "concat": OP_CONCAT, "relu": OP_RELU, "relu6": OP_RELU6}
-
-
-def graph_from_spec(spec, params: Dict[str, Dict[str, np.ndarray]], in_dtype=DTYPE_F32, in_layout=LAYOUT_NCHW,
-                    hw: Optional[HwInfo] = None):
-    """Feeds the operator records of a workload graph to the C API, one add_op per record.
-    Returns (Graph, {tensor name: id})."""
-    g = Graph(hw)
-    ids = {"input": g.add_input(in_dtype, in_layout, *spec.in_shape)}
-    for o in spec.ops:
-        ins = [ids[n] for n in o["inputs"]]
-        p = params.get(o["name"], {})
-        k = o["kind"]
-        if k == "conv":
-            t = g.add_op(OP_CONV, ins, cout=o["cout"], k=o["k"], stride=o["stride"], pad=o["pad"], groups=o["groups"],
-                         weight=p["w"], bias=p.get("b"))
-        elif k == "fc":
-            t = g.add_op(OP_FC, ins, cout=o["cout"], k=1, weight=p["w"], bias=p.get("b"))
-        elif k == "bn":
-            t = g.add_op(OP_BATCHNORM, ins, bn=(p["gamma"], p["beta"], p["mean"], p["var"]), bn_eps=1e-5)
-        elif k in ("maxpool", "avgpool"):
-            t = g.add_op(_KIND[k], ins, k=o["k"], stride=o["stride"], pad=o["pad"])
-        else:
-            t = g.add_op(_KIND[k], ins)
-        ids[o["out"]] = t
-    fp32 = spec.precision == "fp32"
-    vec = len(spec.shapes[spec.output]) == 1
-    g.mark_output(ids[spec.output], DTYPE_F32 if (fp32 or vec) else DTYPE_BF16,
-                  LAYOUT_NCHW if (fp32 or vec) else LAYOUT_NHWC)
-    return g, ids

@@ -34,7 +34,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += [os.path.join(CSRC, s) for s in SOURCES]
-    cmd += ["-x", "cu"] if False else []
     subprocess.run(cmd, check=True, cwd=CSRC)
     return LIB
 

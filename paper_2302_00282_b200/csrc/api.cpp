@@ -38,6 +38,24 @@ static thread_local std::string g_create_err;
         return XENOS_E_INVALID;                                                       \
     }
 
+// Shared argument checks of the three run entry points.  Device buffers are read and written with
+// 16-byte vector accesses and by TMA, so every input and output pointer must be 16-byte aligned.
+static xenos_status_t check_run_args(const Graph &g, const char *who, int32_t batch, const void *const *inputs_dev,
+                                     void *const *outputs_dev) {
+    const std::string w(who);
+    if (batch < 1 || batch > g.max_batch) return fail(g, XENOS_E_INVALID, w + ": batch exceeds max_batch given to compile");
+    if (!inputs_dev || !outputs_dev) return fail(g, XENOS_E_INVALID, w + ": NULL pointer array");
+    for (size_t i = 0; i < g.inputs.size(); ++i) {
+        if (!inputs_dev[i]) return fail(g, XENOS_E_INVALID, w + ": NULL input pointer");
+        if ((uintptr_t)inputs_dev[i] & 15u) return fail(g, XENOS_E_INVALID, w + ": input pointer is not 16-byte aligned");
+    }
+    for (size_t i = 0; i < g.outputs.size(); ++i) {
+        if (!outputs_dev[i]) return fail(g, XENOS_E_INVALID, w + ": NULL output pointer");
+        if ((uintptr_t)outputs_dev[i] & 15u) return fail(g, XENOS_E_INVALID, w + ": output pointer is not 16-byte aligned");
+    }
+    return XENOS_OK;
+}
+
 extern "C" {
 
 xenos_status_t xenos_graph_create(const xenos_hw_info_t *hw, xenos_graph_t **out) {
@@ -222,12 +240,7 @@ xenos_status_t xenos_graph_run(xenos_graph_t *gp, int32_t batch, const void *con
     XENOS_GUARD_BEGIN
     Graph &g = gp->g;
     if (g.state != ST_BOUND) return fail(g, XENOS_E_STATE, "run before bind");
-    if (batch < 1 || batch > g.max_batch) return fail(g, XENOS_E_INVALID, "run: batch exceeds max_batch given to compile");
-    if (!inputs_dev || !outputs_dev) return fail(g, XENOS_E_INVALID, "run: NULL pointer array");
-    for (size_t i = 0; i < g.inputs.size(); ++i)
-        if (!inputs_dev[i]) return fail(g, XENOS_E_INVALID, "run: NULL input pointer");
-    for (size_t i = 0; i < g.outputs.size(); ++i)
-        if (!outputs_dev[i]) return fail(g, XENOS_E_INVALID, "run: NULL output pointer");
+    if (xenos_status_t st = check_run_args(g, "run", batch, inputs_dev, outputs_dev)) return st;
     return runtime_run(g, batch, inputs_dev, outputs_dev, cuda_stream);
     XENOS_GUARD_END(gp)
 }
@@ -239,13 +252,9 @@ xenos_status_t xenos_graph_profile(xenos_graph_t *gp, int32_t batch, const void 
     XENOS_GUARD_BEGIN
     Graph &g = gp->g;
     if (g.state != ST_BOUND) return fail(g, XENOS_E_STATE, "profile before bind");
-    if (batch < 1 || batch > g.max_batch) return fail(g, XENOS_E_INVALID, "profile: batch exceeds max_batch given to compile");
-    if (!inputs_dev || !outputs_dev || !ms_per_launch) return fail(g, XENOS_E_INVALID, "profile: NULL pointer");
+    if (xenos_status_t st = check_run_args(g, "profile", batch, inputs_dev, outputs_dev)) return st;
+    if (!ms_per_launch) return fail(g, XENOS_E_INVALID, "profile: NULL pointer");
     if (n_launches != (int32_t)g.launches.size()) return fail(g, XENOS_E_INVALID, "profile: n_launches must equal xenos_graph_launch_count");
-    for (size_t i = 0; i < g.inputs.size(); ++i)
-        if (!inputs_dev[i]) return fail(g, XENOS_E_INVALID, "profile: NULL input pointer");
-    for (size_t i = 0; i < g.outputs.size(); ++i)
-        if (!outputs_dev[i]) return fail(g, XENOS_E_INVALID, "profile: NULL output pointer");
     return runtime_run(g, batch, inputs_dev, outputs_dev, cuda_stream, ms_per_launch);
     XENOS_GUARD_END(gp)
 }
@@ -256,6 +265,15 @@ xenos_status_t xenos_graph_status(xenos_graph_t *gp, void *cuda_stream) {
     Graph &g = gp->g;
     if (g.state != ST_BOUND) return fail(g, XENOS_E_STATE, "status before bind");
     return runtime_status(g, cuda_stream);
+    XENOS_GUARD_END(gp)
+}
+
+xenos_status_t xenos_graph_selftest_wait_expiry(xenos_graph_t *gp, void *cuda_stream) {
+    if (!gp) return XENOS_E_INVALID;
+    XENOS_GUARD_BEGIN
+    Graph &g = gp->g;
+    if (g.state != ST_BOUND) return fail(g, XENOS_E_STATE, "selftest before bind");
+    return runtime_selftest_wait_expiry(g, cuda_stream);
     XENOS_GUARD_END(gp)
 }
 
@@ -288,13 +306,7 @@ xenos_status_t xenos_graph_run_builtin_scratch(xenos_graph_t *gp, int32_t batch,
     XENOS_GUARD_BEGIN
     Graph &g = gp->g;
     if (g.state < ST_COMPILED) return fail(g, XENOS_E_STATE, "run_builtin_scratch before compile");
-    if (batch < 1 || batch > g.max_batch)
-        return fail(g, XENOS_E_INVALID, "run_builtin_scratch: batch exceeds max_batch given to compile");
-    if (!inputs_dev || !outputs_dev) return fail(g, XENOS_E_INVALID, "run_builtin_scratch: NULL pointer array");
-    for (size_t i = 0; i < g.inputs.size(); ++i)
-        if (!inputs_dev[i]) return fail(g, XENOS_E_INVALID, "run_builtin_scratch: NULL input pointer");
-    for (size_t i = 0; i < g.outputs.size(); ++i)
-        if (!outputs_dev[i]) return fail(g, XENOS_E_INVALID, "run_builtin_scratch: NULL output pointer");
+    if (xenos_status_t st = check_run_args(g, "run_builtin_scratch", batch, inputs_dev, outputs_dev)) return st;
     if (g.workspace_bytes > runtime_builtin_scratch_bytes())
         return fail(g, XENOS_E_WORKSPACE,
                     "run_builtin_scratch: this graph needs " + std::to_string(g.workspace_bytes) +

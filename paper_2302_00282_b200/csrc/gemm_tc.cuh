@@ -93,8 +93,9 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// Bounded wait for the phase with the given parity.  Returns false when it gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+// Bounded wait for the phase with the given parity: one plain test, then at most `limit` polls that each
+// sleep in hardware up to `hint_ns`.  Returns false when it gave up.
+__device__ __forceinline__ bool mbar_wait_limited(uint32_t bar, uint32_t parity, int limit, uint32_t hint_ns) {
     {
         // most waits find their phase complete: a plain test is cheaper than a suspending wait
         uint32_t done;
@@ -105,16 +106,19 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
             : "=r"(done) : "r"(bar), "r"(parity) : "memory");
         if (done) return true;
     }
-    for (int i = 0; i < kSpinLimit; ++i) {
+    for (int i = 0; i < limit; ++i) {
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
             "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
             "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done) : "r"(bar), "r"(parity), "r"(kSuspendHintNs) : "memory");
+            : "=r"(done) : "r"(bar), "r"(parity), "r"(hint_ns) : "memory");
         if (done) return true;
     }
     return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    return mbar_wait_limited(bar, parity, kSpinLimit, kSuspendHintNs);
 }
 // One lane polls, the warp follows: keeps 32x fewer pollers on the barrier word.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, int lane) {
@@ -638,6 +642,19 @@ __device__ __forceinline__ void store_chunks(const GemmParams &g, uint32_t t_lan
     }
 }
 
+// Self-test of the give-up path every role uses: one thread waits, for a few short polls only, on a
+// barrier that nothing ever signals, records the expiry in the status word exactly as the roles of the
+// chain kernel do, and returns normally.
+__global__ void wait_expiry_probe_kernel(unsigned int *status, int polls) {
+    __shared__ __align__(8) unsigned long long bar;
+    if (threadIdx.x == 0) {
+        const uint32_t b = smem_u32(&bar);
+        mbar_init(b, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (!mbar_wait_limited(b, 0u, polls, 1000u)) atomicCAS(status, 0u, kStatusTimeout);
+    }
+}
+
 // ---- the kernel --------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmH, const GemmParams g) {
@@ -1002,15 +1019,12 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
             const RowPos rq = map_row(g, w, rl, row);
             const int n0 = nt * g.tile_n;
             const size_t pix = ((size_t)rq.n * g.P + rq.p) * g.Q + rq.q;
-            if (g.epi == GE_STORE && !new_bias) {
-                // plain stores share nothing between the warps: each waits for the accumulator by itself
-                if (!mbar_wait_warp(accf_bar(b), (i >> 1) & 1, lane)) { ok = false; break; }
-            } else {
-                // the four epilogue warps share named barriers below, so they must agree on giving up
-                if (!mbar_wait_warp(accf_bar(b), (i >> 1) & 1, lane) && lane == 0) *fail_flag = 1;
-                epi_bar();
-                if (*fail_flag) { ok = false; break; }
-            }
+            // The four epilogue warps share named barriers (bias slice, pool and average staging), so they
+            // agree on giving up before any of them can reach one: a warp whose wait ran out raises the
+            // flag, all four meet, and all four leave together.
+            if (!mbar_wait_warp(accf_bar(b), (i >> 1) & 1, lane) && lane == 0) *fail_flag = 1;
+            epi_bar();
+            if (*fail_flag) { ok = false; break; }
             tc_fence_after();
             const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * g.acc_stride;
             // (on the CTA's last tile the producer warps store the columns behind help_per)

@@ -202,6 +202,7 @@ xenos_status_t runtime_bind(Graph &g, void *ws, size_t bytes, void *stream);
 xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *const *out, void *stream,
                            float *ms_per_launch = nullptr);
 xenos_status_t runtime_status(Graph &g, void *stream);
+xenos_status_t runtime_selftest_wait_expiry(Graph &g, void *stream);
 void runtime_free(Graph &g);
 xenos_status_t runtime_run_builtin(Graph &g, int batch, const void *const *in, void *const *out, void *stream);
 void runtime_free_builtin(Graph &g);

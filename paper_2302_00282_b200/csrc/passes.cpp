@@ -907,7 +907,7 @@ xenos_status_t split_and_lower(Graph &g) {
 
 // ------------------------------------------------------------------------------------------------
 // Workspace: parameters, status words, then an arena for the tensors that live between kernels,
-// placed first-fit by live interval (the paper's "middleware for memory management", Section 6).
+// placed first-fit by live interval (the memory-management part of the paper's runtime layer, Section 6).
 // ------------------------------------------------------------------------------------------------
 xenos_status_t plan_workspace(Graph &g) {
     int nt = (int)g.tensors.size();

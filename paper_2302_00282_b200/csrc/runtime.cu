@@ -8,6 +8,7 @@
 
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <string>
 #include <vector>
 
@@ -43,9 +44,11 @@ static uint32_t make_idesc(int tile_n) {
 
 // 4-D map (C, W, H, N) over the NHWC bf16 input of a linked depthwise stage; box = one halo tile.
 // Out-of-range coordinates read zeros, which is the convolution's zero padding.
-static xenos_status_t encode_halo_map(const Graph &g, Runtime *rt, const Launch &L, void *base, CUtensorMap *out) {
+// `images` is the extent of the outermost dimension: boxes that reach past it (the last image group of
+// an odd batch) read zeros there and never touch memory behind the buffer.
+static xenos_status_t encode_halo_map(const Graph &g, Runtime *rt, const Launch &L, void *base, int images, CUtensorMap *out) {
     const ASeg &a = L.seg[0];
-    cuuint64_t dims[4] = {(cuuint64_t)a.C, (cuuint64_t)a.W, (cuuint64_t)a.H, (cuuint64_t)g.max_batch};
+    cuuint64_t dims[4] = {(cuuint64_t)a.C, (cuuint64_t)a.W, (cuuint64_t)a.H, (cuuint64_t)images};
     cuuint64_t strides[3] = {(cuuint64_t)a.C * 2, (cuuint64_t)a.W * a.C * 2, (cuuint64_t)a.H * a.W * a.C * 2};
     cuuint32_t box[4] = {(cuuint32_t)L.halo_cb, (cuuint32_t)L.halo_w, (cuuint32_t)L.halo_h, (cuuint32_t)L.ni};
     cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
@@ -59,11 +62,11 @@ static xenos_status_t encode_halo_map(const Graph &g, Runtime *rt, const Launch 
 }
 
 // 4-D map (W, H, C, N) over a small-channel NCHW image; box = one tile's input patch, all channels.
-static xenos_status_t encode_stem_map(const Graph &g, Runtime *rt, const Launch &L, void *base, CUtensorMap *out) {
+static xenos_status_t encode_stem_map(const Graph &g, Runtime *rt, const Launch &L, void *base, int images, CUtensorMap *out) {
     const ASeg &a = L.seg[0];
     const bool f32 = a.src_dtype == XENOS_DTYPE_F32;
     const cuuint64_t es = f32 ? 4 : 2;
-    cuuint64_t dims[4] = {(cuuint64_t)a.W, (cuuint64_t)a.H, (cuuint64_t)a.C, (cuuint64_t)g.max_batch};
+    cuuint64_t dims[4] = {(cuuint64_t)a.W, (cuuint64_t)a.H, (cuuint64_t)a.C, (cuuint64_t)images};
     cuuint64_t strides[3] = {(cuuint64_t)a.W * es, (cuuint64_t)a.H * a.W * es, (cuuint64_t)a.C * a.H * a.W * es};
     cuuint32_t box[4] = {(cuuint32_t)L.halo_w, (cuuint32_t)L.halo_h, (cuuint32_t)a.C, 1u};
     cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
@@ -135,7 +138,7 @@ xenos_status_t runtime_bind(Graph &g, void *ws, size_t bytes, void *stream_v) {
                                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
             if (r != CUDA_SUCCESS) return fail(g, XENOS_E_CUDA, "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r));
             if (L.seg[0].mode == AM_DW && g.tensors[L.seg[0].tensor].input_slot < 0) {
-                xenos_status_t st = encode_halo_map(g, rt, L, static_cast<uint8_t *>(ws) + g.place[L.seg[0].tensor].off, &rt->hmaps[i]);
+                xenos_status_t st = encode_halo_map(g, rt, L, static_cast<uint8_t *>(ws) + g.place[L.seg[0].tensor].off, g.max_batch, &rt->hmaps[i]);
                 if (st != XENOS_OK) return st;
             }
         }
@@ -301,7 +304,7 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
                 // the image is a caller buffer: encode its patch map now
                 if (((uintptr_t)ptr(L.seg[0].tensor) & 15u) != 0) p.stem_tma = 0;      // unaligned image: direct loads
                 else {
-                    xenos_status_t st = encode_stem_map(g, rt, L, ptr(L.seg[0].tensor), &tmh_now);
+                    xenos_status_t st = encode_stem_map(g, rt, L, ptr(L.seg[0].tensor), N, &tmh_now);
                     if (st != XENOS_OK) return st;
                     tmh = &tmh_now;
                 }
@@ -309,7 +312,7 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
             if (L.seg[0].mode == AM_DW) {
                 const Tensor &hx = g.tensors[L.seg[0].tensor];
                 if (hx.input_slot >= 0) {
-                    xenos_status_t st = encode_halo_map(g, rt, L, ptr(L.seg[0].tensor), &tmh_now);
+                    xenos_status_t st = encode_halo_map(g, rt, L, ptr(L.seg[0].tensor), N, &tmh_now);
                     if (st != XENOS_OK) return st;
                     tmh = &tmh_now;
                 } else {
@@ -363,6 +366,15 @@ xenos_status_t runtime_status(Graph &g, void *stream_v) {
     return fail(g, code, code == XENOS_E_TIMEOUT ? "a kernel gave up a bounded wait" : "a kernel failed an index check");
 }
 
+xenos_status_t runtime_selftest_wait_expiry(Graph &g, void *stream_v) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    unsigned int *status = reinterpret_cast<unsigned int *>(static_cast<uint8_t *>(g.ws) + g.status_off);
+    xk::wait_expiry_probe_kernel<<<1, 32, 0, stream>>>(status, 4);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(g, "kernel launch", e);
+    return XENOS_OK;
+}
+
 // ------------------------------------------------------------------------------------------------
 // Built-in scratch: a workspace that lives inside the library image, for callers that must not
 // allocate device memory themselves.
@@ -374,10 +386,12 @@ static __device__ __align__(256) unsigned char g_builtin_scratch[kBuiltinScratch
 // the address is looked up once per device and cached here.
 static void *g_builtin_ptr[kMaxDevices] = {};
 static uint64_t g_builtin_owner[kMaxDevices] = {};    // serial of the graph whose parameters the array holds
+static std::mutex g_builtin_mutex;                    // guards the two host tables above (not the device array)
 
 size_t runtime_builtin_scratch_bytes() { return kBuiltinScratchBytes; }
 
 void runtime_free_builtin(Graph &g) {
+    std::lock_guard<std::mutex> lock(g_builtin_mutex);
     delete static_cast<Runtime *>(g.rt_builtin);
     g.rt_builtin = nullptr;
     for (int d = 0; d < kMaxDevices; ++d)
@@ -390,6 +404,7 @@ xenos_status_t runtime_run_builtin(Graph &g, int batch, const void *const *in, v
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return cuda_fail(g, "no CUDA device (this library has no CPU fallback)", e);
     if (dev < 0 || dev >= kMaxDevices) return fail(g, XENOS_E_CUDA, "run_builtin_scratch: device index out of range");
+    std::lock_guard<std::mutex> lock(g_builtin_mutex);
     if (!g_builtin_ptr[dev]) {
         void *p = nullptr;
         e = cudaGetSymbolAddress(&p, g_builtin_scratch);
@@ -399,14 +414,19 @@ xenos_status_t runtime_run_builtin(Graph &g, int batch, const void *const *in, v
     void *scratch = g_builtin_ptr[dev];
     // run with the graph temporarily bound to the built-in scratch; the caller's own binding
     // (xenos_graph_bind) is put back afterwards
-    void *save_ws = g.ws, *save_rt = g.rt;
+    // (put back on every way out of this function, an exception from the bind included)
+    struct Restore {
+        Graph &g; void *ws, *rt;
+        ~Restore() { g.rt_builtin = g.rt; g.ws = ws; g.rt = rt; }
+    } restore{g, g.ws, g.rt};
     g.rt = g.rt_builtin;
+    g.rt_builtin = nullptr;               // g.rt owns the built-in binding until Restore hands it back
     xenos_status_t st = XENOS_OK;
-    Runtime *rb = static_cast<Runtime *>(g.rt_builtin);
+    Runtime *rb = static_cast<Runtime *>(g.rt);
     if (!rb || rb->device != dev || g_builtin_owner[dev] != g.serial) {
         // the array holds nothing or another graph's data: upload parameters, clear status, encode maps
+        g_builtin_owner[dev] = 0;
         st = runtime_bind(g, scratch, kBuiltinScratchBytes, stream);
-        g.rt_builtin = g.rt;
         g_builtin_owner[dev] = st == XENOS_OK ? g.serial : 0;
     } else {
         g.ws = scratch;
@@ -416,8 +436,6 @@ xenos_status_t runtime_run_builtin(Graph &g, int batch, const void *const *in, v
     }
     if (st == XENOS_OK) st = runtime_run(g, batch, in, out, stream, nullptr);
     if (st == XENOS_OK) st = runtime_status(g, stream);
-    g.ws = save_ws;
-    g.rt = save_rt;
     return st;
 }
 

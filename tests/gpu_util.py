@@ -7,13 +7,14 @@ import os
 
 import numpy as np
 
-LOG = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "gpurun_out", "parity_log.jsonl")
-
-
 def log(rec: dict):
+    """Appends one record to the file named by XENOS_PARITY_LOG (no log when the variable is unset)."""
+    path = os.environ.get("XENOS_PARITY_LOG")
+    if not path:
+        return
     try:
-        os.makedirs(os.path.dirname(LOG), exist_ok=True)
-        with open(LOG, "a") as f:
+        os.makedirs(os.path.dirname(os.path.abspath(path)), exist_ok=True)
+        with open(path, "a") as f:
             f.write(json.dumps(rec) + "\n")
     except OSError:
         pass
@@ -30,11 +31,12 @@ class GpuGraph:
     def __init__(self, spec, params, max_batch, linked=True, in_mode="f32_nchw", splits=(), links=None):
         import torch
         from paper_2302_00282_b200 import binding as xb
+        from xenos_workloads.feed import graph_from_spec
         self.xb, self.torch, self.spec = xb, torch, spec
         dt, lay = {"f32_nchw": (xb.DTYPE_F32, xb.LAYOUT_NCHW), "bf16_nchw": (xb.DTYPE_BF16, xb.LAYOUT_NCHW),
                    "bf16_nhwc": (xb.DTYPE_BF16, xb.LAYOUT_NHWC)}[in_mode]
         self.in_mode = in_mode
-        self.g, self.ids = xb.graph_from_spec(spec, params, in_dtype=dt, in_layout=lay)
+        self.g, self.ids = graph_from_spec(spec, params, in_dtype=dt, in_layout=lay)
         if links is not None:
             for chain in links:
                 self.g.link([self.ids[n] for n in chain])

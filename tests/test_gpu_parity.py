@@ -251,6 +251,67 @@ def test_bf16_batch_smaller_than_max_batch():
     check_bf16("mbv1_batch3_of_8", spec, 3, linked=True, max_batch=8)
 
 
+def test_bf16_dw_first_odd_batch_at_the_end_of_the_callers_buffer():
+    """A depthwise chain that reads the caller's NHWC buffer, tiles that hold two images, an odd batch below
+    max_batch: the last image group's halo box reaches past the batch and must read zeros, not the memory
+    behind the caller's buffer (here a guard band of NaN that sits right after the input)."""
+    import torch
+    def build(g):
+        x = g.cbr("dw", "input", 64, 3, 1, 1, groups=64, act="relu6")
+        g.cbr("pw", x, 64, 1, act="relu6")
+    spec = _one(build, 64, 7)
+    P = graphs.make_params(spec)
+    batch, max_batch = 3, 160         # enough images that the planner keeps two per tile
+    x = xo.round_bf16(graphs.make_input(spec, batch))
+    gg = GpuGraph(spec, P, max_batch, linked=True, in_mode="bf16_nhwc")
+    L = gg.g.plan()["launches"][0]
+    assert L["a0"] == "dw" and L["ni"] >= 2
+    n_in = batch * 7 * 7 * 64
+    guard = 4 * 7 * 7 * 64
+    buf = torch.full((n_in + guard,), float("nan"), dtype=torch.bfloat16, device="cuda")
+    buf[:n_in] = torch.from_numpy(np.ascontiguousarray(x.transpose(0, 2, 3, 1))).to(torch.bfloat16).reshape(-1).cuda()
+    out = gg.alloc_out(batch)
+    gg.g.run(batch, [buf.data_ptr()], [out.data_ptr()], gg.stream)
+    gg.g.status(gg.stream)
+    y = np.ascontiguousarray(out.float().cpu().numpy().transpose(0, 3, 1, 2))
+    o = interp.run_graph(spec, P, x)
+    assert not np.isnan(y).any()
+    assert abs_err_scaled(y, o) <= BF16_TOL
+
+
+def test_misaligned_device_pointers_are_refused():
+    import torch
+    from paper_2302_00282_b200 import binding as xb
+    spec = _one(lambda g: g.cbr("c", "input", 32, 1), 32, 8)
+    P = graphs.make_params(spec)
+    gg = GpuGraph(spec, P, 2, linked=False, in_mode="bf16_nhwc")
+    xin = torch.zeros(2 * 8 * 8 * 32 + 8, dtype=torch.bfloat16, device="cuda")
+    out = gg.alloc_out(2)
+    for ins, outs in (([xin.data_ptr() + 2], [out.data_ptr()]), ([xin.data_ptr()], [out.data_ptr() + 8])):
+        with pytest.raises(xb.XenosError) as e:
+            gg.g.run(2, ins, outs, gg.stream)
+        assert e.value.code == xb.E_INVALID and "16-byte aligned" in str(e.value)
+    gg.g.run(2, [xin.data_ptr()], [out.data_ptr()], gg.stream)
+    gg.g.status(gg.stream)
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_device_stays_usable():
+    """The give-up path of the bounded waits, in the one form that cannot hang: a one-thread kernel waits four
+    short polls on a barrier nothing signals, records XENOS_E_TIMEOUT in the status word and returns."""
+    from paper_2302_00282_b200 import binding as xb
+    spec = graphs.mobilenet_v1(hw=32, width=0.25, classes=16)
+    P = graphs.make_params(spec)
+    x = graphs.make_input(spec, 2)
+    gg = GpuGraph(spec, P, 2, linked=True)
+    ref = gg.run(x)
+    gg.g.selftest_wait_expiry(gg.stream)
+    with pytest.raises(xb.XenosError) as e:
+        gg.g.status(gg.stream)
+    assert e.value.code == xb.E_TIMEOUT
+    gg.g.status(gg.stream)                       # the word was cleared by the read
+    assert np.array_equal(gg.run(x), ref)        # and the next run is a normal one
+
+
 # ---- bf16: whole graphs ---------------------------------------------------------------------------
 @pytest.mark.parametrize("linked", [True, False])
 @pytest.mark.parametrize("name,kw", [("mobilenet_v1", dict(hw=64, width=0.25, classes=24)),

@@ -11,6 +11,7 @@ import pytest
 
 from paper_2302_00282_b200 import binding as xb
 from xenos_workloads import graphs
+from xenos_workloads.feed import graph_from_spec
 from xenos_workloads.graphs import GraphSpec
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
@@ -19,7 +20,7 @@ GOLD = os.path.join(os.path.dirname(__file__), "golden", "link_patterns.txt")
 
 def compiled(spec, batch=2, linked=True, splits=(), links=None, hw=None):
     P = graphs.make_params(spec)
-    g, ids = xb.graph_from_spec(spec, P, hw=hw)
+    g, ids = graph_from_spec(spec, P, hw=hw)
     if links is not None:
         for ch in links:
             g.link([ids[n] for n in ch])
@@ -274,8 +275,6 @@ def test_gemm_split_prefers_output_channels_until_units_are_busy():
             assert L["smem_bytes"] <= 227 * 1024
             if L["a0"] == "dw":
                 assert L["ni"] * L["patch_rh"] * L["patch_rw"] <= 128 and L["hstages"] >= 2
-    g, ids = compiled(spec, 32, splits=[("pw7.relu6", dict(parts_outc=4))])
-    L = [l for l in g.plan()["launches"] if l["kind"] == "gemm" and l["K"] == 512][1]
     hw = xb.HwInfo(16, 227 * 1024, 512, 1 << 20)
     g2, _ = compiled(spec, 1, hw=hw)
     assert g2.plan()["hw"]["sm_count"] == 16

@@ -13,6 +13,7 @@ import pytest
 
 from oracle import interp
 from xenos_workloads import graphs
+from xenos_workloads.feed import graph_from_spec
 
 from paper_2302_00282_b200 import binding as xb
 
@@ -20,7 +21,7 @@ from paper_2302_00282_b200 import binding as xb
 def test_oversized_graph_is_refused_with_both_sizes():
     spec = graphs.mobilenet_v1()                 # batch 32 needs far more than 16 MiB
     P = graphs.make_params(spec)
-    g, _ = xb.graph_from_spec(spec, P)
+    g, _ = graph_from_spec(spec, P)
     g.link()
     need = g.compile(32, xb.PRECISION_BF16_TENSOR)
     assert need > (16 << 20)
@@ -28,6 +29,33 @@ def test_oversized_graph_is_refused_with_both_sizes():
         g.run_builtin_scratch(32, [256], [256])
     assert e.value.code == xb.E_WORKSPACE
     assert str(need) in str(e.value) and str(16 << 20) in str(e.value)
+
+
+@pytest.mark.gpu
+def test_builtin_scratch_on_an_unbound_graph_and_with_a_partial_batch():
+    """compile only, no bind: the entry point needs no caller workspace at all; and batch < max_batch."""
+    import torch
+    from gpu_util import GpuGraph, abs_err_scaled
+
+    spec = graphs.mobilenet_v1(hw=32, width=0.25, classes=16)
+    P = graphs.make_params(spec)
+    x = graphs.make_input(spec, 3)
+    g, _ = graph_from_spec(spec, P)
+    g.link()
+    assert g.compile(8, xb.PRECISION_BF16_TENSOR) <= (16 << 20)
+    stream = torch.cuda.current_stream().cuda_stream
+    xin = torch.from_numpy(x).cuda()
+    out = torch.full((3, 16), float("nan"), dtype=torch.float32, device="cuda")
+    for _ in range(2):
+        g.run_builtin_scratch(3, [xin.data_ptr()], [out.data_ptr()], stream)
+        y = out.cpu().numpy()
+        assert not np.isnan(y).any()
+        assert abs_err_scaled(y, interp.run_graph(spec, P, x)) <= 2e-2
+    ref = GpuGraph(spec, P, 8, linked=True).run(x)
+    assert np.array_equal(y, ref)
+    with pytest.raises(xb.XenosError) as e:
+        g.run(3, [xin.data_ptr()], [out.data_ptr()], stream)      # still unbound for the ordinary path
+    assert e.value.code == xb.E_STATE
 
 
 @pytest.mark.gpu
