@@ -32,10 +32,21 @@ WORKLOADS = {
     "resnet50_stress_b64": (4, 64), "single_chain_b1": (0, 1),
 }
 L2_FLUSH_BYTES = 256 << 20
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel (average over the launches of one
-# step), from the ncu capture summarised in profiles/<workload>_gemm_chain_dram.txt.  Only for the workload and
-# arm that capture covers; set back to None whenever the kernel changes after the capture.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {("mobilenet_v1_b32", "linked", "gemm"): 217.23e6 / 15}
+MIN_TIMED_SECONDS = 0.3      # the K timed steps are repeated until the timed region covers at least this long
+
+
+def ncu_traffic_table():
+    """Measured DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum, averaged over the launches of
+    one step) by (workload, arm, kernel), from the table kept beside the ncu summaries.  A row is removed there
+    whenever its kernel changes after the capture, and the bench then reports null."""
+    table = {}
+    path = os.path.join(ROOT, "profiles", "dram_traffic_table.txt")
+    if os.path.exists(path):
+        for line in open(path):
+            f = line.split()
+            if len(f) >= 4 and not line.startswith("#"):
+                table[(f[0], f[1], f[2])] = float(f[3])
+    return table
 
 
 def max_over_ranks(value: float, device: str) -> float:
@@ -259,8 +270,14 @@ def main():
     g_main, ws_main = make(not args.unlinked)
     sampler = ClockSampler(local)
     sampler.start()
-    total_ms = time_steps(g_main, args.steps, args.warmup)
+    # K timed steps per repeat; repeats until the timed region is long enough for the clock sampler and for a
+    # stable mean.  ms_per_step is the mean over all repeats, the median of the repeats is reported beside it.
+    rep_ms = [time_steps(g_main, args.steps, args.warmup)]
+    repeats = int(min(200, max(1, np.ceil(MIN_TIMED_SECONDS * 1e3 / max(rep_ms[0], 1e-3)))))
+    for _ in range(repeats - 1):
+        rep_ms.append(time_steps(g_main, args.steps, 0))
     clocks = sampler.stop()
+    total_ms = float(np.mean(rep_ms))
     value = whole_job_throughput(world, batch, args.steps, total_ms)
     e2e_steps = max(8, args.steps // 2)
     e2e_ms = time_e2e(g_main, e2e_steps, 3)
@@ -291,23 +308,40 @@ def main():
     dk = by_kind[dom]
     t_mem = dk["bytes"] / (peaks["hbm_gbs"] * 1e9)
     t_tc = dk["flops"] / (peaks["bf16_tflops"] * 1e12)
+    # In-stream duration of the dominant kernel's launches: the timed step minus the other kernels' share of it
+    # (shares from the serialised per-launch times; when the step runs one kernel only, as the linked tensor-core
+    # graphs do, this is the timed step itself).
+    all_ms = sum(d["ms"] for d in by_kind.values())
+    step_ms = total_ms / args.steps
+    dom_ms_in_stream = step_ms * dk["ms"] / all_ms
     if t_tc > t_mem and not fp32:
-        roof = dict(bound="tensor", achieved=dk["flops"] / (dk["ms"] * 1e-3) / 1e12, peak=peaks["bf16_tflops"], unit="TFLOP/s")
+        roof = dict(bound="tensor", achieved=dk["flops"] / (dom_ms_in_stream * 1e-3) / 1e12, peak=peaks["bf16_tflops"], unit="TFLOP/s")
+        serial = dk["flops"] / (dk["ms"] * 1e-3) / 1e12
     else:
-        roof = dict(bound="hbm", achieved=dk["bytes"] / (dk["ms"] * 1e-3) / 1e9, peak=peaks["hbm_gbs"], unit="GB/s")
-    traffic = NCU_TRAFFIC_BYTES_PER_LAUNCH.get((args.workload, "unlinked" if args.unlinked else "linked", dom))
+        roof = dict(bound="hbm", achieved=dk["bytes"] / (dom_ms_in_stream * 1e-3) / 1e9, peak=peaks["hbm_gbs"], unit="GB/s")
+        serial = dk["bytes"] / (dk["ms"] * 1e-3) / 1e9
+    traffic = ncu_traffic_table().get((args.workload, "unlinked" if args.unlinked else "linked", dom))
     roof.update(frac=roof["achieved"] / roof["peak"], traffic=traffic, kernel=dom, launches_per_step=dk["launches"],
-                avg_launch_us=1e3 * dk["ms"] / dk["launches"], peak_source=peaks["source"],
-                algorithmic_bytes_per_step=dk["bytes"], flops_per_step=dk["flops"])
+                avg_launch_us=1e3 * dom_ms_in_stream / dk["launches"], peak_source=peaks["source"],
+                algorithmic_bytes_per_launch=dk["bytes"] / dk["launches"],
+                algorithmic_bytes_per_step=dk["bytes"], flops_per_step=dk["flops"],
+                timing="launches in the stream of the timed step (CUDA events around each step)",
+                serialised=dict(achieved=serial, frac=serial / roof["peak"], avg_launch_us=1e3 * dk["ms"] / dk["launches"],
+                                note="each launch timed alone between its own events: no overlap of one launch's "
+                                     "set-up with its predecessor's drain; the per-chain list uses these times as shares"))
     chains = []
     for c in plan["chains"]:
         ms = float(sum(acc[i] for i in c["launches"]))
         tm, tt = c["bytes_linked"] / (peaks["hbm_gbs"] * 1e9), c["flops"] / (peaks["bf16_tflops"] * 1e12)
-        chains.append(dict(id=c["id"], kind=c["kind"], us=1e3 * ms, bound="tensor" if tt > tm else "hbm",
-                           frac=(max(tm, tt) * 1e3) / ms if ms > 0 else None))
+        # in-stream time of the chain = its share of the serialised times, applied to the timed step
+        us = 1e3 * step_ms * ms / all_ms if all_ms > 0 else 0.0
+        chains.append(dict(id=c["id"], kind=c["kind"], us=us, us_serialised=1e3 * ms, share=ms / all_ms if all_ms > 0 else None,
+                           bound="tensor" if tt > tm else "hbm", roofline_us=max(tm, tt) * 1e6,
+                           frac=(max(tm, tt) * 1e6) / us if us > 0 else None))
 
     line = dict(metric="images/sec per linked CNN graph", value=value, unit="images/s", n_gpus=world, steps=args.steps,
-                warmup=args.warmup, ms_per_step=total_ms / args.steps, higher_is_better=True, scaling="weak",
+                warmup=args.warmup, ms_per_step=total_ms / args.steps, ms_per_step_median=float(np.median(rep_ms)) / args.steps,
+                repeats=repeats, higher_is_better=True, scaling="weak",
                 vs_baseline=None, dtype="f32" if fp32 else "bf16", data="synthetic",
                 config=dict(workload=args.workload, graph=spec.name, global_batch=batch * world, input=list(spec.in_shape),
                             mode="unlinked" if args.unlinked else "linked", l2="flushed between timed steps (256 MiB write)",
@@ -316,7 +350,7 @@ def main():
                 e2e=dict(value=e2e_val, unit="images/s", h2d_bytes_per_step=x_pin.numel() * x_pin.element_size(),
                          d2h_bytes_per_step=out_pin.numel() * out_pin.element_size(), steps=e2e_steps,
                          loop="copy of step i+1 overlaps compute of step i (two device buffers); L2 flush inside the timed loop"),
-                gpu_launches=g_main.launch_count() * args.steps,
+                gpu_launches=g_main.launch_count() * args.steps * repeats,
                 roofline=roof,
                 linked_vs_unlinked=dict(other_mode="linked" if args.unlinked else "unlinked", other_value=other_val,
                                         speedup=(value / other_val) if not args.unlinked else (other_val / value),
