@@ -152,6 +152,8 @@ def main():
     ap.add_argument("--workload", default="mobilenet_v1_b32", choices=sorted(WORKLOADS))
     ap.add_argument("--ref-images", type=int, default=8, help="images per step of the CPU oracle arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_SECONDS,
+                    help="repeat the K timed steps until they cover this long (0: one pass, for profiler captures)")
     ap.add_argument("--unlinked", action="store_true", help="time the unlinked execution as the main arm")
     args = ap.parse_args()
     cfg, batch = WORKLOADS[args.workload]
@@ -273,7 +275,7 @@ def main():
     # K timed steps per repeat; repeats until the timed region is long enough for the clock sampler and for a
     # stable mean.  ms_per_step is the mean over all repeats, the median of the repeats is reported beside it.
     rep_ms = [time_steps(g_main, args.steps, args.warmup)]
-    repeats = int(min(200, max(1, np.ceil(MIN_TIMED_SECONDS * 1e3 / max(rep_ms[0], 1e-3)))))
+    repeats = int(min(200, max(1, np.ceil(args.min_seconds * 1e3 / max(rep_ms[0], 1e-3)))))
     for _ in range(repeats - 1):
         rep_ms.append(time_steps(g_main, args.steps, 0))
     clocks = sampler.stop()

@@ -148,12 +148,19 @@ XENOS_API xenos_status_t xenos_graph_mark_output(xenos_graph_t *g, xenos_id_t te
 XENOS_API xenos_status_t xenos_graph_link(xenos_graph_t *g, const xenos_id_t *ops, int32_t n_ops);
 
 /* Operator split (Section 4.2, Eq. 1).  op == -1: automatic for every chain (output
- * channels first, then rows / columns of the feature map; a reduction split is never
- * chosen).  Otherwise fix the split of the chain that produces tensor `op`:
+ * channels first, then rows / columns of the feature map; the reduction is cut only when
+ * the tiles would leave most units idle and the reduction is long: fc, late convolutions
+ * at small batch).  Otherwise fix the split of the chain that produces tensor `op`:
  * parts_outc x parts_h x parts_w pieces (0 = automatic for that dimension); parts_k > 1
- * requests a reduction (C/R/S) split and is XENOS_E_UNSUPPORTED in this version.
+ * requests the reduction (C / R / S) split of Section 4.2.2: the reduction index, in the
+ * kernel's (tap, channel) order and in blocks of 64 elements, is cut into parts_k chunks
+ * of equal size (the last may be shorter); each chunk's partial sums are fp32 and are
+ * added in ascending chunk order, so results do not vary from run to run, but they are not
+ * bit-equal to the unsplit plan.  parts_k applies to tensor-core convolutions and fc
+ * without a linked depthwise stage, image stem, linked shortcut convolution or pooling
+ * epilogue (XENOS_E_UNSUPPORTED otherwise, from compile).
  * XENOS_E_BAD_SPLIT (from this call or from compile) if a count exceeds the extent it
- * divides or breaks a kernel limit. */
+ * divides, leaves a chunk empty or breaks a kernel limit. */
 XENOS_API xenos_status_t xenos_graph_split(xenos_graph_t *g, xenos_id_t op, int32_t parts_outc,
                                            int32_t parts_h, int32_t parts_w, int32_t parts_k);
 

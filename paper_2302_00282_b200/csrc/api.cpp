@@ -189,10 +189,8 @@ xenos_status_t xenos_graph_split(xenos_graph_t *gp, xenos_id_t op, int32_t parts
         return fail(g, XENOS_E_INVALID, "split: id is not an operator output");
     if (parts_outc < 0 || parts_h < 0 || parts_w < 0 || parts_k < 0)
         return fail(g, XENOS_E_BAD_SPLIT, "split: negative part count");
-    if (parts_k > 1)
-        return fail(g, XENOS_E_UNSUPPORTED, "split: reduction (C/R/S) split is not implemented; only K, H, W");
     SplitRequest s;
-    s.outc = parts_outc; s.h = parts_h; s.w = parts_w; s.k = 1; s.user = true;
+    s.outc = parts_outc; s.h = parts_h; s.w = parts_w; s.k = parts_k > 1 ? parts_k : 1; s.user = true;
     g.split_requests.push_back({op, s});
     return XENOS_OK;
     XENOS_GUARD_END(gp)

@@ -79,6 +79,13 @@ struct GemmParams {
     int off_halo, off_stg, off_dww, off_bias, off_bar;   // shared-memory offsets from the 1024-aligned base
     int act, act2, epi, out_ctot, out_coff, out_f32, skip_ctot;
     uint32_t idesc;
+    // reduction split (Section 4.2.2, the C / R / S split that "requires additional reduction"): the K blocks are cut into
+    // ksplit chunks of kb_per blocks; n_tiles counts (channel tile, chunk) pairs, chunk fastest; partial sums go to
+    // split_part [chunk][output pixel][split_ld] as fp32 and the CTA that finishes a tile last adds them in chunk order
+    int ksplit, kb_per, split_ld;
+    long long split_stride;
+    float *split_part;
+    unsigned int *split_cnt;
 };
 
 // ---- PTX wrappers ------------------------------------------------------------------------------
@@ -275,6 +282,19 @@ struct TileWalk {
         }
     }
 };
+
+// (channel tile, K chunk) of a tile: n_tiles counts pairs when the reduction is split.
+struct TileK { int nt, kb0, kb1, ks; };
+template <int kSplit>
+__device__ __forceinline__ TileK tile_k(const GemmParams &g, int ntv) {
+    TileK t;
+    t.nt = ntv; t.ks = 0; t.kb0 = 0; t.kb1 = g.kblocks;
+    if (kSplit && g.ksplit > 1) {
+        t.nt = ntv / g.ksplit; t.ks = ntv - t.nt * g.ksplit;
+        t.kb0 = t.ks * g.kb_per; t.kb1 = min(g.kblocks, t.kb0 + g.kb_per);
+    }
+    return t;
+}
 
 // Position of tile row r inside a patch tile: fixed for a thread over the whole kernel.
 struct RowLocal { int img, dy, dx; };
@@ -642,6 +662,48 @@ __device__ __forceinline__ void store_chunks(const GemmParams &g, uint32_t t_lan
     }
 }
 
+// The general store epilogue for 16 columns of one tile row: bias, activation, identity-shortcut add, second
+// activation, then fp32 or bf16 values at the row's position (channel offset included).
+__device__ __forceinline__ void finish_store16(const GemmParams &g, float *v, uint32_t sbias, int ch, int nc, const RowPos &rq, size_t pix) {
+    const float lo1 = act_lo(g.act), hi1 = act_hi(g.act), lo2 = act_lo(g.act2), hi2 = act_hi(g.act2);
+#pragma unroll
+    for (int q4 = 0; q4 < 16; q4 += 4) {
+        const float4 bz = ld_shared_f4(sbias + (uint32_t)(ch * 16 + q4) * 4u);
+        v[q4] = fminf(fmaxf(v[q4] + bz.x, lo1), hi1); v[q4 + 1] = fminf(fmaxf(v[q4 + 1] + bz.y, lo1), hi1);
+        v[q4 + 2] = fminf(fmaxf(v[q4 + 2] + bz.z, lo1), hi1); v[q4 + 3] = fminf(fmaxf(v[q4 + 3] + bz.w, lo1), hi1);
+    }
+    if (!rq.valid) return;
+    // shortcut connection with an identity branch: the skip tile is read once, here
+    if (g.skip) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            if (nc + h * 8 + 8 > g.N) break;
+            const f8 sv = unpack8(__ldg(reinterpret_cast<const uint4 *>(g.skip + pix * g.skip_ctot + nc + h * 8)));
+#pragma unroll
+            for (int c = 0; c < 8; ++c) v[h * 8 + c] += sv.v[c];
+        }
+    }
+    if (g.act2) {
+#pragma unroll
+        for (int c = 0; c < 16; ++c) v[c] = fminf(fmaxf(v[c], lo2), hi2);
+    }
+    if (g.out_f32) {
+        float *o = reinterpret_cast<float *>(g.out) + pix * g.out_ctot + g.out_coff + nc;
+#pragma unroll
+        for (int c = 0; c < 16; ++c) if (nc + c < g.N) o[c] = v[c];
+    } else {
+        __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(g.out) + pix * g.out_ctot + g.out_coff + nc;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            if (nc + h * 8 + 8 > g.N) break;
+            f8 pv;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) pv.v[c] = v[h * 8 + c];
+            *reinterpret_cast<uint4 *>(o + h * 8) = pack8(pv);
+        }
+    }
+}
+
 // Self-test of the give-up path every role uses: one thread waits, for a few short polls only, on a
 // barrier that nothing ever signals, records the expiry in the status word exactly as the roles of the
 // chain kernel do, and returns normally.
@@ -656,6 +718,9 @@ __global__ void wait_expiry_probe_kernel(unsigned int *status, int polls) {
 }
 
 // ---- the kernel --------------------------------------------------------------------------------
+// kSplit = 1: the instance that also carries the reduction-split path (launches with ksplit > 1 use it; the
+// common instance is compiled without that code).
+template <int kSplit>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmH, const GemmParams g) {
     extern __shared__ uint8_t smem_raw[];
@@ -674,7 +739,11 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
     auto hfull_bar = [&](int s) { return bar_base + 8u * (2 * kMaxStages + 4 + s); };
     auto hempty_bar = [&](int s) { return bar_base + 8u * (2 * kMaxStages + 4 + kMaxHaloStages + s); };
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(sm + g.off_bar + 8 * (2 * kMaxStages + 4 + 2 * kMaxHaloStages));
-    volatile int *fail_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    volatile int *fail_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);      // [0] give-up flag, [1] "this CTA completes the split tile"
+    // Completion of the CTA's LAST tile, for the producer warps that help with its epilogue.  They take no part in
+    // the earlier tiles, so the phase parity of the accumulator barriers would tell them nothing: a parity wait
+    // cannot tell the wanted phase from the one two tiles before it.
+    const uint32_t lastf_bar = bar_base + 8u * (2 * kMaxStages + 4 + 2 * kMaxHaloStages) + 16u;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int total_tiles = g.m_tiles * g.n_tiles;
@@ -686,7 +755,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
     const int dw_quads = g.halo_cb > 32 ? 16 : 8;
     const int dw_br = g.halo_cb > 32 ? 2 : 1;       // block rows
     // On a CTA's last tile the producer warps take two thirds of the columns of a plain store epilogue.
-    const bool help_last = g.epi == GE_STORE && !g.skip && !g.act2 && !g.out_f32 && g.tile_n >= 96;
+    const bool help_last = g.epi == GE_STORE && !g.skip && !g.act2 && !g.out_f32 && g.tile_n >= 96 && g.ksplit <= 1;
     const int help_per = (((g.tile_n / 16) + 2) / 3 + 1) & ~1;      // 16-column chunks per sharing warp, even
 
     if (threadIdx.x == 0) {
@@ -697,6 +766,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
         for (int s = 0; s < g.stages; ++s) { mbar_init(full_bar(s), full_count); mbar_init(empty_bar(s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), kEpilogueThreads / 32); }
         for (int s = 0; s < g.hstages; ++s) { mbar_init(hfull_bar(s), 1); mbar_init(hempty_bar(s), prod_warps); }
+        mbar_init(lastf_bar, 1);
         *fail_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
@@ -768,7 +838,8 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                     tma_load_4d(sbase + g.off_halo + hr.s * g.halo_stride, &tmH, hx & ~(g.stem_align - 1), hy, 0, hn, hfull_bar(hr.s));
                     hr.next(g.hstages);
                 }
-                for (int kb = 0; kb < g.kblocks && ok; ++kb) {
+                const TileK tk = tile_k<kSplit>(g, w.nt);
+                for (int kb = tk.kb0; kb < tk.kb1 && ok; ++kb) {
                     if (dw_mode) {
                         ok = mbar_wait(hempty_bar(hr.s), hr.ph ^ 1u);
                         if (!ok) break;
@@ -779,7 +850,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                     ok = mbar_wait(empty_bar(st.s), st.ph ^ 1u);
                     if (!ok) break;
                     mbar_arrive_expect_tx(full_bar(st.s), (uint32_t)g.tile_n * 128u);
-                    tma_load_2d(sbase + st.s * stage_bytes + kABytes, &tmB, kb * kTileK, w.nt * g.tile_n, full_bar(st.s));
+                    tma_load_2d(sbase + st.s * stage_bytes + kABytes, &tmB, kb * kTileK, tk.nt * g.tile_n, full_bar(st.s));
                     st.next(g.stages);
                 }
             }
@@ -796,7 +867,8 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + b * g.acc_stride;
-                for (int kb = 0; kb < g.kblocks && ok; ++kb) {
+                const TileK tk = tile_k<kSplit>(g, kSplit ? ti % g.n_tiles : 0);
+                for (int kb = tk.kb0; kb < tk.kb1 && ok; ++kb) {
                     const int s = st.s;
                     ok = mbar_wait(full_bar(s), st.ph);
                     if (!ok) break;
@@ -809,10 +881,13 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
 #pragma unroll
                     for (int k4 = 0; k4 < kTileK / 16; ++k4)
                         umma_bf16(d_tmem, umma_desc_sw128(a + k4 * 32), umma_desc_sw128(bb + k4 * 32), g.idesc,
-                                  (kb > 0 || k4 > 0) ? 1u : 0u);
+                                  (kb > tk.kb0 || k4 > 0) ? 1u : 0u);
                     umma_commit(empty_bar(s));
                 }
-                if (ok) umma_commit(accf_bar(b));
+                if (ok) {
+                    umma_commit(accf_bar(b));
+                    if (ti + (int)gridDim.x >= total_tiles) umma_commit(lastf_bar);
+                }
             }
             if (!ok) atomicCAS(g.status, 0u, kStatusTimeout);
         }
@@ -922,6 +997,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
         for (; !g.stem_tma && !dw_mode && w.ti < total_tiles && ok; w.next(g)) {
             RowPos rp;
             rp.valid = 0; rp.n = 0; rp.p = 0; rp.q = 0;
+            const TileK tk = tile_k<kSplit>(g, w.nt);
             if (g.seg[0].mode == GA_STEM) rp = map_row(g, w, rl, grow);
             GatherRow gr0[4], gr1[4];
             GatherState gs0 = {0, 0, 0}, gs1 = {0, 0, 0};
@@ -932,10 +1008,10 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                     gr0[i] = gather_row(g.seg[0], r4);
                     gr1[i] = gather_row(g.seg[1], r4);       // (unused without a second segment)
                 }
-                if (gj) gather_advance(gs0, gj, g.seg[0].C >> 3, g.seg[0].k);
+                if (gj + 8 * tk.kb0) gather_advance(gs0, gj + 8 * tk.kb0, g.seg[0].C >> 3, g.seg[0].k);
                 if (g.seg[1].mode == GA_GATHER && gj) gather_advance(gs1, gj, g.seg[1].C >> 3, g.seg[1].k);
             }
-            for (int kb = 0; kb < g.kblocks && ok; ++kb) {
+            for (int kb = tk.kb0; kb < tk.kb1 && ok; ++kb) {
                 const int s = st.s;
                 const uint32_t sph = st.ph;
                 st.next(g.stages);
@@ -975,7 +1051,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                 const size_t pix = ((size_t)rq.n * g.P + rq.p) * g.Q + rq.q;
                 const uint32_t plo = g.act >= 1 ? 0u : 0xff80ff80u, phi = g.act == 2 ? 0x40c040c0u : 0x7f807f80u;
                 const bool wide_ok = ((reinterpret_cast<uintptr_t>(g.out) | (uintptr_t)(g.out_ctot * 2) | (uintptr_t)(g.out_coff * 2)) & 31u) == 0;
-                if (mbar_wait_warp(accf_bar(b), ((cnt - 1) >> 1) & 1, lane)) {
+                if (mbar_wait_warp(lastf_bar, 0u, lane)) {
                     tc_fence_after();
                     const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * g.acc_stride;
                     const int nch = g.tile_n / 16;
@@ -1005,7 +1081,8 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
         w.init(g);
         int i = 0, bias_nt = -1, bias_buf = 0;
         for (; w.ti < total_tiles; w.next(g), ++i) {
-            const int mt = w.mt, nt = w.nt;
+            const TileK tk = tile_k<kSplit>(g, w.nt);
+            const int mt = w.mt, nt = tk.nt;
             const int b = i & 1;
             // the bias slice of this channel tile goes to shared memory when the channel tile changes
             // (two buffers: a warp is at most one tile ahead of the others)
@@ -1027,6 +1104,52 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
             if (*fail_flag) { ok = false; break; }
             tc_fence_after();
             const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * g.acc_stride;
+            if (kSplit && g.ksplit > 1) {
+                // ---- reduction split: park this chunk's fp32 partial sums; the CTA that completes the tile adds
+                // the chunks in ascending order (a fixed order: results do not depend on which CTA came last)
+                float *part = g.split_part + (size_t)tk.ks * g.split_stride + pix * g.split_ld + n0;
+                for (int cbase = 0; cbase < nchunks; cbase += 2) {
+                    float vv[32];
+                    const int nsub = (cbase + 1 < nchunks) ? 2 : 1;
+                    if (nsub == 2) tmem_ld32(t_lane + cbase * 16, vv); else tmem_ld16(t_lane + cbase * 16, vv);
+                    if (cbase + nsub >= nchunks) {
+                        tc_fence_before();
+                        warp_arrive(acce_bar(b), lane);
+                    }
+                    if (rq.valid)
+#pragma unroll
+                        for (int q4 = 0; q4 < 32; q4 += 4)
+                            if (q4 < nsub * 16) __stcg(reinterpret_cast<float4 *>(part + cbase * 16 + q4), make_float4(vv[q4], vv[q4 + 1], vv[q4 + 2], vv[q4 + 3]));
+                }
+                __threadfence();
+                epi_bar();
+                if (et == 0) {
+                    unsigned int *cnt = g.split_cnt + (size_t)mt * (g.n_tiles / g.ksplit) + nt;
+                    const unsigned int old = atomicAdd(cnt, 1u);
+                    const int last = old == (unsigned int)(g.ksplit - 1);
+                    if (last) *cnt = 0u;                    // every chunk has arrived: ready for the next run
+                    fail_flag[1] = last;
+                }
+                epi_bar();
+                if (!fail_flag[1]) continue;
+                __threadfence();
+                for (int ch = 0; ch < nchunks; ++ch) {
+                    float v[16];
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) v[c] = 0.0f;
+                    if (rq.valid)
+                        for (int sp = 0; sp < g.ksplit; ++sp) {
+                            const float *ps = g.split_part + (size_t)sp * g.split_stride + pix * g.split_ld + n0 + ch * 16;
+#pragma unroll
+                            for (int q4 = 0; q4 < 16; q4 += 4) {
+                                const float4 x4 = __ldcg(reinterpret_cast<const float4 *>(ps + q4));
+                                v[q4] += x4.x; v[q4 + 1] += x4.y; v[q4 + 2] += x4.z; v[q4 + 3] += x4.w;
+                            }
+                        }
+                    finish_store16(g, v, sbias, ch, n0 + ch * 16, rq, pix);
+                }
+                continue;
+            }
             // (on the CTA's last tile the producer warps store the columns behind help_per)
             const int nchunks_own = (help_last && w.ti + (int)gridDim.x >= total_tiles) ? min(nchunks, help_per) : nchunks;
             for (int cbase = 0; cbase < nchunks_own; cbase += 2) {
@@ -1078,13 +1201,14 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                         }
                         continue;
                     }
+                    if (g.epi == GE_STORE) { finish_store16(g, v, sbias, ch, nc, rq, pix); continue; }
+                    // (pool and global-average tiles: bias, activation, [identity shortcut, activation], values kept)
 #pragma unroll
                     for (int q4 = 0; q4 < 16; q4 += 4) {
                         const float4 bz = ld_shared_f4(sbias + (uint32_t)(ch * 16 + q4) * 4u);
                         v[q4] = fminf(fmaxf(v[q4] + bz.x, lo1), hi1); v[q4 + 1] = fminf(fmaxf(v[q4 + 1] + bz.y, lo1), hi1);
                         v[q4 + 2] = fminf(fmaxf(v[q4 + 2] + bz.z, lo1), hi1); v[q4 + 3] = fminf(fmaxf(v[q4 + 3] + bz.w, lo1), hi1);
                     }
-                    // shortcut connection with an identity branch: the skip tile is read once, here
                     if (g.skip && rq.valid) {
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
@@ -1098,24 +1222,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
 #pragma unroll
                         for (int c = 0; c < 16; ++c) v[c] = fminf(fmaxf(v[c], lo2), hi2);
                     }
-                    if (g.epi == GE_STORE) {
-                        if (!rq.valid) continue;
-                        if (g.out_f32) {
-                            float *o = reinterpret_cast<float *>(g.out) + pix * g.out_ctot + g.out_coff + nc;
-#pragma unroll
-                            for (int c = 0; c < 16; ++c) if (nc + c < g.N) o[c] = v[c];
-                        } else {
-                            __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(g.out) + pix * g.out_ctot + g.out_coff + nc;
-#pragma unroll
-                            for (int h = 0; h < 2; ++h) {
-                                if (nc + h * 8 + 8 > g.N) break;
-                                f8 pv;
-#pragma unroll
-                                for (int c = 0; c < 8; ++c) pv.v[c] = v[h * 8 + c];
-                                *reinterpret_cast<uint4 *>(o + h * 8) = pack8(pv);
-                            }
-                        }
-                    } else if (g.epi == GE_POOL) {
+                    if (g.epi == GE_POOL) {
                         // rows outside the conv output never win a max
                         f8 lo, hi;
 #pragma unroll

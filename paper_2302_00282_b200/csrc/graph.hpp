@@ -128,6 +128,10 @@ struct Launch {
     int hstages = 0, halo_bytes = 0, halo_stride = 0, halo_cb = 0;   // depthwise halo ring (halo_h x halo_w input pixels per image)
     int stem_tma = 0, stem_align = 1;                              // stem: image patch by TMA, x alignment in elements
     int off_halo = 0, off_stg = 0, off_dww = 0, off_bias = 0, off_bar = 0;                    // shared-memory layout
+    // reduction split: ksplit chunks of kb_per K blocks; fp32 partial sums [chunk][pixel][npad] in the workspace's
+    // split scratch, one arrival counter per (row tile, channel tile)
+    int ksplit = 1, kb_per = 0;
+    size_t split_cnt_off = 0;
     // ---- fp32 linked chain (conv kxk -> conv1x1 -> pool)
     int Cmid = 0, K2 = 0, act2 = 0;
     int parts_outc = 1, tile_h = 0, tile_w = 0, tiles_h = 0, tiles_w = 0;   // tile of POOL outputs
@@ -176,6 +180,8 @@ struct Graph {
     std::vector<TensorPlace> place;
     std::vector<uint8_t> param_blob;      // packed parameters, uploaded to workspace offset 0
     size_t act_off = 0;                   // start of the activation arena
+    size_t cnt_bytes = 0;                 // arrival counters of reduction-split launches, right behind the status words
+    size_t split_off = 0, split_bytes = 0;   // fp32 partial sums of reduction-split launches (shared: launches run in turn)
     size_t status_off = 0;                // 64-byte device status area
     size_t workspace_bytes = 0;
     std::string plan_json;

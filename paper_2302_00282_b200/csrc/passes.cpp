@@ -459,7 +459,7 @@ struct Lower {
             L.flops = 2.0 * node_macs(n);
             L.bytes = tbytes(n.in[0]) + tbytes(n.out) + node_param_bytes(n);
             L.block = 256;
-            if (g.chains[ci].split.user && (g.chains[ci].split.outc > 1 || g.chains[ci].split.h > 1 || g.chains[ci].split.w > 1))
+            if (g.chains[ci].split.user && (g.chains[ci].split.outc > 1 || g.chains[ci].split.h > 1 || g.chains[ci].split.w > 1 || g.chains[ci].split.k > 1))
                 return fail(g, XENOS_E_BAD_SPLIT, "split: unlinked fp32 operators are split one output element per thread; no explicit split");
             push(L, ci);
             return XENOS_OK;
@@ -486,6 +486,8 @@ struct Lower {
         L.w_off = put_f32(A.w); L.b_off = put_f32(A.b);
         L.w2_off = put_f32(B.w); L.b2_off = put_f32(B.b);
         const SplitRequest &rq = ch.split;
+        if (rq.user && rq.k > 1)
+            return fail(g, XENOS_E_UNSUPPORTED, "split: the fp32 CUDA-core chain keeps every reduction inside one thread; parts_k applies to tensor-core convolutions and fc");
         const int smem_cap = std::min(g.hw.smem_bytes_per_cta, 227 * 1024) - 1024;
         auto region = [&](int t) { return (t - 1) * C.stride + C.k; };        // conv-output rows a tile of t pool rows reads
         auto smem_need = [&](int th, int tw) {
@@ -731,6 +733,28 @@ struct Lower {
             }
         }
         L.npad = L.n_tiles * L.tile_n;
+        // --- reduction split (Section 4.2.2: C, R, S after K; it needs an additional reduction).  The K blocks
+        // (64 elements of the (tap, channel) order) are cut into chunks of equal size, ascending; a chunk's partial
+        // sums are fp32 and the chunks are added in ascending order.  Chosen automatically only when the tiles
+        // leave most units idle and K is long (fc, late convolutions at small batch).
+        {
+            const bool can = s0.mode == AM_GATHER && s1.mode == AM_NONE && L.epi == EPI_STORE && L.map_mode == MAP_FLAT;
+            int want = 1;
+            if (rq.user && rq.k > 1) {
+                if (!can) return fail(g, XENOS_E_UNSUPPORTED, "split: parts_k applies to a plain convolution or fc (no linked depthwise stage, image stem, second K segment or pooling epilogue)");
+                if (rq.k > L.kblocks) return fail(g, XENOS_E_BAD_SPLIT, "split: parts_k exceeds the number of 64-element K blocks");
+                want = rq.k;
+            } else if (!rq.user && can && L.kblocks >= 4 && (long)L.m_tiles * L.n_tiles * 2 <= g.hw.sm_count) {
+                want = std::min(L.kblocks / 2, g.hw.sm_count / (L.m_tiles * L.n_tiles));
+            }
+            if (want > 1) {
+                L.kb_per = ceil_div(L.kblocks, want);
+                L.ksplit = ceil_div(L.kblocks, L.kb_per);
+                if (rq.user && rq.k > 1 && L.ksplit != want)
+                    return fail(g, XENOS_E_BAD_SPLIT, "split: parts_k does not cut the K blocks into that many non-empty chunks of equal size");
+                if (L.ksplit < 2) { L.ksplit = 1; L.kb_per = 0; }
+            }
+        }
         // two accumulators in tensor memory so the epilogue of one tile overlaps the MMAs of the next
         L.acc_stride = round_up(L.tile_n, 32);
         L.tmem_cols = 32;
@@ -761,7 +785,7 @@ struct Lower {
         L.off_bar = L.off_bias + 2048;
         L.pipe_bytes = L.off_bar;
         L.smem_bytes = L.off_bar + 256 + 1024;     // + barriers, alignment slack
-        L.grid = std::min(L.m_tiles * L.n_tiles, g.hw.sm_count);
+        L.grid = std::min(L.m_tiles * L.n_tiles * L.ksplit, g.hw.sm_count);
         L.block = 448;
         // --- pack weights + bias
         L.w_off = blob_reserve(g, (size_t)L.npad * L.kpad * 2);
@@ -821,7 +845,7 @@ struct Lower {
             if (n.cin % 8) return fail(g, XENOS_E_UNSUPPORTED, "fc input length must be a multiple of 8");
             return make_gemm(ci, {ni}, nullptr, &n, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, true);
         }
-        if (g.chains[ci].split.user && (g.chains[ci].split.outc > 1 || g.chains[ci].split.h > 1 || g.chains[ci].split.w > 1))
+        if (g.chains[ci].split.user && (g.chains[ci].split.outc > 1 || g.chains[ci].split.h > 1 || g.chains[ci].split.w > 1 || g.chains[ci].split.k > 1))
             return fail(g, XENOS_E_BAD_SPLIT, "split: element-wise, pooling and depthwise kernels are split one vector per thread; no explicit split");
         const Tensor &x = g.tensors[n.in[0]];
         if (!x.is_vec && x.c % 8) return fail(g, XENOS_E_UNSUPPORTED, "bf16 NHWC tensors need a channel count that is a multiple of 8");
@@ -929,6 +953,16 @@ xenos_status_t plan_workspace(Graph &g) {
     size_t off = align_up(g.param_blob.size(), 256);
     g.status_off = off;
     off += 256;
+    // arrival counters of the reduction-split launches sit behind the status words and are cleared with them
+    g.cnt_bytes = 0; g.split_bytes = 0;
+    for (Launch &L : g.launches)
+        if (L.kind == LK_GEMM && L.ksplit > 1) {
+            L.split_cnt_off = off + g.cnt_bytes;
+            g.cnt_bytes += align_up((size_t)L.m_tiles * L.n_tiles * 4, 16);
+            g.split_bytes = std::max(g.split_bytes, (size_t)L.ksplit * g.max_batch * L.rows_per_image * L.npad * 4);
+        }
+    g.cnt_bytes = align_up(g.cnt_bytes, 256);
+    off += g.cnt_bytes;
     g.act_off = off;
     struct Live { size_t off, bytes; int last; };
     std::vector<Live> live;
@@ -961,7 +995,8 @@ xenos_status_t plan_workspace(Graph &g) {
         live.push_back({cand, p.bytes, p.last});
         arena = std::max(arena, cand + p.bytes);
     }
-    g.workspace_bytes = g.act_off + arena;
+    g.split_off = align_up(g.act_off + arena, 256);
+    g.workspace_bytes = g.split_off + g.split_bytes;
     // a graph input that is also read late must outlive everything: external, nothing to do.
     return XENOS_OK;
 }
@@ -1045,6 +1080,7 @@ void emit_plan_json(Graph &g) {
             jint(s, "ni", L.ni); jint(s, "step_y", L.step_y); jint(s, "step_x", L.step_x); jint(s, "off_y", L.off_y); jint(s, "off_x", L.off_x);
             jint(s, "hstages", L.hstages); jint(s, "halo_h", L.halo_h); jint(s, "halo_w", L.halo_w); jint(s, "halo_cb", L.halo_cb);
             jint(s, "halo_bytes", L.halo_bytes);
+            jint(s, "ksplit", L.ksplit); jint(s, "kb_per", L.kb_per);
         }
         if (L.kind == LK_F32_CONV_CONV_POOL) {
             jint(s, "parts_outc", L.parts_outc); jint(s, "tile_h", L.tile_h); jint(s, "tile_w", L.tile_w);

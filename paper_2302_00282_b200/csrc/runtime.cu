@@ -102,7 +102,7 @@ xenos_status_t runtime_bind(Graph &g, void *ws, size_t bytes, void *stream_v) {
     if (!g.param_blob.empty())
         if ((e = cudaMemcpyAsync(ws, g.param_blob.data(), g.param_blob.size(), cudaMemcpyHostToDevice, stream)) != cudaSuccess)
             return cuda_fail(g, "parameter upload", e);
-    if ((e = cudaMemsetAsync(static_cast<uint8_t *>(ws) + g.status_off, 0, 256, stream)) != cudaSuccess)
+    if ((e = cudaMemsetAsync(static_cast<uint8_t *>(ws) + g.status_off, 0, 256 + g.cnt_bytes, stream)) != cudaSuccess)
         return cuda_fail(g, "status clear", e);
     if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return cuda_fail(g, "parameter upload sync", e);
     g.ws = ws;
@@ -149,7 +149,8 @@ xenos_status_t runtime_bind(Graph &g, void *ws, size_t bytes, void *stream_v) {
     if (max_gemm_smem > optin || max_chain_smem > optin)
         return fail(g, XENOS_E_CUDA, "a kernel of this plan needs more shared memory than the device offers");
     if (any_gemm)
-        if ((e = cudaFuncSetAttribute(xk::gemm_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin)) != cudaSuccess)
+        if ((e = cudaFuncSetAttribute(xk::gemm_chain_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, optin)) != cudaSuccess ||
+            (e = cudaFuncSetAttribute(xk::gemm_chain_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, optin)) != cudaSuccess)
             return cuda_fail(g, "cudaFuncSetAttribute(gemm)", e);
     if (max_chain_smem > 0)
         if ((e = cudaFuncSetAttribute(xk::f32_conv_conv_pool_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin)) != cudaSuccess)
@@ -284,7 +285,11 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
             p.step_y = L.step_y; p.step_x = L.step_x; p.off_y = L.off_y; p.off_x = L.off_x;
             p.pool_k = L.pool_k; p.pool_stride = L.pool_stride; p.PP = L.PP; p.PQ = L.PQ; p.pth = L.patch_th; p.ptw = L.patch_tw;
             p.gap_imgs = L.gap_imgs; p.gap_area = L.gap_area; p.gap_rpi = L.gap_rpi;
-            p.kblocks = L.kblocks; p.stages = L.stages; p.tile_n = L.tile_n; p.n_tiles = L.n_tiles; p.N = L.K;
+            p.kblocks = L.kblocks; p.stages = L.stages; p.tile_n = L.tile_n; p.n_tiles = L.n_tiles * L.ksplit; p.N = L.K;
+            p.ksplit = L.ksplit; p.kb_per = L.kb_per; p.split_ld = L.npad;
+            p.split_stride = (long long)N * L.rows_per_image * L.npad;
+            p.split_part = reinterpret_cast<float *>(ws + g.split_off);
+            p.split_cnt = reinterpret_cast<unsigned int *>(ws + L.split_cnt_off);
             p.acc_stride = L.acc_stride; p.tmem_cols = L.tmem_cols;
             p.hstages = L.hstages; p.halo_bytes = L.halo_bytes; p.halo_stride = L.halo_stride;
             p.halo_h = L.halo_h; p.halo_w = L.halo_w; p.halo_cb = L.halo_cb;
@@ -319,7 +324,7 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
                     tmh = &rt->hmaps[li];
                 }
             }
-            const int grid = std::min(p.m_tiles * L.n_tiles, sms);
+            const int grid = std::min(p.m_tiles * p.n_tiles, sms);
             // Programmatic dependent launch: the kernel may be scheduled while its predecessor in the
             // stream drains, runs its set-up (barriers, tensor memory, constant staging) and then
             // waits (griddepcontrol.wait) before it touches any activation.
@@ -330,7 +335,8 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
             at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
             at[0].val.programmaticStreamSerializationAllowed = 1;
             cfg.attrs = at; cfg.numAttrs = 1;
-            cudaError_t le = cudaLaunchKernelEx(&cfg, xk::gemm_chain_kernel, rt->tmaps[li], *tmh, p);
+            cudaError_t le = L.ksplit > 1 ? cudaLaunchKernelEx(&cfg, xk::gemm_chain_kernel<1>, rt->tmaps[li], *tmh, p)
+                                          : cudaLaunchKernelEx(&cfg, xk::gemm_chain_kernel<0>, rt->tmaps[li], *tmh, p);
             if (le != cudaSuccess) return cuda_fail(g, "kernel launch", le);
             break;
         }
@@ -361,7 +367,7 @@ xenos_status_t runtime_status(Graph &g, void *stream_v) {
     uint8_t *ws = static_cast<uint8_t *>(g.ws);
     if ((e = cudaMemcpy(&word, ws + g.status_off, 4, cudaMemcpyDeviceToHost)) != cudaSuccess) return cuda_fail(g, "status read", e);
     if (word == 0) return XENOS_OK;
-    cudaMemset(ws + g.status_off, 0, 4);
+    cudaMemset(ws + g.status_off, 0, 256 + g.cnt_bytes);      // (the arrival counters of a run that gave up are stale too)
     int code = -(int)(word & 0xffu);
     return fail(g, code, code == XENOS_E_TIMEOUT ? "a kernel gave up a bounded wait" : "a kernel failed an index check");
 }
@@ -431,7 +437,7 @@ xenos_status_t runtime_run_builtin(Graph &g, int batch, const void *const *in, v
     } else {
         g.ws = scratch;
         // the status word keeps the last call's contents: start from zero
-        if ((e = cudaMemsetAsync(static_cast<uint8_t *>(scratch) + g.status_off, 0, 256, stream)) != cudaSuccess)
+        if ((e = cudaMemsetAsync(static_cast<uint8_t *>(scratch) + g.status_off, 0, 256 + g.cnt_bytes, stream)) != cudaSuccess)
             st = cuda_fail(g, "status clear", e);
     }
     if (st == XENOS_OK) st = runtime_run(g, batch, in, out, stream, nullptr);

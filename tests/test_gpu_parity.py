@@ -22,13 +22,16 @@ FP32_TOL = 1e-4
 # elements by the order of that range.  The bound is 2^-7.
 LINKED_VS_UNLINKED_TOL = 2.0 ** -7
 # Against the oracle run with bf16 rounding of every stored tensor (same rounding points as the device, fp32
-# sums in another order): the drift of the un-rounded comparison is gone, what remains is the same one-step
-# effect as above.
+# sums in another order), on graphs a few operators deep: the drift of the un-rounded comparison is gone, what
+# remains is the same one-step effect as above.  (On the 53-convolution stress graph, and already on its first
+# stage, two bf16 evaluations differ from each other by as much as either differs from the un-rounded oracle,
+# measured 2.4e-2 / 1.7e-2 against 1.8e-2 / 1.5e-2, so the emulation separates drift from indexing errors only on
+# graphs a few operators deep.)
 EMULATED_TOL = 2.0 ** -7
 
 
 def check_bf16(name, spec, batch, linked=True, in_mode="f32_nchw", seed=gen.DEFAULT_SEED, max_batch=None,
-               splits=(), images=None, links=None, against_unlinked=False, emulated=False):
+               splits=(), images=None, links=None, against_unlinked=False, emulated=False, unlinked_tol=None):
     P = graphs.make_params(spec, seed)
     x = graphs.make_input(spec, batch, seed)
     if in_mode != "f32_nchw":
@@ -54,7 +57,7 @@ def check_bf16(name, spec, batch, linked=True, in_mode="f32_nchw", seed=gen.DEFA
         erru = abs_err_scaled(y, yu)
         log(dict(test=name + ":linked_vs_unlinked", err=erru, images=batch))
         assert not np.isnan(yu).any()
-        assert erru <= LINKED_VS_UNLINKED_TOL, f"{name}: linked vs unlinked, all {batch} images: {erru:.3e}"
+        assert erru <= (unlinked_tol or LINKED_VS_UNLINKED_TOL), f"{name}: linked vs unlinked, all {batch} images: {erru:.3e}"
         return y, o, gu
     return y, o, gg
 
@@ -122,6 +125,17 @@ def test_bf16_conv(case):
     cin, hw, cout, k, st, pad, batch = case
     spec = _one(lambda g: g.cbr("c", "input", cout, k, st, pad, act="relu"), cin, hw)
     check_bf16(f"conv{case}", spec, batch, linked=False, in_mode="bf16_nhwc")
+
+
+def test_bf16_pointwise_many_tiles_per_unit():
+    """A pointwise convolution with fourteen 128-row tiles per CTA, one K block each and a 256-wide channel tile:
+    the producer warps run several tiles ahead of the tensor core and join the store epilogue of their CTA's last
+    tile, which they must not mistake for an earlier one (every image is compared)."""
+    spec = _one(lambda g: g.cbr("c", "input", 256, 1, act=None), 64, 128)
+    y, o, gg = check_bf16("pointwise_many_tiles", spec, 16, linked=False, in_mode="bf16_nhwc")
+    x = xo.round_bf16(graphs.make_input(spec, 16))
+    for _ in range(3):
+        assert np.array_equal(gg.run(x), y)
 
 
 def test_bf16_conv1x1_equals_matmul():
@@ -250,6 +264,46 @@ def test_bf16_shortcut_block(proj):
     assert gg.g.launch_count() == 2      # c1, then {c2 [+proj] + add + relu}
 
 
+# ---- reduction split (Section 4.2.2: the C / R / S split with its additional reduction) ----------------
+@pytest.mark.parametrize("parts_k", [2, 3, 6])
+def test_bf16_conv_reduction_split(parts_k):
+    """K = 128 * 9 = 18 blocks cut into chunks; ragged M (243 rows) and N = 40; the chunks are added in a fixed
+    order, so two runs agree bit for bit, and the sum differs from the unsplit plan by fp32 rounding only."""
+    spec = _one(lambda g: g.cbr("c", "input", 40, 3, 1, 1, act="relu"), 128, 9)
+    y, o, gg = check_bf16(f"conv_splitk{parts_k}", spec, 3, linked=False, in_mode="bf16_nhwc", splits=[("c", dict(parts_k=parts_k))])
+    L = gg.g.plan()["launches"][0]
+    assert L["ksplit"] == parts_k and L["grid"] == L["m_tiles"] * L["n_tiles"] * parts_k
+    x = xo.round_bf16(graphs.make_input(spec, 3))
+    assert np.array_equal(gg.run(x), y)
+    base, _, _ = check_bf16("conv_splitk_base", spec, 3, linked=False, in_mode="bf16_nhwc")
+    assert abs_err_scaled(y, base) <= 2.0 ** -8
+
+
+def test_bf16_shortcut_block_with_reduction_split():
+    def build(g):
+        y = g.cbr("c1", "input", 64, 3, 1, 1)
+        y = g.cbr("c2", y, 64, 3, 1, 1, act=None)
+        y = g.add("add", y, "input")
+        g.act("relu", y, "relu")
+    spec = _one(build, 64, 10)
+    _, _, gg = check_bf16("shortcut_splitk", spec, 2, linked=True, in_mode="bf16_nhwc", splits=[("add", dict(parts_k=3))])
+    assert gg.g.plan()["launches"][1]["ksplit"] == 3
+
+
+def test_bf16_fc_reduction_split_is_automatic_and_repeatable():
+    """fc with few rows and a long reduction: the planner cuts K by itself (the other dimensions leave the units idle)."""
+    def build(g):
+        x = g.gap("gap", "input")
+        g.fc("fc", x, 1000)
+    spec = _one(build, 1024, 3)
+    y, _, gg = check_bf16("fc_splitk_auto", spec, 5, linked=False, in_mode="bf16_nhwc")
+    L = [l for l in gg.g.plan()["launches"] if l["kind"] == "gemm"][0]
+    assert L["ksplit"] >= 2
+    x = xo.round_bf16(graphs.make_input(spec, 5))
+    for _ in range(3):
+        assert np.array_equal(gg.run(x), y)
+
+
 @pytest.mark.parametrize("pool", [False, True])
 def test_bf16_fire_module(pool):
     def build(g):
@@ -370,4 +424,25 @@ def test_bf16_full_configs_batch32_sampled(cfg):
 def test_bf16_stress_graph_batch64_sampled():
     """Config 4 at full size; the oracle evaluates images 0 and 63 (images are independent)."""
     spec, _ = graphs.config(4)
-    check_bf16("cfg4_n64", spec, 64, linked=True, in_mode="bf16_nchw", images=[0, 63], against_unlinked=True, emulated=True)
+    # 53 convolutions without any normalisation between the blocks: outputs reach 6.5e4 and rounding differences grow
+    # from block to block, so two correct bf16 evaluations differ by about as much (1.9e-2 of the range, every image)
+    # as each differs from the oracle (1.5e-2 to 1.8e-2).  A tile written by the wrong CTA showed up here as 1.4e-1
+    # on the two images it touched.
+    check_bf16("cfg4_n64", spec, 64, linked=True, in_mode="bf16_nchw", images=[0, 63], against_unlinked=True, unlinked_tol=2.0 ** -5)
+
+
+@pytest.mark.parametrize("linked", [True, False])
+def test_bf16_stress_graph_block_at_full_size_against_the_rounding_oracle(linked):
+    """The first bottleneck of the stress graph in isolation, at its full 128 x 128 x 64 input (the chain-by-chain
+    form of the comparison: a few operators deep, so the oracle with bf16 rounding at every stored tensor tracks
+    the device to a rounding step and an indexing error in the full-size tiles cannot hide in the tolerance that the
+    53-convolution graph needs)."""
+    def build(g):
+        y = g.cbr("r", "input", 64, 1, 1, 0)
+        y = g.cbr("c3", y, 64, 3, 1, 1)
+        y = g.cbr("e", y, 256, 1, 1, 0, act=None)
+        skip = g.cbr("proj", "input", 256, 1, 1, 0, act=None)
+        y = g.add("add", y, skip)
+        g.act("relu", y, "relu")
+    spec = _one(build, 64, 128)
+    check_bf16("cfg4_block_n2", spec, 2, linked=linked, in_mode="bf16_nhwc", emulated=True)

@@ -18,9 +18,9 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 GOLD = os.path.join(os.path.dirname(__file__), "golden", "link_patterns.txt")
 
 
-def compiled(spec, batch=2, linked=True, splits=(), links=None, hw=None):
+def compiled(spec, batch=2, linked=True, splits=(), links=None, hw=None, nhwc=False):
     P = graphs.make_params(spec)
-    g, ids = graph_from_spec(spec, P, hw=hw)
+    g, ids = graph_from_spec(spec, P, hw=hw, in_dtype=xb.DTYPE_BF16 if nhwc else None, in_layout=xb.LAYOUT_NHWC if nhwc else None)
     if links is not None:
         for ch in links:
             g.link([ids[n] for n in ch])
@@ -75,8 +75,8 @@ def test_state_machine_and_argument_errors():
         g.link([z, y])                                       # not producer -> consumer
     assert e.value.code == xb.E_NOT_LINKABLE
     with pytest.raises(xb.XenosError) as e:
-        g.split(y, parts_k=2)
-    assert e.value.code == xb.E_UNSUPPORTED
+        g.split(y, parts_k=-2)
+    assert e.value.code == xb.E_BAD_SPLIT
     for call in (lambda: g.bind(256, 256), lambda: g.run(1, [1], [1]), lambda: g.plan(), lambda: g.status()):
         with pytest.raises(xb.XenosError) as e:
             call()
@@ -266,7 +266,7 @@ def test_gemm_split_prefers_output_channels_until_units_are_busy():
                 continue
             assert L["tile_n"] % 16 == 0 and 16 <= L["tile_n"] <= 256
             assert L["npad"] == L["tile_n"] * L["n_tiles"] and (L["n_tiles"] - 1) * L["tile_n"] < L["K"] <= L["npad"]
-            assert L["grid"] == min(148, L["m_tiles"] * L["n_tiles"])     # one persistent CTA per unit
+            assert L["grid"] == min(148, L["m_tiles"] * L["n_tiles"] * L["ksplit"])     # one persistent CTA per unit
             if L["n_tiles"] > -(-L["K"] // 256):               # split finer than the 256-wide maximum
                 assert L["m_tiles"] * (L["n_tiles"] // 2) < 148   # ... only because units would idle otherwise
                 if L["a0"] == "dw":
@@ -278,6 +278,50 @@ def test_gemm_split_prefers_output_channels_until_units_are_busy():
     hw = xb.HwInfo(16, 227 * 1024, 512, 1 << 20)
     g2, _ = compiled(spec, 1, hw=hw)
     assert g2.plan()["hw"]["sm_count"] == 16
+
+
+def _unit(build, cin, hw):
+    g = GraphSpec("unit", (cin, hw, hw))
+    build(g)
+    return g
+
+
+@pytest.mark.parametrize("parts_k", [2, 3, 4, 6, 9, 18, 36])
+def test_reduction_split_is_an_ascending_exact_cover_of_the_k_blocks(parts_k):
+    """Section 4.2.2: the reduction (C, R, S) is cut last and needs an additional reduction.  Here: chunks of
+    64-element K blocks, equal size, ascending, disjoint, complete."""
+    spec = _unit(lambda g: g.cbr("c", "input", 48, 3, 1, 1), 256, 6)        # K = 256 * 9 = 36 blocks
+    g, _ = compiled(spec, 2, linked=False, splits=[("c", dict(parts_k=parts_k))], nhwc=True)
+    L = g.plan()["launches"][0]
+    assert L["kblocks"] == 36 and L["ksplit"] == parts_k
+    chunks = [(s * L["kb_per"], min(L["kblocks"], (s + 1) * L["kb_per"])) for s in range(L["ksplit"])]
+    assert chunks[0][0] == 0 and chunks[-1][1] == L["kblocks"]
+    assert all(a < b for a, b in chunks) and all(chunks[i][1] == chunks[i + 1][0] for i in range(len(chunks) - 1))
+    assert L["grid"] == min(148, L["m_tiles"] * L["n_tiles"] * parts_k)
+
+
+def test_reduction_split_requests_that_cannot_be_met():
+    spec = _unit(lambda g: g.cbr("c", "input", 48, 3, 1, 1), 256, 6)
+    for pk, code in ((37, xb.E_BAD_SPLIT), (7, xb.E_BAD_SPLIT), (10, xb.E_BAD_SPLIT)):     # 36 blocks: 7 -> 6 chunks of 6, 10 -> 9 of 4
+        with pytest.raises(xb.XenosError) as e:
+            compiled(spec, 2, linked=False, splits=[("c", dict(parts_k=pk))], nhwc=True)
+        assert e.value.code == code, pk
+    m = graphs.mobilenet_v1(hw=32, width=0.25, classes=8)
+    with pytest.raises(xb.XenosError) as e:
+        compiled(m, 1, splits=[("pw1.relu6", dict(parts_k=2))])        # linked depthwise stage
+    assert e.value.code == xb.E_UNSUPPORTED
+    with pytest.raises(xb.XenosError) as e:
+        compiled(graphs.single_chain(), 1, splits=[("mp", dict(parts_k=2))])     # fp32 CUDA-core chain
+    assert e.value.code == xb.E_UNSUPPORTED
+
+
+def test_reduction_split_is_automatic_only_where_units_would_idle():
+    spec = graphs.mobilenet_v1()
+    g, _ = compiled(spec, 32)
+    L = g.plan()["launches"]
+    assert [l["ksplit"] for l in L[:-1]] == [1] * (len(L) - 1)
+    fc = L[-1]
+    assert fc["ksplit"] >= 2 and fc["m_tiles"] * fc["n_tiles"] * fc["ksplit"] <= 148 and fc["kb_per"] >= 2
 
 
 def test_user_outc_split_sets_tiles():
