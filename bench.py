@@ -30,7 +30,18 @@ WORKLOADS = {
     "resnet18_b32": (2, 32), "resnet18_b1": (2, 1),
     "squeezenet11_b32": (3, 32), "squeezenet11_b1": (3, 1),
     "resnet50_stress_b64": (4, 64), "single_chain_b1": (0, 1),
+    # the paper's operator micro-benchmarks (Table 4): the first two exercise linking (other arm: unlinked), the
+    # last two the split (other arm: the coarsest split the kernels allow, 256-wide channel tiles, K uncut)
+    "op_cbr_maxpool_b32": ("cbr_maxpool", 32), "op_cbr_avgpool_b32": ("cbr_avgpool", 32),
+    "op_fc_b32": ("fc", 32), "op_cbr_b32": ("cbr", 32),
+    "op_cbr_maxpool_b1": ("cbr_maxpool", 1), "op_cbr_avgpool_b1": ("cbr_avgpool", 1),
+    "op_fc_b1": ("fc", 1), "op_cbr_b1": ("cbr", 1),
 }
+SPLIT_WORKLOADS = {"fc": "fc", "cbr": "c"}      # operator benchmark -> the operator whose split the other arm coarsens
+
+
+def workload_spec(key):
+    return graphs.operator_benchmark(key) if isinstance(key, str) else graphs.config(key)[0]
 L2_FLUSH_BYTES = 256 << 20
 MIN_TIMED_SECONDS = 0.3      # the K timed steps are repeated until the timed region covers at least this long
 
@@ -157,7 +168,7 @@ def main():
     ap.add_argument("--unlinked", action="store_true", help="time the unlinked execution as the main arm")
     args = ap.parse_args()
     cfg, batch = WORKLOADS[args.workload]
-    spec, _ = graphs.config(cfg)
+    spec = workload_spec(cfg)
     if args.impl == "reference":
         reference_arm(args, spec, batch)
         return
@@ -178,9 +189,21 @@ def main():
     P = graphs.make_params(spec)
     x = graphs.make_input(spec, batch)
 
+    # images enter as NCHW; feature maps with 8 or more channels enter as NHWC bf16, the layout between kernels
+    nhwc = (not fp32) and spec.in_shape[0] >= 8
+    split_op = SPLIT_WORKLOADS.get(cfg) if isinstance(cfg, str) else None
+    other_name = "coarsest split" if split_op else "unlinked"
+
     def make(linked):
-        g, ids = graph_from_spec(spec, P, in_dtype=xb.DTYPE_F32 if fp32 else xb.DTYPE_BF16, in_layout=xb.LAYOUT_NCHW)
-        if linked:
+        g, ids = graph_from_spec(spec, P, in_dtype=xb.DTYPE_F32 if fp32 else xb.DTYPE_BF16,
+                                 in_layout=xb.LAYOUT_NHWC if nhwc else xb.LAYOUT_NCHW)
+        if split_op:
+            # main arm: the automatic split; other arm: as few, as wide tiles as the kernels allow
+            g.link()
+            if not linked:
+                cout = [o for o in spec.ops if o["name"] == split_op][0]["cout"]
+                g.split(ids[split_op], parts_outc=-(-cout // 256), parts_k=1)
+        elif linked:
             g.link()
         nbytes = g.compile(batch, xb.PRECISION_FP32_CUDA_CORE if fp32 else xb.PRECISION_BF16_TENSOR)
         ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device="cuda")
@@ -188,6 +211,9 @@ def main():
         return g, ws
 
     stream = torch.cuda.current_stream().cuda_stream
+    x_nchw = x
+    if nhwc:
+        x = np.ascontiguousarray(x.transpose(0, 2, 3, 1))
     x_host = torch.from_numpy(x) if fp32 else torch.from_numpy(x).to(torch.bfloat16)
     x_pin = x_host.pin_memory()
     x_dev = x_host.cuda()
@@ -354,7 +380,7 @@ def main():
                          loop="copy of step i+1 overlaps compute of step i (two device buffers); L2 flush inside the timed loop"),
                 gpu_launches=g_main.launch_count() * args.steps * repeats,
                 roofline=roof,
-                linked_vs_unlinked=dict(other_mode="linked" if args.unlinked else "unlinked", other_value=other_val,
+                linked_vs_unlinked=dict(other_mode="linked" if args.unlinked else other_name, other_value=other_val,
                                         speedup=(value / other_val) if not args.unlinked else (other_val / value),
                                         launches_linked=(g_other if args.unlinked else g_main).launch_count(),
                                         launches_unlinked=(g_main if args.unlinked else g_other).launch_count(),
@@ -365,10 +391,10 @@ def main():
         from oracle import interp
         # a bounded sample of the same workload: whole passes of up to 16 images until about 10 s of CPU work
         sample = min(batch, 16)
-        interp.run_graph(spec, P, x[:1])
+        interp.run_graph(spec, P, x_nchw[:1])
         passes, t0 = 0, time.perf_counter()
         while True:
-            interp.run_graph(spec, P, x[:sample])
+            interp.run_graph(spec, P, x_nchw[:sample])
             passes += 1
             dt = time.perf_counter() - t0
             if dt >= 10.0 or passes >= 64:

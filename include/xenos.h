@@ -164,6 +164,24 @@ XENOS_API xenos_status_t xenos_graph_link(xenos_graph_t *g, const xenos_id_t *op
 XENOS_API xenos_status_t xenos_graph_split(xenos_graph_t *g, xenos_id_t op, int32_t parts_outc,
                                            int32_t parts_h, int32_t parts_w, int32_t parts_k);
 
+/* Profiling-driven split search (Algorithm 1, "Enumerating Partition Schemes", Section 5, restated for one
+ * GPU): for every chain the library enumerates split schemes (output-channel parts and reduction parts of a
+ * tensor-core chain; output-channel / row / column parts of the fp32 chain), compiles trial plans, runs each
+ * `repeats` times at batch = max_batch on the caller's buffers and keeps, per chain, the fastest scheme, which
+ * it records as if xenos_graph_split had been called; chains whose split the caller fixed are left alone.
+ * Call it after the link requests and before xenos_graph_compile, with the same max_batch and precision.
+ * workspace_dev: DEVICE, 256-byte aligned, large enough for every trial plan (a little more than the plain
+ * plan: XENOS_E_WORKSPACE names the size when it is not); inputs_dev / outputs_dev as for xenos_graph_run, with
+ * valid images in the inputs (outputs are overwritten).  The call synchronises the stream.  report_json
+ * (HOST, may be NULL) receives {"trials", "chains":[{"id","tensor","chosen","candidates":[{"label",
+ * "parts_outc","parts_h","parts_w","parts_k","us"}]}]}; *needed (HOST) the bytes it takes.
+ * Errors: XENOS_E_STATE after compile, XENOS_E_CUDA without an sm_100 device, otherwise those of compile / run. */
+XENOS_API xenos_status_t xenos_graph_search_split(xenos_graph_t *g, int32_t max_batch, int32_t precision,
+                                                  void *workspace_dev, size_t workspace_bytes,
+                                                  const void *const *inputs_dev, void *const *outputs_dev,
+                                                  void *cuda_stream, int32_t max_trials, int32_t repeats,
+                                                  char *report_json, size_t cap, size_t *needed);
+
 /* Host only: pre-fusion, BatchNorm folding, link + split plans, weight packing, workspace
  * layout.  *workspace_bytes receives the device bytes xenos_graph_bind needs. */
 XENOS_API xenos_status_t xenos_graph_compile(xenos_graph_t *g, int32_t max_batch, int32_t precision,

@@ -41,7 +41,7 @@ class OpDesc(ctypes.Structure):
 
 
 EXPORTS = ["xenos_graph_create", "xenos_graph_add_input", "xenos_graph_add_op", "xenos_graph_mark_output",
-           "xenos_graph_link", "xenos_graph_split", "xenos_graph_compile", "xenos_graph_bind", "xenos_graph_run",
+           "xenos_graph_link", "xenos_graph_split", "xenos_graph_search_split", "xenos_graph_compile", "xenos_graph_bind", "xenos_graph_run",
            "xenos_graph_profile", "xenos_graph_run_builtin_scratch", "xenos_graph_status", "xenos_graph_selftest_wait_expiry", "xenos_graph_get_plan", "xenos_graph_launch_count", "xenos_graph_destroy",
            "xenos_last_error"]
 
@@ -61,6 +61,8 @@ def lib() -> ctypes.CDLL:
         L.xenos_graph_mark_output.argtypes = [vp, i32, i32, i32]
         L.xenos_graph_link.argtypes = [vp, ctypes.POINTER(i32), i32]
         L.xenos_graph_split.argtypes = [vp, i32, i32, i32, i32, i32]
+        L.xenos_graph_search_split.argtypes = [vp, i32, i32, vp, sz, ctypes.POINTER(vp), ctypes.POINTER(vp), vp, i32, i32,
+                                               ctypes.c_char_p, sz, ctypes.POINTER(sz)]
         L.xenos_graph_compile.argtypes = [vp, i32, i32, ctypes.POINTER(sz)]
         L.xenos_graph_bind.argtypes = [vp, vp, sz, vp]
         L.xenos_graph_run.argtypes = [vp, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), vp]
@@ -137,6 +139,17 @@ class Graph:
 
     def split(self, op: int = -1, parts_outc=0, parts_h=0, parts_w=0, parts_k=1):
         self._check(lib().xenos_graph_split(self._h, op, parts_outc, parts_h, parts_w, parts_k))
+
+    def search_split(self, max_batch: int, precision: int, workspace_ptr: int, nbytes: int, inputs: Sequence[int],
+                     outputs: Sequence[int], stream: int = 0, max_trials: int = 8, repeats: int = 5) -> dict:
+        ins = (ctypes.c_void_p * len(inputs))(*inputs)
+        outs = (ctypes.c_void_p * len(outputs))(*outputs)
+        need = ctypes.c_size_t()
+        cap = 1 << 20
+        buf = ctypes.create_string_buffer(cap)
+        self._check(lib().xenos_graph_search_split(self._h, max_batch, precision, workspace_ptr, nbytes, ins, outs, stream,
+                                                   max_trials, repeats, buf, cap, ctypes.byref(need)))
+        return json.loads(buf.value.decode())
 
     def compile(self, max_batch: int, precision: int) -> int:
         n = ctypes.c_size_t()

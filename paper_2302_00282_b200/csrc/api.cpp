@@ -196,6 +196,38 @@ xenos_status_t xenos_graph_split(xenos_graph_t *gp, xenos_id_t op, int32_t parts
     XENOS_GUARD_END(gp)
 }
 
+xenos_status_t xenos_graph_search_split(xenos_graph_t *gp, int32_t max_batch, int32_t precision, void *workspace_dev,
+                                        size_t workspace_bytes, const void *const *inputs_dev, void *const *outputs_dev,
+                                        void *cuda_stream, int32_t max_trials, int32_t repeats, char *report_json, size_t cap,
+                                        size_t *needed) {
+    if (!gp) return XENOS_E_INVALID;
+    XENOS_GUARD_BEGIN
+    Graph &g = gp->g;
+    if (g.state != ST_BUILD) return fail(g, XENOS_E_STATE, "search_split after compile");
+    if (max_batch < 1 || max_batch > 65535) return fail(g, XENOS_E_INVALID, "search_split: max_batch out of range");
+    if (precision != XENOS_PRECISION_FP32_CUDA_CORE && precision != XENOS_PRECISION_BF16_TENSOR)
+        return fail(g, XENOS_E_INVALID, "search_split: unknown precision");
+    if (!workspace_dev || ((uintptr_t)workspace_dev & 255u)) return fail(g, XENOS_E_WORKSPACE, "search_split: workspace is NULL or not 256-byte aligned");
+    if (max_trials < 1 || max_trials > 64 || repeats < 1 || repeats > 1000) return fail(g, XENOS_E_INVALID, "search_split: max_trials must be 1..64 and repeats 1..1000");
+    if (!inputs_dev || !outputs_dev || !needed) return fail(g, XENOS_E_INVALID, "search_split: NULL pointer");
+    for (size_t i = 0; i < g.inputs.size(); ++i)
+        if (!inputs_dev[i] || ((uintptr_t)inputs_dev[i] & 15u)) return fail(g, XENOS_E_INVALID, "search_split: input pointer is NULL or not 16-byte aligned");
+    for (size_t i = 0; i < g.outputs.size(); ++i)
+        if (!outputs_dev[i] || ((uintptr_t)outputs_dev[i] & 15u)) return fail(g, XENOS_E_INVALID, "search_split: output pointer is NULL or not 16-byte aligned");
+    std::string report;
+    xenos_status_t st = search_splits(g, max_batch, precision, workspace_dev, workspace_bytes, inputs_dev, outputs_dev, cuda_stream,
+                                      max_trials, repeats, report);
+    if (st != XENOS_OK) return st;
+    *needed = report.size() + 1;
+    if (report_json && cap > 0) {
+        size_t n = report.size() < cap - 1 ? report.size() : cap - 1;
+        std::memcpy(report_json, report.data(), n);
+        report_json[n] = '\0';
+    }
+    return XENOS_OK;
+    XENOS_GUARD_END(gp)
+}
+
 xenos_status_t xenos_graph_compile(xenos_graph_t *gp, int32_t max_batch, int32_t precision, size_t *workspace_bytes) {
     if (!gp) return XENOS_E_INVALID;
     XENOS_GUARD_BEGIN

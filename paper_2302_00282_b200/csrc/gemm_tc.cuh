@@ -86,7 +86,14 @@ struct GemmParams {
     long long split_stride;
     float *split_part;
     unsigned int *split_cnt;
+    int launch_id;                                  // position of this launch in the plan, reported with a give-up
 };
+
+// Status word of a wait that gave up: the code, the role that waited (1 TMA, 2 MMA, 3 producer, 4 producer helping
+// with the last tile, 5 epilogue) and the launch.
+__device__ __forceinline__ unsigned timeout_word(const GemmParams &g, int role) {
+    return kStatusTimeout | ((unsigned)role << 8) | (((unsigned)g.launch_id & 0xfffu) << 12);
+}
 
 // ---- PTX wrappers ------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -541,6 +548,22 @@ struct DwUnit {
     int live;
 };
 
+// The unit of producer thread pt: (pixel block, channel quad) of the tile's depthwise stage.
+__device__ __forceinline__ DwUnit make_dw_unit(const GemmParams &g, int pt, int dw_quads, int dw_br) {
+    DwUnit du;
+    du.q = pt & (dw_quads - 1);
+    const int blk = pt / dw_quads;               // (image, block row, block column)
+    const int upr = g.rw >> 2, upi = ((g.rh + dw_br - 1) / dw_br) * upr;
+    const int img = blk / upi, rem = blk - img * upi;
+    const int uy = rem / upr, ux = rem - uy * upr;
+    const int S = g.seg[0].stride;
+    du.live = img < g.ni && du.q * 4 < g.halo_cb;
+    du.base = ((img * g.halo_h + dw_br * uy * S) * g.halo_w + 4 * ux * S) * g.halo_cb * 2 + du.q * 8;
+    du.row0 = img * g.rh * g.rw + dw_br * uy * g.rw + 4 * ux;
+    du.nrows = min(dw_br, max(0, g.rh - dw_br * uy));
+    return du;
+}
+
 __device__ __forceinline__ uint32_t clamp_bf16x2(uint32_t v, uint32_t lo, uint32_t hi) {
     __nv_bfloat162 x = *reinterpret_cast<__nv_bfloat162 *>(&v);
     x = __hmin2(__hmax2(x, *reinterpret_cast<__nv_bfloat162 *>(&lo)), *reinterpret_cast<__nv_bfloat162 *>(&hi));
@@ -854,7 +877,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                     st.next(g.stages);
                 }
             }
-            if (!ok) atomicCAS(g.status, 0u, kStatusTimeout);
+            if (!ok) atomicCAS(g.status, 0u, timeout_word(g, 1));
         }
     } else if (warp == 1) {
         // ---- MMA issue ----
@@ -889,7 +912,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                     if (ti + (int)gridDim.x >= total_tiles) umma_commit(lastf_bar);
                 }
             }
-            if (!ok) atomicCAS(g.status, 0u, kStatusTimeout);
+            if (!ok) atomicCAS(g.status, 0u, timeout_word(g, 2));
         }
     } else if (warp < 2 + kProducerThreads / 32) {
         // ---- activation operand ----
@@ -900,16 +923,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
         int zero_from = 8;                               // chunks >= zero_from of every row are K padding
         if (dw_mode) {
             zero_from = g.halo_cb >> 3;
-            du.q = pt & (dw_quads - 1);
-            const int blk = pt / dw_quads;               // (image, block row, block column)
-            const int upr = g.rw >> 2, upi = ((g.rh + dw_br - 1) / dw_br) * upr;
-            const int img = blk / upi, rem = blk - img * upi;
-            const int uy = rem / upr, ux = rem - uy * upr;
-            const int S = g.seg[0].stride;
-            du.live = img < g.ni && du.q * 4 < g.halo_cb;
-            du.base = ((img * g.halo_h + dw_br * uy * S) * g.halo_w + 4 * ux * S) * g.halo_cb * 2 + du.q * 8;
-            du.row0 = img * g.rh * g.rw + dw_br * uy * g.rw + 4 * ux;
-            du.nrows = min(dw_br, max(0, g.rh - dw_br * uy));
+            du = make_dw_unit(g, pt, dw_quads, dw_br);
         }
         // K-padding chunks of a depthwise stage are only ever written with zeros: when no other
         // producer shares the ring they are cleared once, here, instead of with every K block
@@ -1035,7 +1049,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                 }
             }
         }
-        if (!ok && lane == 0) atomicCAS(g.status, 0u, kStatusTimeout);
+        if (!ok && lane == 0) atomicCAS(g.status, 0u, timeout_word(g, 3));
         cp_async_wait<0>();      // nothing of this thread is in flight when the CTA retires
         if (help_last && ok) {
             // this CTA's last tile: which one it is, which accumulator it sits in
@@ -1058,7 +1072,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                     const int ch0 = min(nch, help_per * (1 + helper)), ch1 = min(nch, help_per * (2 + helper));
                     store_chunks(g, t_lane, g.bias + last.nt * g.tile_n, last.nt * g.tile_n, ch0, ch1, rq, pix, plo, phi, wide_ok);
                     tc_fence_before();
-                } else if (lane == 0) atomicCAS(g.status, 0u, kStatusTimeout);
+                } else if (lane == 0) atomicCAS(g.status, 0u, timeout_word(g, 4));
             }
         }
     } else {
@@ -1301,7 +1315,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                 epi_bar();          // the staging tile is free for the next tile
             }
         }
-        if (!ok && lane == 0) atomicCAS(g.status, 0u, kStatusTimeout);
+        if (!ok && lane == 0) atomicCAS(g.status, 0u, timeout_word(g, 5));
     }
     tc_fence_before();
     __syncthreads();

@@ -203,6 +203,9 @@ xenos_status_t split_and_lower(Graph &g);
 xenos_status_t plan_workspace(Graph &g);
 void emit_plan_json(Graph &g);
 uint16_t f32_to_bf16_rne(float f);
+// search.cpp
+xenos_status_t search_splits(Graph &g, int max_batch, int precision, void *ws, size_t ws_bytes, const void *const *in,
+                             void *const *out, void *stream, int max_trials, int repeats, std::string &report);
 // runtime.cu
 xenos_status_t runtime_bind(Graph &g, void *ws, size_t bytes, void *stream);
 xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *const *out, void *stream,

@@ -298,6 +298,7 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
             p.act = L.act; p.act2 = L.act2; p.epi = L.epi; p.out_ctot = L.out_ctot; p.out_coff = L.out_coff;
             p.out_f32 = L.out_dtype == XENOS_DTYPE_F32;
             p.idesc = make_idesc(L.tile_n);
+            p.launch_id = (int)li;
             if (L.map_mode == MAP_PATCH) p.m_tiles = ((N + L.ni - 1) / L.ni) * L.tiles_y * L.tiles_x;
             else if (L.epi == EPI_GAP) p.m_tiles = (N + L.imgs_per_tile - 1) / L.imgs_per_tile;
             else p.m_tiles = (int)(((long long)N * L.rows_per_image + 127) / 128);
@@ -369,7 +370,12 @@ xenos_status_t runtime_status(Graph &g, void *stream_v) {
     if (word == 0) return XENOS_OK;
     cudaMemset(ws + g.status_off, 0, 256 + g.cnt_bytes);      // (the arrival counters of a run that gave up are stale too)
     int code = -(int)(word & 0xffu);
-    return fail(g, code, code == XENOS_E_TIMEOUT ? "a kernel gave up a bounded wait" : "a kernel failed an index check");
+    if (code == XENOS_E_TIMEOUT) {
+        static const char *role[] = {"a wait", "the TMA warp", "the MMA warp", "a producer warp", "a producer warp at the last tile", "an epilogue warp"};
+        const unsigned r = (word >> 8) & 0xfu;
+        return fail(g, code, std::string("a kernel gave up a bounded wait (") + role[r < 6 ? r : 0] + ", launch " + std::to_string((word >> 12) & 0xfffu) + ")");
+    }
+    return fail(g, code, "a kernel failed an index check");
 }
 
 xenos_status_t runtime_selftest_wait_expiry(Graph &g, void *stream_v) {

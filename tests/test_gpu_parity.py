@@ -391,6 +391,84 @@ def test_a_wait_that_runs_out_is_reported_and_the_device_stays_usable():
     assert np.array_equal(gg.run(x), ref)        # and the next run is a normal one
 
 
+# ---- profiling-driven split search (Algorithm 1 on one GPU) ---------------------------------------------
+def _searched(spec, batch, in_mode):
+    """Builds the graph twice: once plainly (for the workspace size), once with the split search before compile."""
+    import torch
+    from paper_2302_00282_b200 import binding as xb
+    from xenos_workloads.feed import graph_from_spec
+    P = graphs.make_params(spec)
+    x = graphs.make_input(spec, batch)
+    if in_mode != "f32_nchw":
+        x = xo.round_bf16(x)
+    plain = GpuGraph(spec, P, batch, linked=True, in_mode=in_mode)
+    y_plain = plain.run(x)
+    dt, lay = {"f32_nchw": (xb.DTYPE_F32, xb.LAYOUT_NCHW), "bf16_nhwc": (xb.DTYPE_BF16, xb.LAYOUT_NHWC)}[in_mode]
+    g, ids = graph_from_spec(spec, P, in_dtype=dt, in_layout=lay)
+    g.link()
+    prec = xb.PRECISION_FP32_CUDA_CORE if spec.precision == "fp32" else xb.PRECISION_BF16_TENSOR
+    ws = torch.empty(2 * plain.ws.numel() + (8 << 20), dtype=torch.uint8, device="cuda")
+    xin, out = plain.upload(x), plain.alloc_out(batch)
+    report = g.search_split(batch, prec, ws.data_ptr(), ws.numel(), [xin.data_ptr()], [out.data_ptr()], plain.stream, max_trials=6, repeats=3)
+    nbytes = g.compile(batch, prec)
+    assert nbytes <= ws.numel()
+    g.bind(ws.data_ptr(), ws.numel(), plain.stream)
+    out2 = plain.alloc_out(batch)
+    g.run(batch, [xin.data_ptr()], [out2.data_ptr()], plain.stream)
+    g.status(plain.stream)
+    y = out2.float().cpu().numpy()
+    if y.ndim == 4 and spec.precision != "fp32":
+        y = np.ascontiguousarray(y.transpose(0, 3, 1, 2))
+    return report, g.plan(), y, y_plain, interp.run_graph(spec, P, x)
+
+
+def test_split_search_keeps_the_fastest_measured_scheme_bf16():
+    def build(g):
+        x = g.cbr("c1", "input", 96, 3, 1, 1)
+        x = g.cbr("c2", x, 320, 1, 1, 0)
+        x = g.gap("gap", x)
+        g.fc("fc", x, 200)
+    spec = _one(build, 64, 12)
+    report, plan, y, y_plain, o = _searched(spec, 4, "bf16_nhwc")
+    assert report["trials"] >= 3 and len(report["chains"]) == len(plan["chains"])
+    for c in report["chains"]:
+        us = [k["us"] for k in c["candidates"]]
+        assert all(u > 0 for u in us) and us[c["chosen"]] == min(us)          # PROFILING, then the minimum
+        assert c["candidates"][0]["label"] == "planner"
+    assert any(len(c["candidates"]) >= 3 for c in report["chains"])
+    # the chosen schemes are in the compiled plan
+    for c in report["chains"]:
+        k = c["candidates"][c["chosen"]]
+        L = plan["launches"][plan["chains"][c["id"]]["launches"][0]]
+        if c["chosen"] > 0 and L["kind"] == "gemm":
+            assert L["n_tiles"] == k["parts_outc"] and L["ksplit"] == k["parts_k"]
+    assert abs_err_scaled(y, o) <= BF16_TOL and abs_err_scaled(y, y_plain) <= 2.0 ** -7
+
+
+def test_split_search_on_the_fp32_chain():
+    spec = graphs.single_chain()
+    report, plan, y, y_plain, o = _searched(spec, 1, "f32_nchw")
+    c = report["chains"][0]
+    assert len(c["candidates"]) >= 4
+    k = c["candidates"][c["chosen"]]
+    L = plan["launches"][0]
+    if c["chosen"] > 0:
+        assert (L["parts_outc"], L["tiles_h"], L["tiles_w"]) == (k["parts_outc"], k["parts_h"], k["parts_w"])
+    assert np.array_equal(y, y_plain)             # Eq. 1: a split changes no value of the fp32 chain
+    assert rel_err_fp32(y, o) <= FP32_TOL
+
+
+# ---- the paper's operator micro-benchmarks (Table 4) ------------------------------------------------------
+@pytest.mark.parametrize("linked", [True, False])
+@pytest.mark.parametrize("name,batch,launches", [("cbr_maxpool", 2, 1), ("cbr_avgpool", 5, 1), ("fc", 5, 2), ("cbr", 2, 1)])
+def test_bf16_operator_benchmarks(name, batch, launches, linked):
+    spec = graphs.operator_benchmark(name)
+    mode = "bf16_nchw" if spec.in_shape[0] < 8 else "bf16_nhwc"
+    _, _, gg = check_bf16(f"op_{name}", spec, batch, linked=linked, in_mode=mode)
+    if linked:
+        assert gg.g.launch_count() == launches
+
+
 # ---- bf16: whole graphs ---------------------------------------------------------------------------
 @pytest.mark.parametrize("linked", [True, False])
 @pytest.mark.parametrize("name,kw", [("mobilenet_v1", dict(hw=64, width=0.25, classes=24)),

@@ -115,6 +115,25 @@ def test_bind_fails_loudly_without_a_device():
     assert e.value.code == xb.E_CUDA
 
 
+def test_split_search_needs_a_device_and_the_build_state():
+    """The PROFILING step of the search runs on the GPU: without one the call fails loudly and leaves the graph as
+    it was; after compile the call is out of order."""
+    spec = graphs.mobilenet_v1(hw=32, width=0.25, classes=8)
+    P = graphs.make_params(spec)
+    g, _ = graph_from_spec(spec, P)
+    g.link()
+    with pytest.raises(xb.XenosError) as e:
+        g.search_split(2, xb.PRECISION_BF16_TENSOR, 256, 1 << 30, [256], [256])
+    assert e.value.code in (xb.E_CUDA, xb.E_WORKSPACE)
+    with pytest.raises(xb.XenosError) as e:
+        g.search_split(2, xb.PRECISION_BF16_TENSOR, 0, 1 << 30, [256], [256])
+    assert e.value.code == xb.E_WORKSPACE
+    g.compile(2, xb.PRECISION_BF16_TENSOR)
+    with pytest.raises(xb.XenosError) as e:
+        g.search_split(2, xb.PRECISION_BF16_TENSOR, 256, 1 << 30, [256], [256])
+    assert e.value.code == xb.E_STATE
+
+
 def test_prefusion_folds_bn_and_activation():
     spec = graphs.single_chain()
     g, _ = compiled(spec, 1, linked=False)

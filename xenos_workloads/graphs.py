@@ -237,6 +237,39 @@ def resnet50_stress(hw: int = 512, base: int = 64, blocks=(3, 4, 6, 3)) -> Graph
     return g
 
 
+# ------------------------------------------------------------------------------------------------
+# The paper's operator micro-benchmarks (Table 4, Section 7.3)
+# ------------------------------------------------------------------------------------------------
+def operator_benchmark(name: str) -> GraphSpec:
+    """One of the four operators of Table 4.  The table gives a feature map and a kernel per row and says which
+    optimisation the row exercises (linking for the first two, split for the last two); pooling windows are not
+    printed, and the first row's sizes are garbled ("224x224x24" with a kernel "3x3x3x224"): it is read as a
+    224 x 224 x 3 image, a 3x3x3x24 kernel with stride 1 and padding 1 (a 224 x 224 x 24 map), then a 2 x 2
+    stride-2 max pool; the average pool of the second row is the global average over the 7 x 7 map.  The fully
+    connected row reads a 1 x 1 x 1536 map, flattened by a global average over its single pixel."""
+    if name == "cbr_maxpool":
+        g = GraphSpec("op_cbr_maxpool", (3, 224, 224))
+        x = g.cbr("c", "input", 24, 3, 1, 1)
+        g.pool("mp", x, "maxpool", 2, 2, 0)
+    elif name == "cbr_avgpool":
+        g = GraphSpec("op_cbr_avgpool", (1024, 7, 7))
+        x = g.cbr("c", "input", 1024, 1, 1, 0)
+        g.gap("ap", x)
+    elif name == "fc":
+        g = GraphSpec("op_fc", (1536, 1, 1))
+        x = g.gap("flat", "input")
+        g.fc("fc", x, 1000)
+    elif name == "cbr":
+        g = GraphSpec("op_cbr", (32, 112, 112))
+        g.cbr("c", "input", 64, 1, 1, 0)
+    else:
+        raise ValueError(name)
+    return g
+
+
+OPERATOR_BENCHMARKS = ("cbr_maxpool", "cbr_avgpool", "fc", "cbr")
+
+
 def config(i: int) -> Tuple[GraphSpec, List[int]]:
     """Workload i of the benchmark list with the batch sizes it is quoted at."""
     if i == 0:
