@@ -79,9 +79,10 @@ struct GemmParams {
     int off_halo, off_stg, off_dww, off_bias, off_bar;   // shared-memory offsets from the 1024-aligned base
     int act, act2, epi, out_ctot, out_coff, out_f32, skip_ctot;
     uint32_t idesc;
-    // reduction split (Section 4.2.2, the C / R / S split that "requires additional reduction"): the K blocks are cut into
-    // ksplit chunks of kb_per blocks; n_tiles counts (channel tile, chunk) pairs, chunk fastest; partial sums go to
-    // split_part [chunk][output pixel][split_ld] as fp32 and the CTA that finishes a tile last adds them in chunk order
+    // reduction split (Section 4.2.2: the C / R / S split, which needs an additional reduction): the K blocks are cut
+    // into ksplit chunks of kb_per blocks; n_tiles counts (channel tile, chunk) pairs, chunk fastest; partial sums go to
+    // split_part [chunk][output pixel][split_ld] as fp32; when all chunks of a tile have arrived (split_cnt), each
+    // chunk's CTA adds the chunks, in ascending order, for its share of the tile's rows
     int ksplit, kb_per, split_ld;
     long long split_stride;
     float *split_part;
@@ -685,6 +686,33 @@ __device__ __forceinline__ void store_chunks(const GemmParams &g, uint32_t t_lan
     }
 }
 
+// Four adjacent columns of one output pixel: bias, activation, identity-shortcut add, second activation, store.
+// (nc is a multiple of 4 and channel counts are multiples of 8, so the four columns are inside the tensor or, for
+// fp32 vector outputs, checked one by one.)
+__device__ __forceinline__ void finish_store4(const GemmParams &g, float4 a, const float4 bz, int nc, size_t pix) {
+    const float lo1 = act_lo(g.act), hi1 = act_hi(g.act), lo2 = act_lo(g.act2), hi2 = act_hi(g.act2);
+    float v[4] = {a.x + bz.x, a.y + bz.y, a.z + bz.z, a.w + bz.w};
+#pragma unroll
+    for (int c = 0; c < 4; ++c) v[c] = fminf(fmaxf(v[c], lo1), hi1);
+    if (g.skip) {
+        const uint2 sk = __ldg(reinterpret_cast<const uint2 *>(g.skip + pix * g.skip_ctot + nc));
+        v[0] += __uint_as_float(sk.x << 16); v[1] += __uint_as_float(sk.x & 0xffff0000u);
+        v[2] += __uint_as_float(sk.y << 16); v[3] += __uint_as_float(sk.y & 0xffff0000u);
+    }
+    if (g.act2) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) v[c] = fminf(fmaxf(v[c], lo2), hi2);
+    }
+    if (g.out_f32) {
+        float *o = reinterpret_cast<float *>(g.out) + pix * g.out_ctot + g.out_coff + nc;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) if (nc + c < g.N) o[c] = v[c];
+    } else {
+        __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(g.out) + pix * g.out_ctot + g.out_coff + nc;
+        *reinterpret_cast<uint2 *>(o) = make_uint2(pack2(v[0], v[1]), pack2(v[2], v[3]));
+    }
+}
+
 // The general store epilogue for 16 columns of one tile row: bias, activation, identity-shortcut add, second
 // activation, then fp32 or bf16 values at the row's position (channel offset included).
 __device__ __forceinline__ void finish_store16(const GemmParams &g, float *v, uint32_t sbias, int ch, int nc, const RowPos &rq, size_t pix) {
@@ -978,7 +1006,8 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
             const uint32_t dww = sbase + g.off_dww;
             const GemmSeg &sg = g.seg[0];
             for (; w.ti < total_tiles && ok; w.next(g)) {
-                for (int kb = 0; kb < g.kblocks && ok; ++kb) {
+                const TileK tk = tile_k<kSplit>(g, w.nt);
+                for (int kb = tk.kb0; kb < tk.kb1 && ok; ++kb) {
                     const int s = st.s, hs = hr.s;
                     ok = mbar_wait2_warp(empty_bar(s), st.ph ^ 1u, hfull_bar(hs), hr.ph, lane);
                     if (!ok) break;
@@ -1119,8 +1148,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
             tc_fence_after();
             const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * g.acc_stride;
             if (kSplit && g.ksplit > 1) {
-                // ---- reduction split: park this chunk's fp32 partial sums; the CTA that completes the tile adds
-                // the chunks in ascending order (a fixed order: results do not depend on which CTA came last)
+                // ---- reduction split: park this chunk's fp32 partial sums
                 float *part = g.split_part + (size_t)tk.ks * g.split_stride + pix * g.split_ld + n0;
                 for (int cbase = 0; cbase < nchunks; cbase += 2) {
                     float vv[32];
@@ -1135,32 +1163,51 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                         for (int q4 = 0; q4 < 32; q4 += 4)
                             if (q4 < nsub * 16) __stcg(reinterpret_cast<float4 *>(part + cbase * 16 + q4), make_float4(vv[q4], vv[q4 + 1], vv[q4 + 2], vv[q4 + 3]));
                 }
+                // Every chunk's CTA then adds the partial sums of ITS share of the tile's rows, chunks in ascending order
+                // (a fixed order: the result does not depend on which CTA arrives when): the reduction's traffic
+                // is spread over the CTAs that made the partial sums, and every load is a coalesced 16 bytes.
                 __threadfence();
                 epi_bar();
+                unsigned int *cnt = g.split_cnt + 2 * ((size_t)mt * (g.n_tiles / g.ksplit) + nt);      // [arrived, reduced]
                 if (et == 0) {
-                    unsigned int *cnt = g.split_cnt + (size_t)mt * (g.n_tiles / g.ksplit) + nt;
-                    const unsigned int old = atomicAdd(cnt, 1u);
-                    const int last = old == (unsigned int)(g.ksplit - 1);
-                    if (last) *cnt = 0u;                    // every chunk has arrived: ready for the next run
-                    fail_flag[1] = last;
+                    atomicAdd(cnt, 1u);
+                    int seen = 0;
+                    // the other chunks of this tile are consecutive tiles of the walk: they run on other units now, or
+                    // on units that are finishing an earlier tile (a wait never points at a later tile, so waits cannot
+                    // form a cycle); bounded like every other wait
+                    for (int spin = 0; spin < (1 << 22); ++spin) {
+                        if (*reinterpret_cast<volatile unsigned int *>(cnt) >= (unsigned int)g.ksplit) { seen = 1; break; }
+                        __nanosleep(64);
+                    }
+                    fail_flag[1] = seen;
+                    if (!seen) *fail_flag = 1;
                 }
                 epi_bar();
-                if (!fail_flag[1]) continue;
+                if (!fail_flag[1]) { ok = false; break; }
                 __threadfence();
-                for (int ch = 0; ch < nchunks; ++ch) {
-                    float v[16];
-#pragma unroll
-                    for (int c = 0; c < 16; ++c) v[c] = 0.0f;
-                    if (rq.valid)
+                {
+                    const int rows_per = (kTileM + g.ksplit - 1) / g.ksplit;
+                    const int r0 = tk.ks * rows_per, r1 = min(kTileM, r0 + rows_per);
+                    const int c4n = g.tile_n >> 2;
+                    for (int idx = et; idx < (r1 - r0) * c4n; idx += kEpilogueThreads) {
+                        const int rr = r0 + idx / c4n, c4 = idx - (rr - r0) * c4n;
+                        const RowPos rp = map_row(g, w, row_local(g, rr), rr);
+                        const int nc = n0 + c4 * 4;
+                        if (!rp.valid || nc >= g.N) continue;
+                        const size_t px = ((size_t)rp.n * g.P + rp.p) * g.Q + rp.q;
+                        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
                         for (int sp = 0; sp < g.ksplit; ++sp) {
-                            const float *ps = g.split_part + (size_t)sp * g.split_stride + pix * g.split_ld + n0 + ch * 16;
-#pragma unroll
-                            for (int q4 = 0; q4 < 16; q4 += 4) {
-                                const float4 x4 = __ldcg(reinterpret_cast<const float4 *>(ps + q4));
-                                v[q4] += x4.x; v[q4 + 1] += x4.y; v[q4 + 2] += x4.z; v[q4 + 3] += x4.w;
-                            }
+                            const float4 x4 = __ldcg(reinterpret_cast<const float4 *>(g.split_part + (size_t)sp * g.split_stride + px * g.split_ld + nc));
+                            a.x += x4.x; a.y += x4.y; a.z += x4.z; a.w += x4.w;
                         }
-                    finish_store16(g, v, sbias, ch, n0 + ch * 16, rq, pix);
+                        finish_store4(g, a, ld_shared_f4(sbias + (uint32_t)(c4 * 16)), nc, px);
+                    }
+                }
+                epi_bar();
+                if (et == 0) {
+                    __threadfence();
+                    const unsigned int old = atomicAdd(cnt + 1, 1u);
+                    if (old == (unsigned int)(g.ksplit - 1)) { cnt[0] = 0u; cnt[1] = 0u; }      // all have read: ready for the next run
                 }
                 continue;
             }

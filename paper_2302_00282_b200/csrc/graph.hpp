@@ -129,7 +129,7 @@ struct Launch {
     int stem_tma = 0, stem_align = 1;                              // stem: image patch by TMA, x alignment in elements
     int off_halo = 0, off_stg = 0, off_dww = 0, off_bias = 0, off_bar = 0;                    // shared-memory layout
     // reduction split: ksplit chunks of kb_per K blocks; fp32 partial sums [chunk][pixel][npad] in the workspace's
-    // split scratch, one arrival counter per (row tile, channel tile)
+    // split scratch, two counters (chunks arrived, chunks reduced) per (row tile, channel tile)
     int ksplit = 1, kb_per = 0;
     size_t split_cnt_off = 0;
     // ---- fp32 linked chain (conv kxk -> conv1x1 -> pool)

@@ -738,13 +738,17 @@ struct Lower {
         // sums are fp32 and the chunks are added in ascending order.  Chosen automatically only when the tiles
         // leave most units idle and K is long (fc, late convolutions at small batch).
         {
-            const bool can = s0.mode == AM_GATHER && s1.mode == AM_NONE && L.epi == EPI_STORE && L.map_mode == MAP_FLAT;
+            // (a linked depthwise stage can be split on request: a chunk's CTA then produces only its own channels of
+            // the depthwise result.  It is not chosen automatically: measured at batch 1 the partial sums and their
+            // reduction cost more than the shorter depthwise loop saves; the split search may still pick it.)
+            const bool plain = s0.mode == AM_GATHER && L.map_mode == MAP_FLAT;
+            const bool can = (plain || s0.mode == AM_DW) && s1.mode == AM_NONE && L.epi == EPI_STORE;
             int want = 1;
             if (rq.user && rq.k > 1) {
-                if (!can) return fail(g, XENOS_E_UNSUPPORTED, "split: parts_k applies to a plain convolution or fc (no linked depthwise stage, image stem, second K segment or pooling epilogue)");
+                if (!can) return fail(g, XENOS_E_UNSUPPORTED, "split: parts_k applies to a convolution, depthwise -> pointwise chain or fc that stores its tile (no image stem, second K segment or pooling epilogue)");
                 if (rq.k > L.kblocks) return fail(g, XENOS_E_BAD_SPLIT, "split: parts_k exceeds the number of 64-element K blocks");
                 want = rq.k;
-            } else if (!rq.user && can && L.kblocks >= 4 && (long)L.m_tiles * L.n_tiles * 2 <= g.hw.sm_count) {
+            } else if (!rq.user && can && plain && L.kblocks >= 4 && (long)L.m_tiles * L.n_tiles * 2 <= g.hw.sm_count) {
                 want = std::min(L.kblocks / 2, g.hw.sm_count / (L.m_tiles * L.n_tiles));
             }
             if (want > 1) {
@@ -958,7 +962,7 @@ xenos_status_t plan_workspace(Graph &g) {
     for (Launch &L : g.launches)
         if (L.kind == LK_GEMM && L.ksplit > 1) {
             L.split_cnt_off = off + g.cnt_bytes;
-            g.cnt_bytes += align_up((size_t)L.m_tiles * L.n_tiles * 4, 16);
+            g.cnt_bytes += align_up((size_t)L.m_tiles * L.n_tiles * 8, 16);      // [arrived, reduced] per tile
             g.split_bytes = std::max(g.split_bytes, (size_t)L.ksplit * g.max_batch * L.rows_per_image * L.npad * 4);
         }
     g.cnt_bytes = align_up(g.cnt_bytes, 256);

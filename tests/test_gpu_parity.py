@@ -279,6 +279,23 @@ def test_bf16_conv_reduction_split(parts_k):
     assert abs_err_scaled(y, base) <= 2.0 ** -8
 
 
+@pytest.mark.parametrize("stride,parts_k", [(1, 2), (1, 4), (2, 4)])
+def test_bf16_dw_pw_reduction_split(stride, parts_k):
+    """Depthwise -> pointwise with the reduction cut: each chunk's CTA computes the depthwise result of its own
+    channels only (256 channels = 4 K blocks)."""
+    def build(g):
+        x = g.cbr("dw", "input", 256, 3, stride, 1, groups=256, act="relu6")
+        g.cbr("pw", x, 96, 1, act="relu6")
+    spec = _one(build, 256, 13)
+    y, o, gg = check_bf16(f"dw_pw_splitk{parts_k}_s{stride}", spec, 3, linked=True, in_mode="bf16_nhwc", splits=[("pw", dict(parts_k=parts_k))])
+    L = gg.g.plan()["launches"][0]
+    assert gg.g.launch_count() == 1 and L["a0"] == "dw" and L["ksplit"] == parts_k
+    base, _, _ = check_bf16("dw_pw_splitk_base", spec, 3, linked=True, in_mode="bf16_nhwc", splits=[("pw", dict(parts_k=1))])
+    assert abs_err_scaled(y, base) <= 2.0 ** -8
+    x = xo.round_bf16(graphs.make_input(spec, 3))
+    assert np.array_equal(gg.run(x), y)
+
+
 def test_bf16_shortcut_block_with_reduction_split():
     def build(g):
         y = g.cbr("c1", "input", 64, 3, 1, 1)

@@ -327,8 +327,11 @@ def test_reduction_split_requests_that_cannot_be_met():
         assert e.value.code == code, pk
     m = graphs.mobilenet_v1(hw=32, width=0.25, classes=8)
     with pytest.raises(xb.XenosError) as e:
-        compiled(m, 1, splits=[("pw1.relu6", dict(parts_k=2))])        # linked depthwise stage
+        compiled(m, 1, splits=[("stem.relu6", dict(parts_k=2))])       # a convolution that reads the image
     assert e.value.code == xb.E_UNSUPPORTED
+    with pytest.raises(xb.XenosError) as e:
+        compiled(m, 1, splits=[("pw1.relu6", dict(parts_k=2))])        # depthwise -> pointwise with one K block
+    assert e.value.code == xb.E_BAD_SPLIT
     with pytest.raises(xb.XenosError) as e:
         compiled(graphs.single_chain(), 1, splits=[("mp", dict(parts_k=2))])     # fp32 CUDA-core chain
     assert e.value.code == xb.E_UNSUPPORTED
@@ -341,6 +344,11 @@ def test_reduction_split_is_automatic_only_where_units_would_idle():
     assert [l["ksplit"] for l in L[:-1]] == [1] * (len(L) - 1)
     fc = L[-1]
     assert fc["ksplit"] >= 2 and fc["m_tiles"] * fc["n_tiles"] * fc["ksplit"] <= 148 and fc["kb_per"] >= 2
+    # a depthwise -> pointwise chain is cut on request only
+    g1, ids = compiled(spec, 1, splits=[("pw7.relu6", dict(parts_k=8))])
+    L1 = g1.plan()["launches"]
+    assert [l["ksplit"] for l in L1 if l.get("a0") == "dw"].count(8) == 1
+    assert all(l["ksplit"] == 1 for l in L1 if l.get("a0") == "stem" or l.get("epi") in (1, 2))
 
 
 def test_user_outc_split_sets_tiles():
