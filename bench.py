@@ -30,6 +30,7 @@ WORKLOADS = {
     "resnet18_b32": (2, 32), "resnet18_b1": (2, 1),
     "squeezenet11_b32": (3, 32), "squeezenet11_b1": (3, 1),
     "resnet50_stress_b64": (4, 64), "single_chain_b1": (0, 1),
+    "resnet50_stress_b8": (4, 8),       # the stress graph at a batch small enough for a profiler capture
     # the paper's operator micro-benchmarks (Table 4): the first two exercise linking (other arm: unlinked), the
     # last two the split (other arm: the coarsest split the kernels allow, 256-wide channel tiles, K uncut)
     "op_cbr_maxpool_b32": ("cbr_maxpool", 32), "op_cbr_avgpool_b32": ("cbr_avgpool", 32),

@@ -58,8 +58,9 @@ enum {
     XENOS_E_BOUNDS = -10        /* a device-side index check failed (status word set)            */
 };
 
-/* Operator kinds: the Table 3 operators the CNN workloads use.  x.mul, x.mac, x.transpose,
- * x.split and general x.matmul are not implemented and yield XENOS_E_UNSUPPORTED. */
+/* Operator kinds: the operators of Table 3.  A matrix is a feature map of width 1: h rows of c columns per
+ * image (in memory [batch][h][c], the NHWC layout of such a map).  x.matmul takes a constant right operand; a
+ * product of two run-time tensors is not implemented (XENOS_E_UNSUPPORTED). */
 enum {
     XENOS_OP_CONV = 1,            /* x.conv; groups == 1 dense, groups == Cin == Cout depthwise      */
     XENOS_OP_FC = 2,              /* x.matmul as y = W x + B (Eq. 1); input is a [C] vector per image */
@@ -70,7 +71,16 @@ enum {
     XENOS_OP_CONCAT = 7,          /* x.concat along channels, inputs in argument order               */
     XENOS_OP_RELU = 8,
     XENOS_OP_RELU6 = 9,
-    XENOS_OP_BATCHNORM = 10       /* inference form: gamma * (x - mean) / sqrt(var + eps) + beta      */
+    XENOS_OP_BATCHNORM = 10,      /* inference form: gamma * (x - mean) / sqrt(var + eps) + beta      */
+    XENOS_OP_MUL = 11,            /* x.mul: element-wise product of two inputs of equal shape          */
+    XENOS_OP_MAC = 12,            /* x.mac: three inputs of equal shape, a * b + c element-wise (product rounded, then sum) */
+    XENOS_OP_TRANSPOSE = 13,      /* x.transpose of a matrix: (c, h, 1) -> (h, c, 1), y[r][q] = x[q][r] */
+    XENOS_OP_SPLIT = 14,          /* x.split, one part per call: channels [pad, pad + cout) of the input */
+    XENOS_OP_MATMUL = 15          /* x.matmul: A (h rows x c columns, or a vector) times the constant matrix
+                                     `weight` = B [c][cout] row-major, plus `bias` [cout] if given; the
+                                     result has cout columns.  MatmulX -> MatmulY (Table 1): two such products
+                                     with no activation between them are linked by multiplying the constants
+                                     when that does not add work */
 };
 
 enum { XENOS_ACT_NONE = 0, XENOS_ACT_RELU = 1, XENOS_ACT_RELU6 = 2 };

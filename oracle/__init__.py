@@ -148,6 +148,54 @@ def concat(xs):
     return y
 
 
+def mul(a, b):
+    a, b = _c(a), _c(b)
+    assert a.shape == b.shape
+    y = np.empty_like(a)
+    lib().xo_mul(_p(a), _p(b), ctypes.c_size_t(a.size), _p(y))
+    return y
+
+
+def mac(a, b, c):
+    a, b, c = _c(a), _c(b), _c(c)
+    assert a.shape == b.shape == c.shape
+    y = np.empty_like(a)
+    lib().xo_mac(_p(a), _p(b), _p(c), ctypes.c_size_t(a.size), _p(y))
+    return y
+
+
+def transpose(x):
+    """Matrix transpose per image: (N, C, H, 1) -> (N, H, C, 1)."""
+    x = _c(x)
+    N, C, H, W = x.shape
+    assert W == 1
+    y = np.empty((N, H, C, 1), np.float32)
+    lib().xo_transpose(_p(x), N, C, H, _p(y))
+    return y
+
+
+def split_part(x, first, count):
+    x = _c(x)
+    N, C, H, W = x.shape
+    assert 0 <= first and first + count <= C
+    y = np.empty((N, count, H, W), np.float32)
+    lib().xo_split_part(_p(x), N, count, H * W, C, first, _p(y))
+    return y
+
+
+def matmul(a, b, bias=None):
+    """a: (N, K, R, 1) matrix per image (R rows of K columns) or (N, K) vectors; b: (K, M) constant."""
+    a, b, bias = _c(a), _c(b), _c(bias)
+    vec = a.ndim == 2
+    N, K = a.shape[0], a.shape[1]
+    R = 1 if vec else a.shape[2]
+    assert b.shape[0] == K and (vec or a.shape[3] == 1)
+    M = b.shape[1]
+    y = np.empty((N, M) if vec else (N, M, R, 1), np.float32)
+    lib().xo_matmul(_p(a), N, K, R, _p(b), M, _p(bias), _p(y))
+    return y
+
+
 def fc(x, w, bias=None):
     x, w, bias = _c(x), _c(w), _c(bias)
     N, C = x.shape

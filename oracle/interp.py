@@ -44,6 +44,16 @@ def run_graph(spec, params, x: np.ndarray, keep: bool = False, bf16_emulate: boo
             y = xo.concat(ins)
         elif k == "fc":
             y = xo.fc(ins[0], p["w"], p.get("b"))
+        elif k == "mul":
+            y = xo.mul(ins[0], ins[1])
+        elif k == "mac":
+            y = xo.mac(ins[0], ins[1], ins[2])
+        elif k == "transpose":
+            y = xo.transpose(ins[0])
+        elif k == "split":
+            y = xo.split_part(ins[0], o["first"], o["cout"])
+        elif k == "matmul":
+            y = xo.matmul(ins[0], p["w"], p.get("b"))
         else:
             raise ValueError(k)
         # BatchNorm and activation follow their conv inside one fused operator on the device,

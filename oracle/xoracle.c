@@ -229,6 +229,55 @@ XO_API void xo_fc(const float *x, int N, int C, const float *w, int K, const flo
     }
 }
 
+/* x.mul (Table 3): element-wise a * b. */
+XO_API void xo_mul(const float *a, const float *b, size_t n, float *y) {
+#pragma omp parallel for schedule(static)
+    for (size_t i = 0; i < n; ++i) y[i] = a[i] * b[i];
+}
+
+/* x.mac (Table 3): element-wise multiply accumulate, a * b + c; the product is a rounded fp32 value. */
+XO_API void xo_mac(const float *a, const float *b, const float *c, size_t n, float *y) {
+#pragma omp parallel for schedule(static)
+    for (size_t i = 0; i < n; ++i) {
+        float p = a[i] * b[i];
+        y[i] = p + c[i];
+    }
+}
+
+/*
+ * x.transpose (Table 3) of one matrix per image.  A matrix is a feature map of width 1, rows = H, columns = C,
+ * stored NCHW as x[n][c][h]; the result has rows = C, columns = H: y[n][h][c] = x[n][c][h].
+ */
+XO_API void xo_transpose(const float *x, int N, int C, int H, float *y) {
+    for (int n = 0; n < N; ++n)
+        for (int c = 0; c < C; ++c)
+            for (int h = 0; h < H; ++h) y[((size_t)n * H + h) * C + c] = x[((size_t)n * C + c) * H + h];
+}
+
+/* x.split (Table 3), one part: channels [coff, coff + Ci) of an input with Ctot channels. */
+XO_API void xo_split_part(const float *x, int N, int Ci, int HW, int Ctot, int coff, float *y) {
+    for (int n = 0; n < N; ++n)
+        memcpy(y + (size_t)n * Ci * HW, x + ((size_t)n * Ctot + coff) * HW, (size_t)Ci * HW * sizeof(float));
+}
+
+/*
+ * x.matmul (Table 3): A * B (+ bias) per image.  A has R rows of K columns and is stored as the feature map
+ * a[n][k][r] (channels = columns); B is the constant [K][M] matrix, row-major; y[n][m][r] = sum_k a[n][k][r] * B[k][m].
+ */
+XO_API void xo_matmul(const float *a, int N, int K, int R, const float *b, int M, const float *bias, float *y) {
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int n = 0; n < N; ++n) {
+        for (int m = 0; m < M; ++m) {
+            for (int r = 0; r < R; ++r) {
+                float acc = 0.0f;
+                for (int k = 0; k < K; ++k) acc += a[((size_t)n * K + k) * R + r] * b[(size_t)k * M + m];
+                if (bias) acc += bias[m];
+                y[((size_t)n * M + m) * R + r] = acc;
+            }
+        }
+    }
+}
+
 /*
  * Diagnostic only: round an fp32 array to the nearest bf16 value (ties to even), kept in
  * fp32.  Lets a test separate precision drift of a bf16 execution from an indexing bug.

@@ -20,6 +20,7 @@ E_INVALID, E_SHAPE, E_UNSUPPORTED, E_NOT_LINKABLE, E_BAD_SPLIT = -1, -2, -3, -4,
 E_STATE, E_WORKSPACE, E_CUDA, E_TIMEOUT, E_BOUNDS = -6, -7, -8, -9, -10
 OP_CONV, OP_FC, OP_POOL_MAX, OP_POOL_AVG, OP_POOL_GLOBAL_AVG = 1, 2, 3, 4, 5
 OP_ADD, OP_CONCAT, OP_RELU, OP_RELU6, OP_BATCHNORM = 6, 7, 8, 9, 10
+OP_MUL, OP_MAC, OP_TRANSPOSE, OP_SPLIT, OP_MATMUL = 11, 12, 13, 14, 15
 ACT_NONE, ACT_RELU, ACT_RELU6 = 0, 1, 2
 DTYPE_F32, DTYPE_BF16 = 0, 1
 LAYOUT_NCHW, LAYOUT_NHWC = 0, 1

@@ -110,13 +110,51 @@ xenos_status_t infer_and_append(Graph &g, const xenos_op_desc_t &d, const int *i
         if (!has_bn) return fail(g, XENOS_E_INVALID, "batchnorm: parameters are NULL");
         y.c = x.c; y.h = x.h; y.w = x.w; y.is_vec = x.is_vec;
         break;
+    case XENOS_OP_MUL:
+    case XENOS_OP_MAC: {
+        const int need = d.kind == XENOS_OP_MUL ? 2 : 3;
+        if (!need_inputs(need)) return fail(g, XENOS_E_INVALID, d.kind == XENOS_OP_MUL ? "mul takes two inputs" : "mac takes three inputs");
+        for (int i = 1; i < need; ++i) {
+            const Tensor &b = g.tensors[in[i]];
+            if (x.c != b.c || x.h != b.h || x.w != b.w || x.is_vec != b.is_vec)
+                return fail(g, XENOS_E_SHAPE, "mul / mac: operand shapes differ");
+        }
+        y.c = x.c; y.h = x.h; y.w = x.w; y.is_vec = x.is_vec;
+        break;
+    }
+    case XENOS_OP_TRANSPOSE:
+        if (!need_inputs(1)) return fail(g, XENOS_E_INVALID, "transpose takes one input");
+        if (x.is_vec || x.w != 1) return fail(g, XENOS_E_SHAPE, "transpose input must be a matrix (a feature map of width 1)");
+        y.c = x.h; y.h = x.c; y.w = 1;
+        break;
+    case XENOS_OP_SPLIT:
+        if (!need_inputs(1)) return fail(g, XENOS_E_INVALID, "split takes one input");
+        if (x.is_vec) return fail(g, XENOS_E_SHAPE, "split input must be a feature map");
+        if (d.cout < 1 || d.pad < 0 || d.pad + d.cout > x.c) return fail(g, XENOS_E_SHAPE, "split: channels [pad, pad + cout) leave the input");
+        y.c = d.cout; y.h = x.h; y.w = x.w;
+        op.cout = d.cout; op.pad = d.pad;
+        break;
+    case XENOS_OP_MATMUL: {
+        if (n_in == 2) return fail(g, XENOS_E_UNSUPPORTED, "matmul of two run-time tensors is not implemented; the right operand is a constant (weight)");
+        if (!need_inputs(1)) return fail(g, XENOS_E_INVALID, "matmul takes one input and a constant matrix");
+        if (!x.is_vec && x.w != 1) return fail(g, XENOS_E_SHAPE, "matmul input must be a matrix (a feature map of width 1) or a vector");
+        if (!d.weight || d.cout < 1) return fail(g, XENOS_E_INVALID, "matmul: weight is NULL or cout < 1");
+        size_t nw = (size_t)x.c * d.cout;
+        if (!finite_all(d.weight, nw)) return fail(g, XENOS_E_INVALID, "matmul: non-finite weight");
+        // kept as [cout][c], the form of a pointwise convolution / fc
+        op.w.resize(nw);
+        for (int k = 0; k < x.c; ++k)
+            for (int n = 0; n < d.cout; ++n) op.w[(size_t)n * x.c + k] = d.weight[(size_t)k * d.cout + n];
+        op.cout = d.cout; op.k = 1; op.groups = 1;
+        y.c = d.cout; y.h = x.h; y.w = x.w; y.is_vec = x.is_vec;
+        break;
+    }
     default:
-        return fail(g, XENOS_E_UNSUPPORTED,
-                    "add_op: operator kind not implemented (x.mul, x.mac, x.transpose, x.split, general x.matmul)");
+        return fail(g, XENOS_E_UNSUPPORTED, "add_op: unknown operator kind");
     }
 
     int cpar = (d.kind == XENOS_OP_BATCHNORM) ? x.c : d.cout;
-    if (d.kind == XENOS_OP_CONV || d.kind == XENOS_OP_FC) {
+    if (d.kind == XENOS_OP_CONV || d.kind == XENOS_OP_FC || d.kind == XENOS_OP_MATMUL) {
         op.act = d.act;
         if (d.bias) {
             if (!finite_all(d.bias, d.cout)) return fail(g, XENOS_E_INVALID, "non-finite bias");
@@ -129,7 +167,7 @@ xenos_status_t infer_and_append(Graph &g, const xenos_op_desc_t &d, const int *i
         op.act = d.act;
     }
     if (has_bn) {
-        if (d.kind != XENOS_OP_CONV && d.kind != XENOS_OP_FC && d.kind != XENOS_OP_BATCHNORM)
+        if (d.kind != XENOS_OP_CONV && d.kind != XENOS_OP_FC && d.kind != XENOS_OP_MATMUL && d.kind != XENOS_OP_BATCHNORM)
             return fail(g, XENOS_E_INVALID, "add_op: BatchNorm parameters on an operator that cannot carry them");
         if (!(d.bn_eps > 0.0f)) return fail(g, XENOS_E_INVALID, "batchnorm: eps must be positive");
         if (!finite_all(d.bn_gamma, cpar) || !finite_all(d.bn_beta, cpar) || !finite_all(d.bn_mean, cpar) ||

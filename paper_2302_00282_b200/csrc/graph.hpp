@@ -37,7 +37,7 @@ struct Op {
 };
 
 // ---- fused operators (after the CBR pre-fusion) ----------------------------------------------
-enum NodeKind { NK_CONV = 1, NK_DW, NK_FC, NK_MAXPOOL, NK_AVGPOOL, NK_GAP, NK_ADD, NK_CONCAT };
+enum NodeKind { NK_CONV = 1, NK_DW, NK_FC, NK_MAXPOOL, NK_AVGPOOL, NK_GAP, NK_ADD, NK_CONCAT, NK_MUL, NK_MAC, NK_TRANSPOSE, NK_SLICE };
 
 struct Node {
     int kind = 0;
@@ -48,6 +48,7 @@ struct Node {
     std::vector<float> b;         // folded bias [cout] (zeros when the op had none)
     std::vector<int> user_ops;    // indices of the user ops folded into this node
     int chain = -1;
+    bool from_matmul = false;     // an x.matmul with a constant right operand (lowered like a pointwise conv / fc)
 };
 
 // ---- chains (after linking) -------------------------------------------------------------------
@@ -56,7 +57,8 @@ enum ChainKind {
     CK_CONV_CONV_POOL,      // fp32: ConvX -> Conv1x1 -> ZPooling in one CUDA-core kernel
     CK_DW_PW,               // depthwise 3x3 -> pointwise [-> global avgpool]
     CK_CONV_TAIL,           // conv [+ linked shortcut conv] [-> add -> relu] [-> max pool | global avgpool]
-    CK_EXPAND_CONCAT        // {conv1x1, conv3x3} on one input -> concat [-> max pool]
+    CK_EXPAND_CONCAT,       // {conv1x1, conv3x3} on one input -> concat [-> max pool]
+    CK_MATMUL_MATMUL        // MatmulX -> MatmulY with constant right operands: one product with the constants multiplied
 };
 
 struct SplitRequest { int outc = 0, h = 0, w = 0, k = 1; bool user = false; };
@@ -87,9 +89,13 @@ enum LaunchKind {
     LK_GAP,               // standalone global average (bf16 NHWC -> vector)
     LK_ADD,               // standalone add (+ relu)
     LK_CONCAT_PART,       // copy one concat input to its channel offset
+    LK_MULMAC,            // element-wise product / multiply-accumulate (bf16 NHWC)
+    LK_TRANSPOSE,         // matrix transpose per image (bf16)
+    LK_SLICE,             // channels [coff, coff + C) of the input (bf16 NHWC)
     LK_F32_CONV,          // fp32 NCHW direct conv (+bias, act), any k / stride / pad, dense or depthwise
     LK_F32_POOL, LK_F32_GAP, LK_F32_ADD, LK_F32_CONCAT_PART, LK_F32_FC,
-    LK_F32_CONV_CONV_POOL // fp32 linked chain
+    LK_F32_CONV_CONV_POOL, // fp32 linked chain
+    LK_F32_MULMAC, LK_F32_TRANSPOSE, LK_F32_SLICE
 };
 
 struct Launch {
@@ -97,7 +103,7 @@ struct Launch {
     int chain = -1;
     std::vector<int> nodes;       // node indices covered
     // ---- common tensor plumbing
-    int in0 = -1, in1 = -1;       // input tensors (in1: second operand of add)
+    int in0 = -1, in1 = -1, in2 = -1;   // input tensors (in1: second operand of add / mul / mac, in2: addend of mac)
     int out = -1;                 // output tensor
     int out_coff = 0, out_ctot = 0;   // channel offset / total channels of the stored tensor
     int act = 0;

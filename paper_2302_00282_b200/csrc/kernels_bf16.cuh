@@ -151,6 +151,54 @@ __global__ void add_kernel(const __nv_bfloat16 *__restrict__ a, const __nv_bfloa
     }
 }
 
+// x.mul (c == nullptr): a * b; x.mac: a * b + c.  The product is rounded to fp32 before the sum (no fused
+// multiply-add), as the operator-at-a-time definition has it.
+__global__ void mulmac_kernel(const __nv_bfloat16 *__restrict__ a, const __nv_bfloat16 *__restrict__ b,
+                              const __nv_bfloat16 *__restrict__ c, __nv_bfloat16 *__restrict__ y, long long n8) {
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n8; i += (long long)gridDim.x * blockDim.x) {
+        f8 av = unpack8(reinterpret_cast<const uint4 *>(a)[i]);
+        const f8 bv = unpack8(reinterpret_cast<const uint4 *>(b)[i]);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) av.v[j] = __fmul_rn(av.v[j], bv.v[j]);
+        if (c) {
+            const f8 cv = unpack8(reinterpret_cast<const uint4 *>(c)[i]);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) av.v[j] = __fadd_rn(av.v[j], cv.v[j]);
+        }
+        reinterpret_cast<uint4 *>(y)[i] = pack8(av);
+    }
+}
+
+// x.transpose: per image x [R][Cc] -> y [Cc][R], through a padded 32 x 32 tile so that reads and writes are coalesced.
+template <typename T>
+__global__ void transpose_kernel(const T *__restrict__ x, T *__restrict__ y, int R, int Cc) {
+    __shared__ T tile[32][33];
+    const size_t img = (size_t)blockIdx.z * R * Cc;
+    const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+    for (int j = threadIdx.y; j < 32; j += blockDim.y) {
+        const int r = r0 + j, c = c0 + threadIdx.x;
+        if (r < R && c < Cc) tile[j][threadIdx.x] = x[img + (size_t)r * Cc + c];
+    }
+    __syncthreads();
+    for (int j = threadIdx.y; j < 32; j += blockDim.y) {
+        const int c = c0 + j, r = r0 + threadIdx.x;
+        if (r < R && c < Cc) y[img + (size_t)c * R + r] = tile[threadIdx.x][j];
+    }
+}
+
+// x.split, one part: y [pixels][Ci] = x [pixels][Ctot] at channel offset coff.
+__global__ void slice_kernel(const __nv_bfloat16 *__restrict__ x, __nv_bfloat16 *__restrict__ y,
+                             long long pixels, int Ci, int Ctot, int coff) {
+    int C8 = Ci >> 3;
+    long long total = pixels * C8;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        long long px = i / C8;
+        int c0 = (int)(i % C8) * 8;
+        *reinterpret_cast<uint4 *>(y + px * Ci + c0) = *reinterpret_cast<const uint4 *>(x + px * Ctot + coff + c0);
+    }
+}
+
 // One concat input: x [pixels][Ci] -> y [pixels][Ctot] at channel offset coff.
 __global__ void concat_part_kernel(const __nv_bfloat16 *__restrict__ x, __nv_bfloat16 *__restrict__ y,
                                    long long pixels, int Ci, int Ctot, int coff) {

@@ -93,6 +93,26 @@ __global__ void f32_add_kernel(const float *__restrict__ a, const float *__restr
         y[i] = apply_act(a[i] + b[i], act);
 }
 
+// x.mul (c == nullptr) / x.mac: the product is rounded before the sum (no fused multiply-add).
+__global__ void f32_mulmac_kernel(const float *__restrict__ a, const float *__restrict__ b, const float *__restrict__ c,
+                                  float *__restrict__ y, long long n) {
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+        const float p = __fmul_rn(a[i], b[i]);
+        y[i] = c ? __fadd_rn(p, c[i]) : p;
+    }
+}
+
+// x.split, one part: y [N][Ci][HW] = x [N][Ctot][HW] at channel offset coff.
+__global__ void f32_slice_kernel(const float *__restrict__ x, float *__restrict__ y, int N, int Ci, int HW,
+                                 int Ctot, int coff) {
+    long long per = (long long)Ci * HW, total = (long long)N * per;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        long long n = i / per, r = i % per;
+        y[i] = x[(n * Ctot + coff) * HW + r];
+    }
+}
+
 // One concat input: x [N][Ci][HW] -> y [N][Ctot][HW] at channel offset coff.
 __global__ void f32_concat_part_kernel(const float *__restrict__ x, float *__restrict__ y, int N, int Ci, int HW,
                                        int Ctot, int coff) {

@@ -48,9 +48,11 @@ xenos_status_t prefuse(Graph &g) {
         int src = g.node_of_tensor[op.in[0]];
         switch (op.kind) {
         case XENOS_OP_CONV:
-        case XENOS_OP_FC: {
+        case XENOS_OP_FC:
+        case XENOS_OP_MATMUL: {
             Node n;
             n.kind = op.kind == XENOS_OP_FC ? NK_FC : (op.groups == 1 ? NK_CONV : NK_DW);
+            if (op.kind == XENOS_OP_MATMUL) { n.kind = x.is_vec ? NK_FC : NK_CONV; n.from_matmul = true; }
             n.in = op.in; n.out = op.out;
             n.cin = x.c; n.cout = op.cout; n.k = op.k; n.stride = op.stride; n.pad = op.pad; n.act = op.act;
             n.w = op.w;
@@ -93,7 +95,9 @@ xenos_status_t prefuse(Graph &g) {
         default: {
             Node n;
             n.kind = op.kind == XENOS_OP_POOL_MAX ? NK_MAXPOOL : op.kind == XENOS_OP_POOL_AVG ? NK_AVGPOOL
-                   : op.kind == XENOS_OP_POOL_GLOBAL_AVG ? NK_GAP : op.kind == XENOS_OP_ADD ? NK_ADD : NK_CONCAT;
+                   : op.kind == XENOS_OP_POOL_GLOBAL_AVG ? NK_GAP : op.kind == XENOS_OP_ADD ? NK_ADD
+                   : op.kind == XENOS_OP_MUL ? NK_MUL : op.kind == XENOS_OP_MAC ? NK_MAC
+                   : op.kind == XENOS_OP_TRANSPOSE ? NK_TRANSPOSE : op.kind == XENOS_OP_SPLIT ? NK_SLICE : NK_CONCAT;
             n.in = op.in; n.out = op.out;
             n.cin = x.c; n.cout = g.tensors[op.out].c; n.k = op.k; n.stride = op.stride; n.pad = op.pad; n.act = op.act;
             n.user_ops.push_back(oi);
@@ -170,6 +174,19 @@ static bool try_match(const LinkCtx &cx, int a, Allowed allowed, Chain &out) {
         return true;
     }
     // ---- bf16 tensor-core chains -----------------------------------------------------------
+    if (A.from_matmul) {
+        // MatmulX -> MatmulY (last row of Table 1) with constant right operands and nothing but a bias between
+        // them: (X B1 + b1) B2 + b2 = X (B1 B2) + (b1 B2 + b2).  The constants are multiplied once at compile time
+        // and the intermediate matrix never exists.  Taken only when it does not add multiplications per row.
+        int b = A.act == XENOS_ACT_NONE ? cx.sole(a) : -1;
+        if (b >= 0 && allowed(b) && g.nodes[b].from_matmul && g.nodes[b].kind == A.kind && A.cin % 8 == 0 &&
+            (long)A.cin * g.nodes[b].cout <= (long)A.cin * A.cout + (long)A.cout * g.nodes[b].cout) {
+            out.kind = CK_MATMUL_MATMUL;
+            out.nodes = {a, b};
+            out.pattern = "MatmulX -> MatmulY (MatA * MatB -> MatC * MatD, constants multiplied)";
+            return true;
+        }
+    }
     if (A.kind == NK_DW) {
         // depthwise -> pointwise: the motivating mismatch of Section 2.2 (ConvX -> ConvY row)
         if (A.k != 3 || A.cin % 8 || A.stride > 2) return false;
@@ -427,6 +444,21 @@ struct Lower {
         case NK_ADD:
             L.kind = f32 ? LK_F32_ADD : LK_ADD;
             L.in1 = n.in[1];
+            break;
+        case NK_MUL:
+        case NK_MAC:
+            L.kind = f32 ? LK_F32_MULMAC : LK_MULMAC;
+            L.in1 = n.in[1];
+            if (n.kind == NK_MAC) L.in2 = n.in[2];
+            break;
+        case NK_TRANSPOSE:
+            L.kind = f32 ? LK_F32_TRANSPOSE : LK_TRANSPOSE;
+            if (!f32 && (L.C % 8 || L.H % 8)) return fail(g, XENOS_E_UNSUPPORTED, "bf16 transpose needs row and column counts that are multiples of 8");
+            break;
+        case NK_SLICE:
+            L.kind = f32 ? LK_F32_SLICE : LK_SLICE;
+            L.out_coff = n.pad;             // first channel of the part
+            if (!f32 && (n.pad % 8 || n.cout % 8)) return fail(g, XENOS_E_UNSUPPORTED, "bf16 split needs channel offsets and counts that are multiples of 8");
             break;
         case NK_CONCAT: {
             int off = 0;
@@ -906,6 +938,29 @@ struct Lower {
             st = make_gemm(ci, ch.nodes, nullptr, mainc, sc, nullptr, addn, find(NK_MAXPOOL), find(NK_GAP), nullptr, false);
             break;
         }
+        case CK_MATMUL_MATMUL: {
+            const Node &A = g.nodes[ch.nodes[0]], &B = g.nodes[ch.nodes[1]];
+            Node M;                      // the one product that stands for both
+            M.kind = A.kind; M.in = A.in; M.out = B.out; M.cin = A.cin; M.cout = B.cout; M.k = 1; M.stride = 1; M.pad = 0; M.act = B.act;
+            M.w.assign((size_t)B.cout * A.cin, 0.0f);
+            M.b.assign(B.cout, 0.0f);
+            for (int o = 0; o < B.cout; ++o) {
+                std::vector<double> row(A.cin, 0.0);
+                double bias = B.b[o];
+                for (int m = 0; m < A.cout; ++m) {
+                    const double w2 = B.w[(size_t)o * A.cout + m];
+                    bias += w2 * A.b[m];
+                    const float *w1 = &A.w[(size_t)m * A.cin];
+                    for (int c = 0; c < A.cin; ++c) row[c] += w2 * w1[c];
+                }
+                for (int c = 0; c < A.cin; ++c) M.w[(size_t)o * A.cin + c] = (float)row[c];
+                M.b[o] = (float)bias;
+            }
+            st = make_gemm(ci, ch.nodes, nullptr, &M, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, A.kind == NK_FC);
+            // (the modelled work of the launch is the merged product's, not the sum of the two it replaces)
+            if (st == XENOS_OK) g.launches.back().flops = 2.0 * node_macs(M);
+            break;
+        }
         case CK_EXPAND_CONCAT: {
             const Node *cat = find(NK_CONCAT);
             const Node *first = &g.nodes[g.node_of_tensor[cat->in[0]]];
@@ -951,7 +1006,7 @@ xenos_status_t plan_workspace(Graph &g) {
     for (int li = 0; li < (int)g.launches.size(); ++li) {
         const Launch &L = g.launches[li];
         touch(L.out, li, true);
-        touch(L.in0, li, false); touch(L.in1, li, false); touch(L.skip, li, false);
+        touch(L.in0, li, false); touch(L.in1, li, false); touch(L.in2, li, false); touch(L.skip, li, false);
         touch(L.seg[0].tensor, li, false); touch(L.seg[1].tensor, li, false);
     }
     size_t off = align_up(g.param_blob.size(), 256);
@@ -1026,10 +1081,10 @@ static void jarr(std::string &s, const char *k, const std::vector<int> &v, bool 
 }
 
 void emit_plan_json(Graph &g) {
-    static const char *nk[] = {"?", "conv", "dwconv", "fc", "maxpool", "avgpool", "gap", "add", "concat"};
-    static const char *ck[] = {"single", "conv_conv_pool", "dw_pw", "conv_tail", "expand_concat"};
-    static const char *lk[] = {"?", "gemm", "dw", "pool", "gap", "add", "concat_part", "f32_conv", "f32_pool",
-                               "f32_gap", "f32_add", "f32_concat_part", "f32_fc", "f32_conv_conv_pool"};
+    static const char *nk[] = {"?", "conv", "dwconv", "fc", "maxpool", "avgpool", "gap", "add", "concat", "mul", "mac", "transpose", "split"};
+    static const char *ck[] = {"single", "conv_conv_pool", "dw_pw", "conv_tail", "expand_concat", "matmul_matmul"};
+    static const char *lk[] = {"?", "gemm", "dw", "pool", "gap", "add", "concat_part", "mulmac", "transpose", "slice", "f32_conv", "f32_pool",
+                               "f32_gap", "f32_add", "f32_concat_part", "f32_fc", "f32_conv_conv_pool", "f32_mulmac", "f32_transpose", "f32_slice"};
     static const char *am[] = {"none", "gather", "stem", "dw"};
     std::string s = "{";
     jstr(s, "precision", g.precision == XENOS_PRECISION_FP32_CUDA_CORE ? "fp32_cuda_core" : "bf16_tensor");
@@ -1068,7 +1123,7 @@ void emit_plan_json(Graph &g) {
         if (i) s += ",";
         s += "{";
         jint(s, "id", (long long)i); jstr(s, "kind", lk[L.kind]); jint(s, "chain", L.chain); jarr(s, "nodes", L.nodes);
-        jint(s, "in0", L.in0); jint(s, "in1", L.in1); jint(s, "skip", L.skip); jint(s, "out", L.out);
+        jint(s, "in0", L.in0); jint(s, "in1", L.in1); jint(s, "in2", L.in2); jint(s, "skip", L.skip); jint(s, "out", L.out);
         jint(s, "out_coff", L.out_coff); jint(s, "out_ctot", L.out_ctot);
         jint(s, "C", L.C); jint(s, "H", L.H); jint(s, "W", L.W); jint(s, "K", L.K); jint(s, "P", L.P); jint(s, "Q", L.Q);
         jint(s, "k", L.k); jint(s, "stride", L.stride); jint(s, "pad", L.pad);

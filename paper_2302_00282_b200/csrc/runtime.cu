@@ -265,6 +265,38 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
             xk::concat_part_kernel<<<ew_grid(pixels * (L.C / 8), 256, sms), 256, 0, stream>>>((const __nv_bfloat16 *)ptr(L.in0), (__nv_bfloat16 *)ptr(L.out), pixels, L.C, L.out_ctot, L.out_coff);
             break;
         }
+        case LK_MULMAC: {
+            const Tensor &t = g.tensors[L.out];
+            long long n8 = (long long)N * (t.is_vec ? t.c : t.c * t.h * t.w) / 8;
+            xk::mulmac_kernel<<<ew_grid(n8, 256, sms), 256, 0, stream>>>((const __nv_bfloat16 *)ptr(L.in0), (const __nv_bfloat16 *)ptr(L.in1),
+                                                                         (const __nv_bfloat16 *)ptr(L.in2), (__nv_bfloat16 *)ptr(L.out), n8);
+            break;
+        }
+        case LK_F32_MULMAC: {
+            const Tensor &t = g.tensors[L.out];
+            long long total = (long long)N * (t.is_vec ? t.c : t.c * t.h * t.w);
+            xk::f32_mulmac_kernel<<<ew_grid(total, 256, sms), 256, 0, stream>>>((const float *)ptr(L.in0), (const float *)ptr(L.in1),
+                                                                                (const float *)ptr(L.in2), (float *)ptr(L.out), total);
+            break;
+        }
+        case LK_TRANSPOSE:      // NHWC: per image [H rows][C columns] -> [C][H]
+            xk::transpose_kernel<__nv_bfloat16><<<dim3((L.C + 31) / 32, (L.H + 31) / 32, N), dim3(32, 8), 0, stream>>>(
+                (const __nv_bfloat16 *)ptr(L.in0), (__nv_bfloat16 *)ptr(L.out), L.H, L.C);
+            break;
+        case LK_F32_TRANSPOSE:  // NCHW: per image [C][H] -> [H][C]
+            xk::transpose_kernel<float><<<dim3((L.H + 31) / 32, (L.C + 31) / 32, N), dim3(32, 8), 0, stream>>>(
+                (const float *)ptr(L.in0), (float *)ptr(L.out), L.C, L.H);
+            break;
+        case LK_SLICE: {
+            long long pixels = (long long)N * L.H * L.W;
+            xk::slice_kernel<<<ew_grid(pixels * (L.K / 8), 256, sms), 256, 0, stream>>>((const __nv_bfloat16 *)ptr(L.in0), (__nv_bfloat16 *)ptr(L.out), pixels, L.K, L.C, L.out_coff);
+            break;
+        }
+        case LK_F32_SLICE: {
+            long long total = (long long)N * L.K * L.H * L.W;
+            xk::f32_slice_kernel<<<ew_grid(total, 256, sms), 256, 0, stream>>>((const float *)ptr(L.in0), (float *)ptr(L.out), N, L.K, L.H * L.W, L.C, L.out_coff);
+            break;
+        }
         case LK_GEMM: {
             xk::GemmParams p;
             std::memset(&p, 0, sizeof p);

@@ -486,6 +486,51 @@ def test_bf16_operator_benchmarks(name, batch, launches, linked):
         assert gg.g.launch_count() == launches
 
 
+# ---- the remaining operators of Table 3 and the MatmulX -> MatmulY link -----------------------------------
+def _matrix_ops_graph(precision):
+    g = GraphSpec("matrix", (64, 24, 1), precision=precision)
+    q = g.matmul("q", "input", 96, bias=True)
+    k = g.matmul("k", "input", 96)
+    lo = g.split("lo", q, 0, 32)
+    hi = g.split("hi", q, 64, 32)
+    mid = g.split("mid", k, 32, 32)
+    m = g.mul("m", lo, hi)
+    a = g.mac("a", m, mid, lo)
+    g.transpose("t", a)
+    return g
+
+
+def test_bf16_matrix_operators():
+    spec = _matrix_ops_graph("bf16")
+    y, o, gg = check_bf16("matrix_ops", spec, 3, linked=True, in_mode="bf16_nhwc")
+    kinds = [l["kind"] for l in gg.g.plan()["launches"]]
+    assert kinds.count("gemm") == 2 and kinds.count("slice") == 3 and kinds.count("mulmac") == 2 and kinds.count("transpose") == 1
+
+
+def test_fp32_matrix_operators():
+    spec = _matrix_ops_graph("fp32")
+    P = graphs.make_params(spec)
+    x = graphs.make_input(spec, 3)
+    gg = GpuGraph(spec, P, 3, linked=False)
+    err = rel_err_fp32(gg.run(x), interp.run_graph(spec, P, x))
+    assert err <= FP32_TOL
+
+
+@pytest.mark.parametrize("linked", [True, False])
+@pytest.mark.parametrize("vec", [False, True])
+def test_bf16_matmul_matmul(linked, vec):
+    """Two products with constant right operands: linked, the constants are multiplied at compile time and one GEMM
+    runs; unlinked, two GEMMs with a bf16 intermediate."""
+    g = GraphSpec("mm", (128, 20, 1))
+    a = "input"
+    if vec:
+        a = g.gap("flat", a)
+    a = g.matmul("m1", a, 192, bias=True)
+    g.matmul("m2", a, 72, bias=True)
+    y, o, gg = check_bf16(f"matmul_matmul_vec{vec}", g, 5, linked=linked, in_mode="bf16_nhwc")
+    assert [l["kind"] for l in gg.g.plan()["launches"]].count("gemm") == (1 if linked else 2)
+
+
 # ---- bf16: whole graphs ---------------------------------------------------------------------------
 @pytest.mark.parametrize("linked", [True, False])
 @pytest.mark.parametrize("name,kw", [("mobilenet_v1", dict(hw=64, width=0.25, classes=24)),

@@ -399,3 +399,58 @@ def test_modelled_work_matches_shapes():
     assert pl["flops"] == 2 * 32 * spec.macs()
     # depthwise-separable chains dominate the saving: linked bytes are well below unlinked ones
     assert pl["bytes_linked"] < 0.7 * pl["bytes_unlinked"]
+
+
+# ---- the remaining operators of Table 3 and the MatmulX -> MatmulY link ---------------------------------
+def _matrix_graph(act_between=None, n1=64, n2=32, bias=True):
+    g = GraphSpec("mm", (64, 16, 1))
+    a = g.matmul("m1", "input", n1, bias=bias)
+    if act_between:
+        a = g.act("m1." + act_between, a, act_between)
+    g.matmul("m2", a, n2, bias=bias)
+    return g
+
+
+def test_matmul_matmul_is_linked_by_multiplying_the_constants():
+    g, _ = compiled(_matrix_graph(), 4, nhwc=True)
+    pl = g.plan()
+    assert [c["kind"] for c in pl["chains"]] == ["matmul_matmul"] and len(pl["launches"]) == 1
+    assert "MatmulX -> MatmulY" in pl["chains"][0]["pattern"]
+    L = pl["launches"][0]
+    assert (L["C"], L["K"]) == (64, 32) and L["flops"] == 2 * 4 * 16 * 64 * 32
+    # an activation between the two products, or a merged product with more multiplications, is not linked
+    g2, _ = compiled(_matrix_graph(act_between="relu"), 4, nhwc=True)
+    assert len(g2.plan()["launches"]) == 2
+    g3, _ = compiled(_matrix_graph(n1=8, n2=256), 4, nhwc=True)          # 64 * 256 > 64 * 8 + 8 * 256
+    assert len(g3.plan()["launches"]) == 2
+    # unlinked: two launches
+    g4, _ = compiled(_matrix_graph(), 4, linked=False, nhwc=True)
+    assert len(g4.plan()["launches"]) == 2
+
+
+def test_matrix_operator_shapes_and_errors():
+    g = xb.Graph()
+    x = g.add_input(xb.DTYPE_BF16, xb.LAYOUT_NHWC, 16, 8, 1)
+    w = np.ones((16, 24), np.float32)
+    m = g.add_op(xb.OP_MATMUL, [x], cout=24, k=1, weight=w)
+    t = g.add_op(xb.OP_TRANSPOSE, [m])
+    s = g.add_op(xb.OP_SPLIT, [m], cout=8, pad=16)
+    g.add_op(xb.OP_MUL, [s, s])
+    g.add_op(xb.OP_MAC, [s, s, s])
+    for call, code in ((lambda: g.add_op(xb.OP_MATMUL, [x, m], cout=24, k=1, weight=w), xb.E_UNSUPPORTED),   # two run-time operands
+                       (lambda: g.add_op(xb.OP_SPLIT, [m], cout=16, pad=16), xb.E_SHAPE),                  # leaves the input
+                       (lambda: g.add_op(xb.OP_MUL, [s, m]), xb.E_SHAPE),
+                       (lambda: g.add_op(xb.OP_MAC, [s, s]), xb.E_INVALID),
+                       (lambda: g.add_op(xb.OP_MATMUL, [x], cout=24, k=1), xb.E_INVALID)):                  # no constant
+        with pytest.raises(xb.XenosError) as e:
+            call()
+        assert e.value.code == code
+    y = g.add_input(xb.DTYPE_BF16, xb.LAYOUT_NHWC, 16, 8, 2)
+    with pytest.raises(xb.XenosError) as e:
+        g.add_op(xb.OP_TRANSPOSE, [y])                       # width 2: not a matrix
+    assert e.value.code == xb.E_SHAPE
+    g.mark_output(t, xb.DTYPE_BF16, xb.LAYOUT_NHWC)
+    g.compile(2, xb.PRECISION_BF16_TENSOR)
+    pl = g.plan()
+    tt = [n for n in pl["nodes"] if n["kind"] == "transpose"][0]
+    assert tt["cin"] == 24 and tt["cout"] == 8               # (24 columns, 8 rows) -> (8 columns, 24 rows)

@@ -148,3 +148,25 @@ def test_avgpool_stage_of_the_tiled_chain_equals_the_plain_average_pool(tile):
     ref = xo.conv2d(xo.relu(xo.conv2d(x, w1, None, 1, 1, 1)), w2, b2, 1, 0, 1).astype(np.float64)
     ref = ref.reshape(2, 4, 7, 2, 7, 2).mean(axis=(3, 5))
     assert np.abs(plain - ref).max() <= 1e-6
+
+
+def test_matrix_operators_equal_hand_written_sequence():
+    """x.matmul (with and without bias), x.transpose, x.split, x.mul and x.mac walked by run_graph against the same
+    operators called by hand; the operands of mac and the parts of the split are all different."""
+    g = GraphSpec("matrix", (8, 6, 1), precision="fp32")
+    q = g.matmul("q", "input", 12, bias=True)
+    k = g.matmul("k", "input", 12)
+    lo = g.split("lo", q, 0, 4)
+    hi = g.split("hi", q, 8, 4)
+    mid = g.split("mid", k, 4, 4)
+    m = g.mul("m", lo, hi)
+    a = g.mac("a", m, mid, lo)
+    g.transpose("t", a)
+    P = graphs.make_params(g)
+    x = graphs.make_input(g, 3)
+    qv = xo.matmul(x, P["q"]["w"], P["q"]["b"])
+    kv = xo.matmul(x, P["k"]["w"], None)
+    lov, hiv, midv = xo.split_part(qv, 0, 4), xo.split_part(qv, 8, 4), xo.split_part(kv, 4, 4)
+    want = xo.transpose(xo.mac(xo.mul(lov, hiv), midv, lov))
+    got = interp.run_graph(g, P, x)
+    assert got.shape == (3, 6, 4, 1) and np.array_equal(got, want)

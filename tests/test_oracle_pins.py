@@ -287,3 +287,58 @@ def test_generator_is_deterministic_and_in_range():
     assert a.min() > -1 and a.max() < 1 and abs(a.mean()) < 0.1
     z = gen.normal(1, 5, (20000,), 0.0, 2.0)
     assert abs(z.mean()) < 0.06 and abs(z.std() - 2.0) < 0.06
+
+
+# ---- the remaining operators of Table 3: x.mul, x.mac, x.transpose, x.split, x.matmul ------------------
+def test_mul_and_mac_against_numpy_and_the_rounded_product():
+    a = gen.uniform(7, 1, (2, 3, 4, 5), -2.0, 2.0)
+    b = gen.uniform(7, 2, (2, 3, 4, 5), -2.0, 2.0)
+    c = gen.uniform(7, 3, (2, 3, 4, 5), -2.0, 2.0)
+    assert np.array_equal(xo.mul(a, b), a * b)
+    assert np.array_equal(xo.mac(a, b, c), (a * b).astype(np.float32) + c)
+    # the product is rounded before the sum: (1 + 2^-12)^2 = 1 + 2^-11 + 2^-24 rounds to 1 + 2^-11 (a tie, to even),
+    # so adding -(1 + 2^-11) gives exactly 0; a fused multiply-add would leave 2^-24
+    one = np.full((1, 1, 1, 1), 1.0 + 2.0 ** -12, np.float32)
+    neg = np.full((1, 1, 1, 1), -(1.0 + 2.0 ** -11), np.float32)
+    assert xo.mac(one, one, neg)[0, 0, 0, 0] == 0.0
+    # swapped roles change the result: a * c + b differs from a * b + c
+    assert not np.array_equal(xo.mac(a, b, c), xo.mac(a, c, b))
+
+
+def test_transpose_is_the_index_swap_and_an_involution():
+    N, C, H = 2, 5, 7
+    x = np.arange(N * C * H, dtype=np.float32).reshape(N, C, H, 1)
+    y = xo.transpose(x)
+    assert y.shape == (N, H, C, 1)
+    for n, c, h in itertools.product(range(N), range(C), range(H)):
+        assert y[n, h, c, 0] == x[n, c, h, 0]
+    assert np.array_equal(xo.transpose(y), x)
+
+
+def test_split_parts_are_slices_and_concat_restores_the_tensor():
+    x = np.arange(2 * 10 * 3 * 4, dtype=np.float32).reshape(2, 10, 3, 4)
+    parts = [(0, 3), (3, 5), (8, 2)]
+    ys = [xo.split_part(x, f, n) for f, n in parts]
+    for (f, n), y in zip(parts, ys):
+        assert np.array_equal(y, x[:, f:f + n])
+    assert np.array_equal(xo.concat(ys), x)
+
+
+def test_matmul_against_float64_identity_and_fc():
+    N, K, R, M = 2, 9, 6, 5
+    a = gen.uniform(11, 1, (N, K, R, 1), -1.0, 1.0)
+    b = gen.normal(11, 2, (K, M), 0.0, 0.5)
+    bias = gen.uniform(11, 3, (M,), -0.1, 0.1)
+    y = xo.matmul(a, b, bias)
+    ref = np.einsum("nkr,km->nmr", a[..., 0].astype(np.float64), b.astype(np.float64)) + bias.astype(np.float64)[None, :, None]
+    assert y.shape == (N, M, R, 1) and np.abs(y[..., 0] - ref).max() <= 1e-5
+    # B = identity returns A
+    assert np.array_equal(xo.matmul(a, np.eye(K, dtype=np.float32)), a)
+    # a vector times B is Eq. 1 with W = B^T: same products, same order of the sum
+    v = gen.uniform(11, 4, (N, K), -1.0, 1.0)
+    assert np.array_equal(xo.matmul(v, b, bias), xo.fc(v, np.ascontiguousarray(b.T), bias))
+    # (A B1) B2 = A (B1 B2) within rounding: the identity the MatmulX -> MatmulY link rests on
+    b2 = gen.normal(11, 5, (M, 4), 0.0, 0.5)
+    two = xo.matmul(xo.matmul(a, b), b2)
+    one = xo.matmul(a, (b.astype(np.float64) @ b2.astype(np.float64)).astype(np.float32))
+    assert np.abs(two - one).max() <= 1e-5 * max(1.0, np.abs(two).max())

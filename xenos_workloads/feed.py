@@ -13,7 +13,7 @@ import numpy as np
 def graph_from_spec(spec, params: Dict[str, Dict[str, np.ndarray]], in_dtype=None, in_layout=None, hw=None):
     """Returns (Graph, {tensor name: id}) for the records of ``spec``."""
     from paper_2302_00282_b200 import binding as xb
-    kind = {"maxpool": xb.OP_POOL_MAX, "avgpool": xb.OP_POOL_AVG, "gap": xb.OP_POOL_GLOBAL_AVG, "add": xb.OP_ADD,
+    kind = {"mul": xb.OP_MUL, "mac": xb.OP_MAC, "transpose": xb.OP_TRANSPOSE, "maxpool": xb.OP_POOL_MAX, "avgpool": xb.OP_POOL_AVG, "gap": xb.OP_POOL_GLOBAL_AVG, "add": xb.OP_ADD,
             "concat": xb.OP_CONCAT, "relu": xb.OP_RELU, "relu6": xb.OP_RELU6}
     in_dtype = xb.DTYPE_F32 if in_dtype is None else in_dtype
     in_layout = xb.LAYOUT_NCHW if in_layout is None else in_layout
@@ -28,6 +28,10 @@ def graph_from_spec(spec, params: Dict[str, Dict[str, np.ndarray]], in_dtype=Non
                          weight=p["w"], bias=p.get("b"))
         elif k == "fc":
             t = g.add_op(xb.OP_FC, ins, cout=o["cout"], k=1, weight=p["w"], bias=p.get("b"))
+        elif k == "matmul":
+            t = g.add_op(xb.OP_MATMUL, ins, cout=o["cout"], k=1, weight=p["w"], bias=p.get("b"))
+        elif k == "split":
+            t = g.add_op(xb.OP_SPLIT, ins, cout=o["cout"], pad=o["first"])
         elif k == "bn":
             t = g.add_op(xb.OP_BATCHNORM, ins, bn=(p["gamma"], p["beta"], p["mean"], p["var"]), bn_eps=1e-5)
         elif k in ("maxpool", "avgpool"):

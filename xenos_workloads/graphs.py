@@ -72,6 +72,30 @@ class GraphSpec:
         c = sum(self.shapes[x][0] for x in xs)
         return self._add(dict(name=name, kind="concat", inputs=list(xs)), (c,) + self.shapes[xs[0]][1:])
 
+    def mul(self, name, a, b) -> str:
+        assert self.shapes[a] == self.shapes[b]
+        return self._add(dict(name=name, kind="mul", inputs=[a, b]), self.shapes[a])
+
+    def mac(self, name, a, b, c) -> str:
+        assert self.shapes[a] == self.shapes[b] == self.shapes[c]
+        return self._add(dict(name=name, kind="mac", inputs=[a, b, c]), self.shapes[a])
+
+    def transpose(self, name, x) -> str:
+        c, h, w = self.shapes[x]
+        assert w == 1
+        return self._add(dict(name=name, kind="transpose", inputs=[x]), (h, c, 1))
+
+    def split(self, name, x, first, cout) -> str:
+        c, h, w = self.shapes[x]
+        assert first + cout <= c
+        return self._add(dict(name=name, kind="split", inputs=[x], first=first, cout=cout), (cout, h, w))
+
+    def matmul(self, name, x, cout, bias=False) -> str:
+        """x (K columns) times a constant [K][cout] matrix."""
+        sh = self.shapes[x]
+        return self._add(dict(name=name, kind="matmul", inputs=[x], cin=sh[0], cout=cout, bias=bias),
+                         (cout,) + tuple(sh[1:]))
+
     def fc(self, name, x, cout, bias=True) -> str:
         return self._add(dict(name=name, kind="fc", inputs=[x], cin=self.shapes[x][0], cout=cout, bias=bias),
                          (cout,))
@@ -113,6 +137,12 @@ def make_params(spec: GraphSpec, seed: int = gen.DEFAULT_SEED) -> Dict[str, Dict
             cg = o["cin"] // o["groups"]
             fan_in = cg * o["k"] * o["k"]
             p["w"] = gen.normal(seed, tid, (o["cout"], cg, o["k"], o["k"]), 0.0, float(np.sqrt(2.0 / fan_in)))
+            tid += 1
+            if o["bias"]:
+                p["b"] = gen.uniform(seed, tid, (o["cout"],), -0.1, 0.1)
+            tid += 1
+        elif o["kind"] == "matmul":
+            p["w"] = gen.normal(seed, tid, (o["cin"], o["cout"]), 0.0, float(np.sqrt(2.0 / o["cin"])))
             tid += 1
             if o["bias"]:
                 p["b"] = gen.uniform(seed, tid, (o["cout"],), -0.1, 0.1)
