@@ -76,6 +76,11 @@ struct GemmParams {
     int acc_stride, tmem_cols;                     // two accumulators, acc_stride columns apart
     int hstages, halo_bytes, halo_stride, halo_h, halo_w, halo_cb;   // halo ring (depthwise input tile / stem image patch)
     int stem_tma, stem_align;                       // stem: patch by TMA; x origin alignment in elements
+    // Activation operand by TMA where a K block of it is a box of the NHWC tensor (stride 1, channels a multiple of
+    // 64): 1 = the tile's 128 rows of the [pixels][C] matrix (1x1 convolution, fc), 2 = the tile's rh x rw patch
+    // shifted by the tap (k x k; out-of-range coordinates read zeros, which is the padding).  The copy engine
+    // writes the 128-byte-swizzled operand layout itself and the producer warps have nothing to do.
+    int a_tma, a_box_bytes, a_cpb;                  // a_cpb: 64-channel blocks per tap
     int off_halo, off_stg, off_dww, off_bias, off_bar;   // shared-memory offsets from the 1024-aligned base
     int act, act2, epi, out_ctot, out_coff, out_f32, skip_ctot;
     uint32_t idesc;
@@ -801,6 +806,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
     const bool dw_mode = g.seg[0].mode == GA_DW;
     // gather stages complete through cp.async arrivals (one per thread); the others through one
     // arrival per producer warp
+    const bool tma_a = g.a_tma != 0;
     const bool async_gather = g.seg[0].mode == GA_GATHER;
     // depthwise: the producer threads are (pixel block, channel quad of the K block) pairs
     const int dw_quads = g.halo_cb > 32 ? 16 : 8;
@@ -813,7 +819,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
         // arrivals on a stage's "full" barrier: the TMA lane plus the producers of that stage (every
         // thread for cp.async gathers, every warp otherwise)
         const uint32_t prod_warps = kProducerThreads / 32;
-        const uint32_t full_count = (async_gather ? kProducerThreads : prod_warps) + 1;
+        const uint32_t full_count = tma_a ? 1u : (async_gather ? kProducerThreads : prod_warps) + 1;
         for (int s = 0; s < g.stages; ++s) { mbar_init(full_bar(s), full_count); mbar_init(empty_bar(s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), kEpilogueThreads / 32); }
         for (int s = 0; s < g.hstages; ++s) { mbar_init(hfull_bar(s), 1); mbar_init(hempty_bar(s), prod_warps); }
@@ -900,7 +906,15 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                     }
                     ok = mbar_wait(empty_bar(st.s), st.ph ^ 1u);
                     if (!ok) break;
-                    mbar_arrive_expect_tx(full_bar(st.s), (uint32_t)g.tile_n * 128u);
+                    mbar_arrive_expect_tx(full_bar(st.s), (uint32_t)g.tile_n * 128u + (tma_a ? (uint32_t)g.a_box_bytes : 0u));
+                    if (g.a_tma == 1) {
+                        tma_load_2d(sbase + st.s * stage_bytes, &tmH, kb * kTileK, w.mt * g.tile_rows, full_bar(st.s));
+                    } else if (g.a_tma == 2) {
+                        const int tap = kb / g.a_cpb, cb = kb - tap * g.a_cpb;
+                        const int tr = tap / g.seg[0].k, ts = tap - tr * g.seg[0].k;
+                        tma_load_4d(sbase + st.s * stage_bytes, &tmH, cb * kTileK, w.tx * g.step_x - g.off_x + ts - g.seg[0].pad,
+                                    w.ty * g.step_y - g.off_y + tr - g.seg[0].pad, hn, full_bar(st.s));
+                    }
                     tma_load_2d(sbase + st.s * stage_bytes + kABytes, &tmB, kb * kTileK, tk.nt * g.tile_n, full_bar(st.s));
                     st.next(g.stages);
                 }
@@ -1037,7 +1051,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
         RowLocal grl[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) grl[i] = row_local(g, grow0 + 32 * i);
-        for (; !g.stem_tma && !dw_mode && w.ti < total_tiles && ok; w.next(g)) {
+        for (; !g.stem_tma && !dw_mode && !tma_a && w.ti < total_tiles && ok; w.next(g)) {
             RowPos rp;
             rp.valid = 0; rp.n = 0; rp.p = 0; rp.q = 0;
             const TileK tk = tile_k<kSplit>(g, w.nt);

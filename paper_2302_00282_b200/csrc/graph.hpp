@@ -133,6 +133,7 @@ struct Launch {
     int acc_stride = 0;                                            // columns between the two accumulators
     int hstages = 0, halo_bytes = 0, halo_stride = 0, halo_cb = 0;   // depthwise halo ring (halo_h x halo_w input pixels per image)
     int stem_tma = 0, stem_align = 1;                              // stem: image patch by TMA, x alignment in elements
+    int a_tma = 0, a_box_bytes = 0;                                // activation operand by TMA: 1 matrix rows, 2 shifted patch
     int off_halo = 0, off_stg = 0, off_dww = 0, off_bias = 0, off_bar = 0;                    // shared-memory layout
     // reduction split: ksplit chunks of kb_per K blocks; fp32 partial sums [chunk][pixel][npad] in the workspace's
     // split scratch, two counters (chunks arrived, chunks reduced) per (row tile, channel tile)

@@ -658,6 +658,36 @@ struct Lower {
             L.tile_rows = L.imgs_per_tile * L.rows_per_image;
             L.gap_imgs = L.imgs_per_tile; L.gap_area = L.rows_per_image; L.gap_rpi = L.rows_per_image;
         }
+        // Where a 64-channel K block of the activation operand is a box of the NHWC tensor (stride 1, channels a
+        // multiple of 64, no second K segment), TMA fetches it and writes the operand layout itself: the rows of
+        // the [pixels][C] matrix for a 1x1 convolution or fc, the tile's patch shifted by the tap for k x k.
+        if (s0.mode == AM_GATHER && !expand2 && !shortcut && !pooln && src.c % 64 == 0 && M.stride == 1) {
+            if (M.k == 1 && M.pad == 0) {
+                L.a_tma = 1;
+                L.a_box_bytes = 128 * 128;
+            } else if (!gapn && !fc) {
+                // patch tiles: ni whole images when one fits 128 rows, else rh x rw output pixels with the fewest tiles
+                L.a_tma = 2;
+                L.map_mode = MAP_PATCH;
+                if (L.P * L.Q <= 128) {
+                    L.patch_rh = L.P; L.patch_rw = L.Q; L.ni = std::min(128 / (L.P * L.Q), g.max_batch);
+                    // (fewer images per tile while units would idle, as for the depthwise chains)
+                    while (L.ni > 1 && (long)ceil_div(g.max_batch, L.ni) * ceil_div(round_up(N, 16), 256) * 2 <= g.hw.sm_count) --L.ni;
+                } else {
+                    L.ni = 1;
+                    long best = -1;
+                    for (int tw = 1; tw <= std::min(L.Q, 128); ++tw) {
+                        int th = std::min(L.P, 128 / tw);
+                        long tiles = (long)ceil_div(L.P, th) * ceil_div(L.Q, tw);
+                        if (best < 0 || tiles < best || (tiles == best && tw > L.patch_rw)) { best = tiles; L.patch_rh = th; L.patch_rw = tw; }
+                    }
+                }
+                L.tiles_y = ceil_div(L.P, L.patch_rh); L.tiles_x = ceil_div(L.Q, L.patch_rw);
+                L.step_y = L.patch_rh; L.step_x = L.patch_rw; L.off_y = L.off_x = 0;
+                L.tile_rows = L.ni * L.patch_rh * L.patch_rw;
+                L.a_box_bytes = L.tile_rows * 128;
+            }
+        }
         if (s0.mode == AM_STEM) {
             // The stem stages the tile's input patch in shared memory, so its tile is a patch too:
             // the pool patch when a pool is linked, else th x tw output pixels with the fewest tiles.
@@ -773,7 +803,7 @@ struct Lower {
             // (a linked depthwise stage can be split on request: a chunk's CTA then produces only its own channels of
             // the depthwise result.  It is not chosen automatically: measured at batch 1 the partial sums and their
             // reduction cost more than the shorter depthwise loop saves; the split search may still pick it.)
-            const bool plain = s0.mode == AM_GATHER && L.map_mode == MAP_FLAT;
+            const bool plain = s0.mode == AM_GATHER && (L.map_mode == MAP_FLAT || L.a_tma == 2);
             const bool can = (plain || s0.mode == AM_DW) && s1.mode == AM_NONE && L.epi == EPI_STORE;
             int want = 1;
             if (rq.user && rq.k > 1) {
@@ -1139,7 +1169,7 @@ void emit_plan_json(Graph &g) {
             jint(s, "ni", L.ni); jint(s, "step_y", L.step_y); jint(s, "step_x", L.step_x); jint(s, "off_y", L.off_y); jint(s, "off_x", L.off_x);
             jint(s, "hstages", L.hstages); jint(s, "halo_h", L.halo_h); jint(s, "halo_w", L.halo_w); jint(s, "halo_cb", L.halo_cb);
             jint(s, "halo_bytes", L.halo_bytes);
-            jint(s, "ksplit", L.ksplit); jint(s, "kb_per", L.kb_per);
+            jint(s, "ksplit", L.ksplit); jint(s, "kb_per", L.kb_per); jint(s, "a_tma", L.a_tma);
         }
         if (L.kind == LK_F32_CONV_CONV_POOL) {
             jint(s, "parts_outc", L.parts_outc); jint(s, "tile_h", L.tile_h); jint(s, "tile_w", L.tile_w);

@@ -61,6 +61,33 @@ static xenos_status_t encode_halo_map(const Graph &g, Runtime *rt, const Launch 
     return XENOS_OK;
 }
 
+// Activation operand by TMA: the [pixels][C] matrix of an NHWC tensor (box = 128 rows of one 64-channel block), or the
+// tensor itself as (C, W, H, N) with a box of one tile's patch; 128-byte swizzle, the layout the MMA descriptor reads.
+static xenos_status_t encode_a_map(const Graph &g, Runtime *rt, const Launch &L, void *base, int images, CUtensorMap *out) {
+    const ASeg &a = L.seg[0];
+    CUresult r;
+    if (((uintptr_t)base & 15u) || (a.C % 64)) return fail(g, XENOS_E_CUDA, "internal: activation operand is not addressable by TMA");
+    if (L.a_tma == 1) {
+        cuuint64_t dims[2] = {(cuuint64_t)a.C, (cuuint64_t)images * a.H * a.W};
+        cuuint64_t strides[1] = {(cuuint64_t)a.C * 2};
+        cuuint32_t box[2] = {64u, 128u};
+        cuuint32_t estr[2] = {1u, 1u};
+        r = rt->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                       CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    } else {
+        cuuint64_t dims[4] = {(cuuint64_t)a.C, (cuuint64_t)a.W, (cuuint64_t)a.H, (cuuint64_t)images};
+        cuuint64_t strides[3] = {(cuuint64_t)a.C * 2, (cuuint64_t)a.W * a.C * 2, (cuuint64_t)a.H * a.W * a.C * 2};
+        cuuint32_t box[4] = {64u, (cuuint32_t)L.patch_rw, (cuuint32_t)L.patch_rh, (cuuint32_t)L.ni};
+        cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+        if (box[1] > 256u || box[2] > 256u || box[3] > 256u || box[1] * box[2] * box[3] > 128u)
+            return fail(g, XENOS_E_CUDA, "internal: activation patch exceeds the TMA box limits");
+        r = rt->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                       CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    }
+    if (r != CUDA_SUCCESS) return fail(g, XENOS_E_CUDA, "cuTensorMapEncodeTiled (activation operand) failed with code " + std::to_string((int)r));
+    return XENOS_OK;
+}
+
 // 4-D map (W, H, C, N) over a small-channel NCHW image; box = one tile's input patch, all channels.
 static xenos_status_t encode_stem_map(const Graph &g, Runtime *rt, const Launch &L, void *base, int images, CUtensorMap *out) {
     const ASeg &a = L.seg[0];
@@ -137,6 +164,10 @@ xenos_status_t runtime_bind(Graph &g, void *ws, size_t bytes, void *stream_v) {
                                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
             if (r != CUDA_SUCCESS) return fail(g, XENOS_E_CUDA, "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r));
+            if (L.a_tma && g.tensors[L.seg[0].tensor].input_slot < 0) {
+                xenos_status_t st = encode_a_map(g, rt, L, static_cast<uint8_t *>(ws) + g.place[L.seg[0].tensor].off, g.max_batch, &rt->hmaps[i]);
+                if (st != XENOS_OK) return st;
+            }
             if (L.seg[0].mode == AM_DW && g.tensors[L.seg[0].tensor].input_slot < 0) {
                 xenos_status_t st = encode_halo_map(g, rt, L, static_cast<uint8_t *>(ws) + g.place[L.seg[0].tensor].off, g.max_batch, &rt->hmaps[i]);
                 if (st != XENOS_OK) return st;
@@ -326,6 +357,7 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
             p.hstages = L.hstages; p.halo_bytes = L.halo_bytes; p.halo_stride = L.halo_stride;
             p.halo_h = L.halo_h; p.halo_w = L.halo_w; p.halo_cb = L.halo_cb;
             p.stem_tma = L.stem_tma; p.stem_align = L.stem_align;
+            p.a_tma = L.a_tma; p.a_box_bytes = L.a_box_bytes; p.a_cpb = L.seg[0].C / 64;
             p.off_halo = L.off_halo; p.off_stg = L.off_stg; p.off_dww = L.off_dww; p.off_bias = L.off_bias; p.off_bar = L.off_bar;
             p.act = L.act; p.act2 = L.act2; p.epi = L.epi; p.out_ctot = L.out_ctot; p.out_coff = L.out_coff;
             p.out_f32 = L.out_dtype == XENOS_DTYPE_F32;
@@ -345,6 +377,16 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
                     xenos_status_t st = encode_stem_map(g, rt, L, ptr(L.seg[0].tensor), N, &tmh_now);
                     if (st != XENOS_OK) return st;
                     tmh = &tmh_now;
+                }
+            }
+            if (L.a_tma) {
+                if (g.tensors[L.seg[0].tensor].input_slot >= 0) {
+                    // the operand is a caller buffer: its map is encoded now (rows / images beyond the batch read zeros)
+                    xenos_status_t st = encode_a_map(g, rt, L, ptr(L.seg[0].tensor), N, &tmh_now);
+                    if (st != XENOS_OK) return st;
+                    tmh = &tmh_now;
+                } else {
+                    tmh = &rt->hmaps[li];
                 }
             }
             if (L.seg[0].mode == AM_DW) {

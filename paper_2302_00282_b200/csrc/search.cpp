@@ -62,7 +62,7 @@ xenos_status_t search_splits(Graph &g, int max_batch, int precision, void *ws, s
         std::vector<Cand> more;
         auto add = [&](const SplitRequest &rq, const std::string &label) { Cand c; c.rq = rq; c.label = label; more.push_back(c); };
         if (L.kind == LK_GEMM) {
-            const bool can_k = ((L.seg[0].mode == AM_GATHER && L.map_mode == MAP_FLAT) || L.seg[0].mode == AM_DW) &&
+            const bool can_k = ((L.seg[0].mode == AM_GATHER && (L.map_mode == MAP_FLAT || L.a_tma == 2)) || L.seg[0].mode == AM_DW) &&
                                L.seg[1].mode == AM_NONE && L.epi == EPI_STORE;
             add(make_rq(L.n_tiles * 2, 0, 0, 1), "outc x2");
             if (L.n_tiles > 1) add(make_rq((L.n_tiles + 1) / 2, 0, 0, 1), "outc /2");

@@ -117,6 +117,12 @@ CONV_CASES = [
     (32, 8, 40, 1, 2, 0, 2),        # strided 1x1 (projection shape), N not a multiple of 16
     (8, 20, 16, 7, 2, 3, 1),        # 7x7
     (256, 7, 1000, 1, 1, 0, 2),     # classifier-like: ragged N = 1000
+    # channel counts that are multiples of 64 at stride 1: the activation operand comes by TMA
+    (128, 28, 96, 3, 1, 1, 2),      # 3x3, two channel blocks per tap, patch tiles 4 x 28 with a ragged last row of tiles
+    (64, 7, 64, 3, 1, 1, 5),        # small maps: whole images per tile (two per tile, odd batch)
+    (64, 19, 48, 5, 1, 2, 1),       # 5x5, pad 2: taps reach two pixels outside the image
+    (192, 10, 72, 3, 1, 0, 2),      # no padding: the output is smaller than the input
+    (64, 33, 32, 1, 1, 0, 3),       # 1x1: 3267 rows, ragged last 128-row box
 ]
 
 
@@ -136,6 +142,28 @@ def test_bf16_pointwise_many_tiles_per_unit():
     x = xo.round_bf16(graphs.make_input(spec, 16))
     for _ in range(3):
         assert np.array_equal(gg.run(x), y)
+
+
+def test_bf16_conv_operand_by_tma_is_planned_where_it_applies():
+    def a_tma(case):
+        cin, hw, cout, k, st, pad, batch = case
+        spec = _one(lambda g: g.cbr("c", "input", cout, k, st, pad, act="relu"), cin, hw)
+        gg = GpuGraph(spec, graphs.make_params(spec), batch, linked=False, in_mode="bf16_nhwc")
+        return gg.g.plan()["launches"][0]["a_tma"]
+    assert [a_tma(c) for c in CONV_CASES] == [1, 1, 0, 0, 2, 0, 0, 1, 2, 2, 2, 2, 1]
+
+
+def test_bf16_tma_conv_with_identity_shortcut_and_caller_input():
+    """conv3x3 (+ identity shortcut, ReLU) whose operand is the caller's NHWC buffer: the TMA map is encoded at run
+    time, here for a batch below max_batch."""
+    def build(g):
+        y = g.cbr("c2", "input", 64, 3, 1, 1, act=None)
+        y = g.add("add", y, "input")
+        g.act("relu", y, "relu")
+    spec = _one(build, 64, 14)
+    _, _, gg = check_bf16("tma_conv_skip", spec, 3, linked=True, in_mode="bf16_nhwc", max_batch=8)
+    L = gg.g.plan()["launches"][0]
+    assert gg.g.launch_count() == 1 and L["a_tma"] == 2 and L["skip"] >= 0
 
 
 def test_bf16_conv1x1_equals_matmul():
