@@ -154,15 +154,17 @@ xenos_status_t xenos_graph_link(xenos_graph_t *gp, const xenos_id_t *ops, int32_
             return fail(g, XENOS_E_INVALID, "link: id is not an operator output");
         r.ops.push_back(ops[i]);
     }
-    // adjacency is checked here so that a bad request fails at the call that made it:
-    // ops[i+1] must read ops[i], possibly through the bn / activation records that follow ops[i]
+    // adjacency is checked here so that a bad request fails at the call that made it: every operator after the
+    // first must read an earlier operator of the list (the one before it in a plain chain; the squeeze convolution
+    // for both expands of a fire module), possibly through the bn / activation records that follow that operator
     for (int i = 0; i + 1 < n_ops; ++i) {
         const Op &nx = g.ops[g.tensors[r.ops[i + 1]].producer];
         bool found = false;
         for (int t : nx.in) {
             int cur = t;
             for (int hop = 0; hop < 3 && cur >= 0; ++hop) {
-                if (cur == r.ops[i]) { found = true; break; }
+                for (int e = 0; e <= i; ++e) if (cur == r.ops[e]) found = true;
+                if (found) break;
                 int p = g.tensors[cur].producer;
                 if (p < 0) break;
                 int kd = g.ops[p].kind;

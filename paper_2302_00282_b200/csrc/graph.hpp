@@ -58,7 +58,9 @@ enum ChainKind {
     CK_DW_PW,               // depthwise 3x3 -> pointwise [-> global avgpool]
     CK_CONV_TAIL,           // conv [+ linked shortcut conv] [-> add -> relu] [-> max pool | global avgpool]
     CK_EXPAND_CONCAT,       // {conv1x1, conv3x3} on one input -> concat [-> max pool]
-    CK_MATMUL_MATMUL        // MatmulX -> MatmulY with constant right operands: one product with the constants multiplied
+    CK_MATMUL_MATMUL,       // MatmulX -> MatmulY with constant right operands: one product with the constants multiplied
+    CK_CONV_CONV            // ConvX -> ConvY with the intermediate tile in shared memory: conv -> conv1x1 | conv3x3
+                            // [-> add (identity shortcut)], or squeeze -> {expand1x1 ; expand3x3} -> concat
 };
 
 struct SplitRequest { int outc = 0, h = 0, w = 0, k = 1; bool user = false; };
@@ -95,7 +97,8 @@ enum LaunchKind {
     LK_F32_CONV,          // fp32 NCHW direct conv (+bias, act), any k / stride / pad, dense or depthwise
     LK_F32_POOL, LK_F32_GAP, LK_F32_ADD, LK_F32_CONCAT_PART, LK_F32_FC,
     LK_F32_CONV_CONV_POOL, // fp32 linked chain
-    LK_F32_MULMAC, LK_F32_TRANSPOSE, LK_F32_SLICE
+    LK_F32_MULMAC, LK_F32_TRANSPOSE, LK_F32_SLICE,
+    LK_GEMM2              // two linked convolutions, intermediate tile in shared memory (chain2_kernel)
 };
 
 struct Launch {
@@ -134,6 +137,8 @@ struct Launch {
     int hstages = 0, halo_bytes = 0, halo_stride = 0, halo_cb = 0;   // depthwise halo ring (halo_h x halo_w input pixels per image)
     int stem_tma = 0, stem_align = 1;                              // stem: image patch by TMA, x alignment in elements
     int a_tma = 0, a_box_bytes = 0;                                // activation operand by TMA: 1 matrix rows, 2 shifted patch
+    // ---- two linked convolutions (LK_GEMM2): producer tile rh1 x rw1 = patch_rh x patch_rw, consumer tile rh2 x rw2
+    int k2 = 1, kblocks2 = 0, n1pad = 0, halo2 = 0, rh2 = 0, rw2 = 0, act3 = 0, off_mid = 0, stage_bytes = 0;
     int off_halo = 0, off_stg = 0, off_dww = 0, off_bias = 0, off_bar = 0;                    // shared-memory layout
     // reduction split: ksplit chunks of kb_per K blocks; fp32 partial sums [chunk][pixel][npad] in the workspace's
     // split scratch, two counters (chunks arrived, chunks reduced) per (row tile, channel tile)

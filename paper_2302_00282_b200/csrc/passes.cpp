@@ -151,8 +151,39 @@ static bool pool_patch(int k, int s, int PP, int PQ, int &th, int &tw, int &rh, 
 typedef bool (*AllowFn)(const void *, int);
 
 // Try to grow a chain anchored at node a.  allowed(n) says whether n may join.
+// Tile geometry of two linked convolutions: the producer tile rh1 x rw1 (<= 128 pixels, rw1 <= 30 so that every tap
+// offset stays inside the middle buffer's spare rows) that needs the fewest tiles for a P x Q map, given the
+// consumer's frame h = (k2 - 1) / 2.
+static bool chain2_tile(int P, int Q, int h, int &rh1, int &rw1) {
+    long best = -1;
+    for (int w = 2 * h + 1; w <= std::min(Q + 2 * h, 30); ++w) {
+        int hh = std::min(P + 2 * h, 128 / w);
+        if (hh < 2 * h + 1) continue;
+        long tiles = (long)((P + hh - 2 * h - 1) / (hh - 2 * h)) * ((Q + w - 2 * h - 1) / (w - 2 * h));
+        if (best < 0 || tiles < best || (tiles == best && w > rw1)) { best = tiles; rh1 = hh; rw1 = w; }
+    }
+    return best > 0;
+}
+
+// Modelled time of linking two convolutions against running them one after the other (per image, arbitrary
+// units): the linked form issues whole 128-row tiles for both products, frame rows included, and moves no
+// intermediate; rates are what this library's kernels reach, not the device's peaks.
+static bool chain2_pays(const Graph &g, const Node &A, const Node &B, bool skip) {
+    const Tensor &o = g.tensors[B.out];
+    const int h = (B.k - 1) / 2;
+    int rh1 = 0, rw1 = 0;
+    if (!chain2_tile(o.h, o.w, h, rh1, rw1)) return false;
+    const double tiles = (double)((o.h + rh1 - 2 * h - 1) / (rh1 - 2 * h)) * ((o.w + rw1 - 2 * h - 1) / (rw1 - 2 * h));
+    const double tc = 0.5e15, hbm = 4.0e12, px = (double)o.h * o.w;
+    const double k1 = (double)A.cin * A.k * A.k, k2 = (double)A.cout * B.k * B.k;
+    const double in = px * A.cin * 2, midb = px * A.cout * 2, outb = px * B.cout * 2 * (skip ? 2 : 1);
+    const double lin = std::max(2.0 * tiles * 128 * (k1 * A.cout + k2 * B.cout) / tc, (in + outb) / hbm);
+    const double unl = std::max(2.0 * px * k1 * A.cout / tc, (in + midb) / hbm) + std::max(2.0 * px * k2 * B.cout / tc, (midb + outb) / hbm);
+    return lin < 0.95 * unl;
+}
+
 template <class Allowed>
-static bool try_match(const LinkCtx &cx, int a, Allowed allowed, Chain &out) {
+static bool try_match(const LinkCtx &cx, int a, Allowed allowed, Chain &out, bool by_model = true) {
     Graph &g = cx.g;
     const Node &A = g.nodes[a];
     out = Chain();
@@ -221,6 +252,26 @@ static bool try_match(const LinkCtx &cx, int a, Allowed allowed, Chain &out) {
         out.kind = CK_EXPAND_CONCAT;
         out.nodes = {e0, e1, a};
         out.pattern = "ConvX -> {ConvY ; ConvZ} -> concat (joined without a layout transformation)";
+        {
+            // the squeeze convolution in front of the two expands: its result stays in shared memory
+            int sq = g.node_of_tensor[E0.in[0]];
+            const std::vector<int> &sc = cx.cons[E0.in[0]];
+            if (sq >= 0 && allowed(sq) && g.nodes[sq].kind == NK_CONV && !g.nodes[sq].from_matmul && g.nodes[sq].stride == 1 &&
+                g.nodes[sq].cin % 64 == 0 && (g.nodes[sq].cout <= 64 || g.nodes[sq].cout % 64 == 0) && g.nodes[sq].cout <= 256 &&
+                g.tensors[E0.in[0]].output_slot < 0 && sc.size() == 2 && cx.sole(a) >= -1 &&
+                !(g.tensors[g.nodes[sq].in[0]].input_slot >= 0 && g.tensors[g.nodes[sq].in[0]].io_layout == XENOS_LAYOUT_NCHW)) {
+                int p2 = cx.sole(a);
+                const bool pooled = p2 >= 0 && g.nodes[p2].kind == NK_MAXPOOL;      // the pooled fire modules keep the pool link
+                Node merged = E0.k == 3 ? E0 : E1;
+                merged.cout = E0.cout + E1.cout;
+                if (!pooled && (!by_model || chain2_pays(g, g.nodes[sq], merged, false))) {
+                    out.kind = CK_CONV_CONV;
+                    out.nodes = {sq, e0, e1, a};
+                    out.pattern = "ConvX -> {ConvY ; ConvZ} -> concat, ConvX's result kept on chip (fire module)";
+                    return true;
+                }
+            }
+        }
         int p = cx.sole(a);
         if (p >= 0 && allowed(p) && g.nodes[p].kind == NK_MAXPOOL) {
             int th, tw, rh, rw;
@@ -239,6 +290,28 @@ static bool try_match(const LinkCtx &cx, int a, Allowed allowed, Chain &out) {
         int b = cx.sole(a);
         if (b < 0 || !allowed(b)) return false;
         const Node &B = g.nodes[b];
+        if (B.kind == NK_CONV && !nchw_in && !A.from_matmul && !B.from_matmul && A.stride == 1 && A.cin % 64 == 0 &&
+            (A.cout <= 64 || A.cout % 64 == 0) && A.cout <= 256 && A.cout % 8 == 0 && B.stride == 1 &&
+            ((B.k == 1 && B.pad == 0) || (B.k == 3 && B.pad == 1)) && B.cout % 8 == 0) {
+            // ConvX -> ConvY (rows 1-4 of Table 1) [-> add with an identity branch]: the intermediate tile stays on chip
+            int c = cx.sole(b);
+            // (a 3x3 consumer that could itself feed a 1x1 convolution is left for that pairing, which needs no frame)
+            if (by_model && B.k == 3 && c >= 0 && g.nodes[c].kind == NK_CONV && g.nodes[c].k == 1 && g.nodes[c].stride == 1 &&
+                g.nodes[c].pad == 0 && B.cin % 64 == 0 && (B.cout <= 64 || B.cout % 64 == 0) && B.cout <= 256)
+                return false;
+            bool with_add = false;
+            if (c >= 0 && allowed(c) && g.nodes[c].kind == NK_ADD && B.act == XENOS_ACT_NONE) {
+                int other = g.nodes[c].in[0] == B.out ? g.nodes[c].in[1] : g.nodes[c].in[0];
+                with_add = other != B.out;
+            }
+            if (!by_model || chain2_pays(g, A, B, with_add)) {
+                out.kind = CK_CONV_CONV;
+                out.nodes = {a, b};
+                out.pattern = B.k == 1 ? "ConvX -> ConvY (Conv kxk -> Conv 1x1, intermediate on chip)" : "ConvX -> ConvY (Conv kxk -> Conv 3x3, intermediate with its halo on chip)";
+                if (with_add) { out.nodes.push_back(c); out.pattern += " + shortcut connection (identity)"; }
+                return true;
+            }
+        }
         if (B.kind == NK_ADD && !nchw_in) {
             int other = B.in[0] == A.out ? B.in[1] : B.in[0];
             if (other == A.out) return false;
@@ -306,7 +379,7 @@ xenos_status_t link_pass(Graph &g) {
         bool done = false;
         for (int a : want) {
             Chain c;
-            if (try_match(cx, a, [&](int n) { return want.count(n) > 0 && g.nodes[n].chain < 0; }, c)) {
+            if (try_match(cx, a, [&](int n) { return want.count(n) > 0 && g.nodes[n].chain < 0; }, c, false)) {
                 std::set<int> got(c.nodes.begin(), c.nodes.end());
                 if (got == want) { commit(c); done = true; break; }
             }
@@ -904,6 +977,94 @@ struct Lower {
         return XENOS_OK;
     }
 
+    // ---- two linked convolutions, intermediate tile in shared memory (chain2_kernel) ---------------------------
+    // A: first convolution (stride 1, input channels a multiple of 64).  Second stage: one convolution B (1x1, or
+    // 3x3 with padding 1), or the two expand convolutions of a fire module merged over the 3x3 window in concat order.
+    xenos_status_t make_gemm2(int ci, const std::vector<int> &cover, const Node &A, const Node *B, const Node *E0, const Node *E1,
+                              const Node *addn, const Node *last) {
+        Launch L;
+        L.kind = LK_GEMM2;
+        L.nodes = cover;
+        const Tensor &src = g.tensors[A.in[0]];
+        const Tensor &ot = g.tensors[last->out];
+        const int k2 = B ? B->k : 3, h = (k2 - 1) / 2;
+        const int N2 = B ? B->cout : E0->cout + E1->cout;
+        L.in0 = A.in[0]; L.out = last->out;
+        L.C = src.c; L.H = src.h; L.W = src.w; L.P = ot.h; L.Q = ot.w; L.K = N2; L.rows_per_image = L.P * L.Q;
+        L.k = A.k; L.stride = 1; L.pad = A.pad; L.k2 = k2; L.halo2 = h;
+        L.Cmid = A.cout; L.n1pad = round_up(A.cout, 64);
+        L.seg[0].tensor = L.in0; L.seg[0].C = src.c; L.seg[0].H = src.h; L.seg[0].W = src.w; L.seg[0].k = A.k; L.seg[0].pad = A.pad;
+        L.kblocks = A.k * A.k * (src.c / 64);
+        L.kblocks2 = k2 * k2 * (L.n1pad / 64);
+        L.act = A.act; L.act2 = B ? B->act : E0->act;
+        if (addn) {
+            L.act3 = addn->act;
+            const int mine = B->out;
+            L.skip = addn->in[0] == mine ? addn->in[1] : addn->in[0];
+        }
+        if (src.c % 64 || g.tensors[A.out].h != ot.h || g.tensors[A.out].w != ot.w)
+            return fail(g, XENOS_E_UNSUPPORTED, "internal: two linked convolutions need 64-channel input blocks and a consumer of equal extent");
+        if (!chain2_tile(L.P, L.Q, h, L.patch_rh, L.patch_rw)) return fail(g, XENOS_E_UNSUPPORTED, "internal: no tile for two linked convolutions");
+        L.rh2 = L.patch_rh - 2 * h; L.rw2 = L.patch_rw - 2 * h;
+        L.tiles_y = ceil_div(L.P, L.rh2); L.tiles_x = ceil_div(L.Q, L.rw2);
+        L.m_tiles = g.max_batch * L.tiles_y * L.tiles_x;
+        L.a_box_bytes = L.patch_rh * L.patch_rw * 128;
+        const int N216 = round_up(N2, 16);
+        L.n_tiles = ceil_div(N216, 256);
+        L.tile_n = round_up(ceil_div(N216, L.n_tiles), 16);
+        L.npad = L.n_tiles * L.tile_n;
+        L.out_ctot = ot.c; L.out_coff = 0;
+        L.stage_bytes = 16384 + std::max(L.n1pad, L.tile_n) * 128;
+        const int mid_bytes = (L.n1pad / 64) * (128 + 64) * 128;
+        const int cap = std::min(g.hw.smem_bytes_per_cta, 227 * 1024) - 1024 - 256;
+        L.stages = std::min(6, (cap - mid_bytes) / L.stage_bytes);
+        if (L.stages < 2) return fail(g, XENOS_E_BAD_SPLIT, "split: two linked convolutions do not fit shared memory");
+        L.off_mid = L.stages * L.stage_bytes;
+        L.off_bar = L.off_mid + mid_bytes;
+        L.smem_bytes = L.off_bar + 256 + 1024;
+        L.tmem_cols = 512;
+        L.grid = std::min(L.m_tiles, g.hw.sm_count);
+        L.block = 320;
+        if (g.chains[ci].split.user && (g.chains[ci].split.outc > 1 || g.chains[ci].split.h > 1 || g.chains[ci].split.w > 1 || g.chains[ci].split.k > 1))
+            return fail(g, XENOS_E_BAD_SPLIT, "split: two linked convolutions keep all output channels of a tile in one CTA; no explicit split");
+        // --- parameters: W1 [n1pad][K1], bias1 [n1pad]; W2 [npad][k2*k2*n1pad], bias2 [npad]; K order (tap, channel)
+        const int K1 = L.kblocks * 64, K2 = L.kblocks2 * 64;
+        L.kpad = K1;
+        L.w_off = blob_reserve(g, (size_t)L.n1pad * K1 * 2);
+        L.b_off = blob_reserve(g, (size_t)L.n1pad * 4);
+        L.w2_off = blob_reserve(g, (size_t)L.npad * K2 * 2);
+        L.b2_off = blob_reserve(g, (size_t)L.npad * 4);
+        uint16_t *w1 = reinterpret_cast<uint16_t *>(g.param_blob.data() + L.w_off);
+        float *b1 = reinterpret_cast<float *>(g.param_blob.data() + L.b_off);
+        uint16_t *w2 = reinterpret_cast<uint16_t *>(g.param_blob.data() + L.w2_off);
+        float *b2 = reinterpret_cast<float *>(g.param_blob.data() + L.b2_off);
+        for (int o = 0; o < A.cout; ++o) {
+            for (int c = 0; c < src.c; ++c)
+                for (int r = 0; r < A.k; ++r)
+                    for (int s2 = 0; s2 < A.k; ++s2)
+                        w1[(size_t)o * K1 + (r * A.k + s2) * src.c + c] = f32_to_bf16_rne(A.w[(((size_t)o * src.c + c) * A.k + r) * A.k + s2]);
+            b1[o] = A.b[o];
+        }
+        auto pack2 = [&](const Node &n, int row0) {
+            const int shift = (k2 - n.k) / 2;
+            for (int o = 0; o < n.cout; ++o) {
+                for (int c = 0; c < A.cout; ++c)
+                    for (int r = 0; r < n.k; ++r)
+                        for (int s2 = 0; s2 < n.k; ++s2)
+                            w2[(size_t)(row0 + o) * K2 + ((r + shift) * k2 + (s2 + shift)) * L.n1pad + c] =
+                                f32_to_bf16_rne(n.w[(((size_t)o * A.cout + c) * n.k + r) * n.k + s2]);
+                b2[row0 + o] = n.b[o];
+            }
+        };
+        if (B) pack2(*B, 0);
+        else { pack2(*E0, 0); pack2(*E1, E0->cout); }
+        for (int ni : cover) L.flops += 2.0 * node_macs(g.nodes[ni]);
+        L.bytes = tbytes(L.in0) + tbytes(L.out) + (double)L.n1pad * K1 * 2 + (double)L.npad * K2 * 2 + 4.0 * (L.n1pad + L.npad);
+        if (L.skip >= 0) L.bytes += tbytes(L.skip);
+        push(L, ci);
+        return XENOS_OK;
+    }
+
     xenos_status_t lower_bf16_single(int ci, int ni) {
         const Node &n = g.nodes[ni];
         if (n.kind == NK_CONV) return make_gemm(ci, {ni}, nullptr, &n, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, false);
@@ -989,6 +1150,19 @@ struct Lower {
             st = make_gemm(ci, ch.nodes, nullptr, &M, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, A.kind == NK_FC);
             // (the modelled work of the launch is the merged product's, not the sum of the two it replaces)
             if (st == XENOS_OK) g.launches.back().flops = 2.0 * node_macs(M);
+            break;
+        }
+        case CK_CONV_CONV: {
+            const Node *cat = find(NK_CONCAT);
+            if (cat) {
+                const Node *first = &g.nodes[g.node_of_tensor[cat->in[0]]];
+                const Node *second = &g.nodes[g.node_of_tensor[cat->in[1]]];
+                st = make_gemm2(ci, ch.nodes, g.nodes[ch.nodes[0]], nullptr, first, second, nullptr, cat);
+            } else {
+                const Node *addn = find(NK_ADD);
+                const Node &B = g.nodes[ch.nodes[1]];
+                st = make_gemm2(ci, ch.nodes, g.nodes[ch.nodes[0]], &B, nullptr, nullptr, addn, addn ? addn : &B);
+            }
             break;
         }
         case CK_EXPAND_CONCAT: {
@@ -1112,9 +1286,9 @@ static void jarr(std::string &s, const char *k, const std::vector<int> &v, bool 
 
 void emit_plan_json(Graph &g) {
     static const char *nk[] = {"?", "conv", "dwconv", "fc", "maxpool", "avgpool", "gap", "add", "concat", "mul", "mac", "transpose", "split"};
-    static const char *ck[] = {"single", "conv_conv_pool", "dw_pw", "conv_tail", "expand_concat", "matmul_matmul"};
+    static const char *ck[] = {"single", "conv_conv_pool", "dw_pw", "conv_tail", "expand_concat", "matmul_matmul", "conv_conv"};
     static const char *lk[] = {"?", "gemm", "dw", "pool", "gap", "add", "concat_part", "mulmac", "transpose", "slice", "f32_conv", "f32_pool",
-                               "f32_gap", "f32_add", "f32_concat_part", "f32_fc", "f32_conv_conv_pool", "f32_mulmac", "f32_transpose", "f32_slice"};
+                               "f32_gap", "f32_add", "f32_concat_part", "f32_fc", "f32_conv_conv_pool", "f32_mulmac", "f32_transpose", "f32_slice", "gemm2"};
     static const char *am[] = {"none", "gather", "stem", "dw"};
     std::string s = "{";
     jstr(s, "precision", g.precision == XENOS_PRECISION_FP32_CUDA_CORE ? "fp32_cuda_core" : "bf16_tensor");
@@ -1170,6 +1344,12 @@ void emit_plan_json(Graph &g) {
             jint(s, "hstages", L.hstages); jint(s, "halo_h", L.halo_h); jint(s, "halo_w", L.halo_w); jint(s, "halo_cb", L.halo_cb);
             jint(s, "halo_bytes", L.halo_bytes);
             jint(s, "ksplit", L.ksplit); jint(s, "kb_per", L.kb_per); jint(s, "a_tma", L.a_tma);
+        }
+        if (L.kind == LK_GEMM2) {
+            jint(s, "k2", L.k2); jint(s, "cmid", L.Cmid); jint(s, "n1pad", L.n1pad); jint(s, "kblocks", L.kblocks); jint(s, "kblocks2", L.kblocks2);
+            jint(s, "tile_n", L.tile_n); jint(s, "n_tiles", L.n_tiles); jint(s, "m_tiles", L.m_tiles); jint(s, "npad", L.npad);
+            jint(s, "patch_rh", L.patch_rh); jint(s, "patch_rw", L.patch_rw); jint(s, "rh2", L.rh2); jint(s, "rw2", L.rw2);
+            jint(s, "tiles_y", L.tiles_y); jint(s, "tiles_x", L.tiles_x); jint(s, "stages", L.stages);
         }
         if (L.kind == LK_F32_CONV_CONV_POOL) {
             jint(s, "parts_outc", L.parts_outc); jint(s, "tile_h", L.tile_h); jint(s, "tile_w", L.tile_w);

@@ -12,6 +12,7 @@
 #include <string>
 #include <vector>
 
+#include "chain2_tc.cuh"
 #include "gemm_tc.cuh"
 #include "graph.hpp"
 #include "kernels_bf16.cuh"
@@ -23,7 +24,8 @@ struct Runtime {
     int device = -1;
     int sm_count = 0;
     std::vector<CUtensorMap> tmaps;     // one per launch record (used by gemm launches only)
-    std::vector<CUtensorMap> hmaps;     // halo maps of linked depthwise stages
+    std::vector<CUtensorMap> hmaps;     // halo maps of linked depthwise stages / activation operand maps
+    std::vector<CUtensorMap> tmaps2;    // second weight matrix of two linked convolutions
     PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
 };
 
@@ -88,6 +90,35 @@ static xenos_status_t encode_a_map(const Graph &g, Runtime *rt, const Launch &L,
     return XENOS_OK;
 }
 
+// Maps of two linked convolutions: the first one's input (C, W, H, N) with a box of the producer tile, and the two
+// packed weight matrices.
+static xenos_status_t encode_chain2_input(const Graph &g, Runtime *rt, const Launch &L, void *base, int images, CUtensorMap *out) {
+    const ASeg &a = L.seg[0];
+    if (((uintptr_t)base & 15u) || (a.C % 64)) return fail(g, XENOS_E_CUDA, "internal: activation operand is not addressable by TMA");
+    cuuint64_t dims[4] = {(cuuint64_t)a.C, (cuuint64_t)a.W, (cuuint64_t)a.H, (cuuint64_t)images};
+    cuuint64_t strides[3] = {(cuuint64_t)a.C * 2, (cuuint64_t)a.W * a.C * 2, (cuuint64_t)a.H * a.W * a.C * 2};
+    cuuint32_t box[4] = {64u, (cuuint32_t)L.patch_rw, (cuuint32_t)L.patch_rh, 1u};
+    cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+    if (box[1] > 256u || box[2] > 256u || box[1] * box[2] > 128u) return fail(g, XENOS_E_CUDA, "internal: producer tile exceeds the TMA box limits");
+    CUresult r = rt->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(g, XENOS_E_CUDA, "cuTensorMapEncodeTiled (linked convolutions) failed with code " + std::to_string((int)r));
+    return XENOS_OK;
+}
+
+static xenos_status_t encode_weight_map(const Graph &g, Runtime *rt, void *gaddr, int kpad, int rows, int box_rows, CUtensorMap *out) {
+    cuuint64_t dims[2] = {(cuuint64_t)kpad, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)kpad * 2};
+    cuuint32_t box[2] = {64u, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1u, 1u};
+    if (((uintptr_t)gaddr & 15u) || (strides[0] & 15u) || box[1] > 256u || box[1] == 0u || box_rows % 16)
+        return fail(g, XENOS_E_CUDA, "internal: weight tensor map fields are misaligned");
+    CUresult r = rt->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, gaddr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(g, XENOS_E_CUDA, "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r));
+    return XENOS_OK;
+}
+
 // 4-D map (W, H, C, N) over a small-channel NCHW image; box = one tile's input patch, all channels.
 static xenos_status_t encode_stem_map(const Graph &g, Runtime *rt, const Launch &L, void *base, int images, CUtensorMap *out) {
     const ASeg &a = L.seg[0];
@@ -136,12 +167,15 @@ xenos_status_t runtime_bind(Graph &g, void *ws, size_t bytes, void *stream_v) {
     // TMA descriptors of the packed weight matrices
     bool any_gemm = false;
     int max_gemm_smem = 0, max_chain_smem = 0;
+    bool any_gemm2 = false;
     for (const Launch &L : g.launches) {
+        if (L.kind == LK_GEMM2) { any_gemm = any_gemm2 = true; max_gemm_smem = std::max(max_gemm_smem, L.smem_bytes); }
         if (L.kind == LK_GEMM) { any_gemm = true; max_gemm_smem = std::max(max_gemm_smem, L.smem_bytes); }
         if (L.kind == LK_F32_CONV_CONV_POOL) max_chain_smem = std::max(max_chain_smem, L.smem_bytes);
     }
     rt->tmaps.resize(g.launches.size());
     rt->hmaps.resize(g.launches.size());
+    rt->tmaps2.resize(g.launches.size());
     if (any_gemm) {
         void *fn = nullptr;
         cudaDriverEntryPointQueryResult qres;
@@ -151,6 +185,14 @@ xenos_status_t runtime_bind(Graph &g, void *ws, size_t bytes, void *stream_v) {
         rt->encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
         for (size_t i = 0; i < g.launches.size(); ++i) {
             const Launch &L = g.launches[i];
+            if (L.kind == LK_GEMM2) {
+                xenos_status_t st = encode_weight_map(g, rt, static_cast<uint8_t *>(ws) + L.w_off, L.kblocks * 64, L.n1pad, L.n1pad, &rt->tmaps[i]);
+                if (st == XENOS_OK) st = encode_weight_map(g, rt, static_cast<uint8_t *>(ws) + L.w2_off, L.kblocks2 * 64, L.npad, L.tile_n, &rt->tmaps2[i]);
+                if (st == XENOS_OK && g.tensors[L.in0].input_slot < 0)
+                    st = encode_chain2_input(g, rt, L, static_cast<uint8_t *>(ws) + g.place[L.in0].off, g.max_batch, &rt->hmaps[i]);
+                if (st != XENOS_OK) return st;
+                continue;
+            }
             if (L.kind != LK_GEMM) continue;
             cuuint64_t dims[2] = {(cuuint64_t)L.kpad, (cuuint64_t)L.npad};
             cuuint64_t strides[1] = {(cuuint64_t)L.kpad * 2};
@@ -183,6 +225,9 @@ xenos_status_t runtime_bind(Graph &g, void *ws, size_t bytes, void *stream_v) {
         if ((e = cudaFuncSetAttribute(xk::gemm_chain_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, optin)) != cudaSuccess ||
             (e = cudaFuncSetAttribute(xk::gemm_chain_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, optin)) != cudaSuccess)
             return cuda_fail(g, "cudaFuncSetAttribute(gemm)", e);
+    if (any_gemm2)
+        if ((e = cudaFuncSetAttribute(xk::chain2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin)) != cudaSuccess)
+            return cuda_fail(g, "cudaFuncSetAttribute(chain2)", e);
     if (max_chain_smem > 0)
         if ((e = cudaFuncSetAttribute(xk::f32_conv_conv_pool_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin)) != cudaSuccess)
             return cuda_fail(g, "cudaFuncSetAttribute(f32 chain)", e);
@@ -326,6 +371,41 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
         case LK_F32_SLICE: {
             long long total = (long long)N * L.K * L.H * L.W;
             xk::f32_slice_kernel<<<ew_grid(total, 256, sms), 256, 0, stream>>>((const float *)ptr(L.in0), (float *)ptr(L.out), N, L.K, L.H * L.W, L.C, L.out_coff);
+            break;
+        }
+        case LK_GEMM2: {
+            xk::Chain2Params p;
+            std::memset(&p, 0, sizeof p);
+            p.bias1 = (const float *)(ws + L.b_off); p.bias2 = (const float *)(ws + L.b2_off);
+            p.skip = (const __nv_bfloat16 *)ptr(L.skip); p.skip_ctot = L.skip >= 0 ? g.tensors[L.skip].c : 0;
+            p.out = (__nv_bfloat16 *)ptr(L.out); p.status = status;
+            p.batch = N; p.P = L.P; p.Q = L.Q;
+            p.k1 = L.k; p.pad1 = L.pad; p.cpb1 = L.C / 64; p.kblocks1 = L.kblocks;
+            p.k2 = L.k2; p.cpb2 = L.n1pad / 64; p.kblocks2 = L.kblocks2;
+            p.n1pad = L.n1pad; p.N2 = L.K; p.tile_n2 = L.tile_n; p.n2_tiles = L.n_tiles;
+            p.rh1 = L.patch_rh; p.rw1 = L.patch_rw; p.halo = L.halo2; p.rh2 = L.rh2; p.rw2 = L.rw2;
+            p.tiles_y = L.tiles_y; p.tiles_x = L.tiles_x; p.m_tiles = N * L.tiles_y * L.tiles_x;
+            p.stages = L.stages; p.stage_bytes = L.stage_bytes; p.a_box_bytes = L.a_box_bytes;
+            p.off_mid = L.off_mid; p.off_bar = L.off_bar;
+            p.act1 = L.act; p.act2 = L.act2; p.act3 = L.act3; p.out_ctot = L.out_ctot; p.out_coff = L.out_coff;
+            p.idesc1 = make_idesc(L.n1pad); p.idesc2 = make_idesc(L.tile_n);
+            p.launch_id = (int)li;
+            const CUtensorMap *tma = &rt->hmaps[li];
+            CUtensorMap tma_now;
+            if (g.tensors[L.in0].input_slot >= 0) {
+                xenos_status_t st = encode_chain2_input(g, rt, L, ptr(L.in0), N, &tma_now);
+                if (st != XENOS_OK) return st;
+                tma = &tma_now;
+            }
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3((unsigned)std::min(p.m_tiles, sms)); cfg.blockDim = dim3((unsigned)xk::kC2Threads);
+            cfg.dynamicSmemBytes = (size_t)L.smem_bytes; cfg.stream = stream;
+            cudaLaunchAttribute at[1];
+            at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            at[0].val.programmaticStreamSerializationAllowed = 1;
+            cfg.attrs = at; cfg.numAttrs = 1;
+            cudaError_t le = cudaLaunchKernelEx(&cfg, xk::chain2_kernel, *tma, rt->tmaps[li], rt->tmaps2[li], p);
+            if (le != cudaSuccess) return cuda_fail(g, "kernel launch", le);
             break;
         }
         case LK_GEMM: {

@@ -514,6 +514,55 @@ def test_bf16_operator_benchmarks(name, batch, launches, linked):
         assert gg.g.launch_count() == launches
 
 
+# ---- ConvX -> ConvY with the intermediate tile in shared memory ---------------------------------------------
+C2_CASES = [
+    # cin, hw, k1, pad1, cmid, k2, cout, add, batch
+    (256, 16, 1, 0, 64, 1, 256, True, 2),    # 1x1 -> 1x1 expand + identity shortcut, one N tile
+    (512, 12, 3, 1, 128, 1, 512, True, 3),   # bottleneck tail: 3x3 -> 1x1 expand + identity shortcut, two output-channel tiles from one middle tile
+    (64, 20, 1, 0, 64, 3, 64, False, 2),     # 1x1 -> 3x3: the producer tile carries the consumer's frame
+    (64, 14, 3, 1, 64, 3, 64, True, 2),      # basic block: 3x3 -> 3x3 + identity shortcut, ragged tiles
+    (128, 7, 3, 1, 256, 3, 96, False, 5),    # small maps (one image per tile), four middle blocks, ragged N
+    (64, 9, 5, 2, 192, 1, 40, False, 1),     # 5x5 -> 1x1
+    (64, 33, 3, 0, 64, 3, 32, False, 1),     # first convolution without padding: its output is smaller than its input
+]
+
+
+@pytest.mark.parametrize("case", C2_CASES)
+def test_bf16_conv_conv_on_chip(case):
+    cin, hw, k1, pad1, cmid, k2, cout, add, batch = case
+    def build(g):
+        y = g.cbr("c1", "input", cmid, k1, 1, pad1)
+        y = g.cbr("c2", y, cout, k2, 1, (k2 - 1) // 2, act=None if add else "relu")
+        if add:
+            y = g.add("add", y, "input")
+            g.act("relu", y, "relu")
+    spec = _one(build, cin, hw)
+    chain = ["c1", "c2"] + (["add"] if add else [])
+    if add and cout != cin:
+        pytest.skip("identity shortcut needs equal channel counts")
+    y, o, gg = check_bf16(f"conv_conv{case}", spec, batch, in_mode="bf16_nhwc", links=[chain])
+    pl = gg.g.plan()
+    assert gg.g.launch_count() == 1 and pl["launches"][0]["kind"] == "gemm2" and pl["chains"][0]["kind"] == "conv_conv"
+    yu, _, _ = check_bf16("conv_conv_unlinked", spec, batch, linked=False, in_mode="bf16_nhwc")
+    assert abs_err_scaled(y, yu) <= LINKED_VS_UNLINKED_TOL
+    x = xo.round_bf16(graphs.make_input(spec, batch))
+    assert np.array_equal(gg.run(x), y)
+
+
+@pytest.mark.parametrize("s,e,cin", [(16, 64, 64), (48, 192, 256), (64, 256, 128)])
+def test_bf16_fire_module_with_the_squeeze_on_chip(s, e, cin):
+    def build(g):
+        sq = g.cbr("sq", "input", s, 1, bn=False, bias=True)
+        e1 = g.cbr("e1", sq, e, 1, bn=False, bias=True)
+        e3 = g.cbr("e3", sq, e, 3, 1, 1, bn=False, bias=True)
+        g.concat("cat", [e1, e3])
+    spec = _one(build, cin, 13)
+    y, o, gg = check_bf16(f"fire_on_chip_s{s}", spec, 3, in_mode="bf16_nhwc", links=[["sq", "e1", "e3", "cat"]])
+    assert gg.g.launch_count() == 1 and gg.g.plan()["launches"][0]["kind"] == "gemm2"
+    yu, _, _ = check_bf16("fire_unlinked", spec, 3, linked=False, in_mode="bf16_nhwc")
+    assert abs_err_scaled(y, yu) <= LINKED_VS_UNLINKED_TOL
+
+
 # ---- the remaining operators of Table 3 and the MatmulX -> MatmulY link -----------------------------------
 def _matrix_ops_graph(precision):
     g = GraphSpec("matrix", (64, 24, 1), precision=precision)

@@ -172,6 +172,8 @@ def _classify(chain, nodes):
         return "dw-pw"
     if chain["kind"] == "expand_concat":
         return "fire"
+    if chain["kind"] == "conv_conv":      # the deeper form of a row: the first convolution's result stays on chip
+        return "fire" if "concat" in kinds else ("shortcut" if "add" in kinds else "conv-conv")
     if chain["kind"] == "conv_tail":
         if "add" in kinds:
             return "shortcut"
