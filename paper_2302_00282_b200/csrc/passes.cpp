@@ -179,7 +179,7 @@ static bool chain2_pays(const Graph &g, const Node &A, const Node &B, bool skip)
     const double in = px * A.cin * 2, midb = px * A.cout * 2, outb = px * B.cout * 2 * (skip ? 2 : 1);
     const double lin = std::max(2.0 * tiles * 128 * (k1 * A.cout + k2 * B.cout) / tc, (in + outb) / hbm);
     const double unl = std::max(2.0 * px * k1 * A.cout / tc, (in + midb) / hbm) + std::max(2.0 * px * k2 * B.cout / tc, (midb + outb) / hbm);
-    return lin < 0.95 * unl;
+    return lin <= 1.02 * unl;      // (when the model sees no difference the link still saves a launch and the bytes)
 }
 
 template <class Allowed>
@@ -303,6 +303,12 @@ static bool try_match(const LinkCtx &cx, int a, Allowed allowed, Chain &out, boo
             if (c >= 0 && allowed(c) && g.nodes[c].kind == NK_ADD && B.act == XENOS_ACT_NONE) {
                 int other = g.nodes[c].in[0] == B.out ? g.nodes[c].in[1] : g.nodes[c].in[0];
                 with_add = other != B.out;
+                // a shortcut with its own 1x1 convolution is better served by the shortcut row's link (that convolution
+                // joins ConvY's reduction and its result never exists): leave ConvY to it
+                int pj = with_add ? g.node_of_tensor[other] : -1;
+                if (by_model && pj >= 0 && pj != a && g.nodes[pj].kind == NK_CONV && g.nodes[pj].k == 1 && g.nodes[pj].pad == 0 &&
+                    g.nodes[pj].act == XENOS_ACT_NONE && cx.sole(pj) == c && g.nodes[pj].chain < 0 && B.k == 1)
+                    return false;
             }
             if (!by_model || chain2_pays(g, A, B, with_add)) {
                 out.kind = CK_CONV_CONV;

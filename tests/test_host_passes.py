@@ -192,6 +192,9 @@ def test_table1_patterns_are_found(name):
         if k:
             got[k] = got.get(k, 0) + 1
     want = _gold_counts()[name]
+    on_chip = want.pop("on-chip", None)
+    if on_chip is not None:
+        assert sum(c["kind"] == "conv_conv" for c in pl["chains"]) == on_chip
     if name == "mobilenet_v1":        # the last dw -> pw chain also absorbs the global average
         want = {"dw-pw": 13}
         assert sum("gap" in [pl["nodes"][i]["kind"] for i in c["nodes"]] for c in pl["chains"]) == 1
@@ -456,3 +459,29 @@ def test_matrix_operator_shapes_and_errors():
     pl = g.plan()
     tt = [n for n in pl["nodes"] if n["kind"] == "transpose"][0]
     assert tt["cin"] == 24 and tt["cout"] == 8               # (24 columns, 8 rows) -> (8 columns, 24 rows)
+
+
+def test_stress_graph_keeps_the_bottleneck_tails_on_chip():
+    """ConvX -> ConvY (3x3 -> 1x1 expand) + identity shortcut in one kernel for the blocks of stages 1-3 that have no
+    shortcut convolution; the blocks that have one keep the shortcut row's link; stage 4 (512 middle channels) does
+    not fit the accumulators."""
+    spec = graphs.resnet50_stress()
+    g, _ = compiled(spec, 64)
+    pl = g.plan()
+    cc = [c for c in pl["chains"] if c["kind"] == "conv_conv"]
+    assert len(cc) == _gold_counts()["resnet50_stress"]["on-chip"] and len(pl["launches"]) == 39
+    for c in cc:
+        kinds = [pl["nodes"][i]["kind"] for i in c["nodes"]]
+        L = pl["launches"][c["launches"][0]]
+        assert kinds == ["conv", "conv", "add"] and L["kind"] == "gemm2" and L["k"] == 3 and L["k2"] == 1 and L["skip"] >= 0
+        assert L["cmid"] in (64, 128, 256) and L["patch_rh"] * L["patch_rw"] <= 128 and (L["rh2"], L["rw2"]) == (L["patch_rh"], L["patch_rw"])
+    assert pl["bytes_linked"] <= 14.7e9
+    # explicit requests reach the chains the model declines: a basic block of ResNet-18, a fire module
+    r = graphs.resnet18()
+    g2, _ = compiled(r, 2, links=[["s1b1.c1", "s1b1.c2", "s1b1.add"]])
+    L = [l for l in g2.plan()["launches"] if l["kind"] == "gemm2"]
+    assert len(L) == 1 and (L[0]["k"], L[0]["k2"]) == (3, 3) and (L[0]["rh2"], L[0]["rw2"]) == (L[0]["patch_rh"] - 2, L[0]["patch_rw"] - 2)
+    q = graphs.squeezenet11()
+    g3, _ = compiled(q, 2, links=[["f3.sq", "f3.e1", "f3.e3", "f3.cat"]])
+    L = [l for l in g3.plan()["launches"] if l["kind"] == "gemm2"]
+    assert len(L) == 1 and L[0]["cmid"] == 32 and L[0]["n1pad"] == 64 and L[0]["K"] == 256
