@@ -475,7 +475,7 @@ def test_stress_graph_keeps_the_bottleneck_tails_on_chip():
         L = pl["launches"][c["launches"][0]]
         assert kinds == ["conv", "conv", "add"] and L["kind"] == "gemm2" and L["k"] == 3 and L["k2"] == 1 and L["skip"] >= 0
         assert L["cmid"] in (64, 128, 256) and L["patch_rh"] * L["patch_rw"] <= 128 and (L["rh2"], L["rw2"]) == (L["patch_rh"], L["patch_rw"])
-    assert pl["bytes_linked"] <= 14.7e9
+    assert pl["bytes_linked"] <= 14.8e9          # 15.9e9 before these links (fp32 image input)
     # explicit requests reach the chains the model declines: a basic block of ResNet-18, a fire module
     r = graphs.resnet18()
     g2, _ = compiled(r, 2, links=[["s1b1.c1", "s1b1.c2", "s1b1.add"]])
