@@ -1,0 +1,230 @@
+// Depthwise 3x3 -> pointwise 1x1 (Sections 2.2 and 4.1 of the Xenos paper: the depthwise result is produced in the
+// layout the pointwise product reads and never leaves the SM), as a kernel of its own for the chains that store
+// their tile.  It takes the same plan record and parameters as the depthwise mode of gemm_chain_kernel and differs
+// in how the warps are used: there are no separate producer and epilogue warps.  Every worker warp runs the
+// depthwise stencil of a tile's K blocks and then a share of the store epilogue of the previous tile, so that no
+// warp waits for another role's stage, and all warps of a scheduler run the same loop.
+//   warp 0   TMA: the tile's input window per 64-channel block (zero fill = padding), pointwise weight blocks
+//   warp 1   MMA: acc[128 x tile_n] += A block x W block, two accumulators in tensor memory
+//   workers  tile i + 1: stencil of every K block into the A|B ring; then tile i: bias, activation, bf16, store
+// With kW = 16 the 512 worker threads each own 1 x 4 output pixels of 4 channels of a 64-channel block; with
+// kW = 8 the 256 threads own 2 x 4 pixels (64-channel blocks) or 1 x 4 (narrower blocks).
+// Every wait is bounded; on expiry the role records XENOS_E_TIMEOUT and the workers leave together.
+#pragma once
+
+#include "gemm_tc.cuh"
+
+namespace xk {
+
+template <int kW>
+__global__ void __launch_bounds__(64 + 32 * kW, 1)
+dwpw_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmH, const GemmParams g) {
+    constexpr int kWorkerThreads = 32 * kW;
+    extern __shared__ uint8_t smem_raw[];
+    pdl_launch_dependents();
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t sbase = (raw + 1023u) & ~1023u;
+    uint8_t *sm = smem_raw + (sbase - raw);
+    const int stage_bytes = kABytes + g.tile_n * 128;
+    const uint32_t bar_base = sbase + g.off_bar;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (kMaxStages + s); };
+    auto accf_bar = [&](int b) { return bar_base + 8u * (2 * kMaxStages + b); };
+    auto acce_bar = [&](int b) { return bar_base + 8u * (2 * kMaxStages + 2 + b); };
+    auto hfull_bar = [&](int s) { return bar_base + 8u * (2 * kMaxStages + 4 + s); };
+    auto hempty_bar = [&](int s) { return bar_base + 8u * (2 * kMaxStages + 4 + kMaxHaloStages + s); };
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(sm + g.off_bar + 8 * (2 * kMaxStages + 4 + 2 * kMaxHaloStages));
+    volatile int *fail_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int total_tiles = g.m_tiles * g.n_tiles;
+    const int dw_quads = g.halo_cb > 32 ? 16 : 8;
+    const int dw_br = (g.halo_cb > 32 && kW == 8) ? 2 : 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < g.stages; ++s) { mbar_init(full_bar(s), kW + 1); mbar_init(empty_bar(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), kW); }
+        for (int s = 0; s < g.hstages; ++s) { mbar_init(hfull_bar(s), 1); mbar_init(hempty_bar(s), kW); }
+        *fail_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmH) : "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)g.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (warp >= 2) {
+        // depthwise tap weights [9][C] followed by the bias [C], fp32, once per CTA
+        const int C = g.seg[0].C;
+        float4 *dst = reinterpret_cast<float4 *>(sm + g.off_dww);
+        const float4 *w4 = reinterpret_cast<const float4 *>(g.seg[0].dw_w), *b4 = reinterpret_cast<const float4 *>(g.seg[0].dw_b);
+        for (int i = threadIdx.x - 64; i < 9 * C / 4; i += kWorkerThreads) dst[i] = __ldg(w4 + i);
+        for (int i = threadIdx.x - 64; i < C / 4; i += kWorkerThreads) dst[9 * C / 4 + i] = __ldg(b4 + i);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    bool ok = true;
+    if (warp != 1) pdl_wait();
+
+    if (warp == 0) {
+        if (lane == 0) {
+            TileWalk w;
+            w.init(g);
+            Ring st = {0, 0u}, hr = {0, 0u};
+            for (; w.ti < total_tiles && ok; w.next(g)) {
+                const int hn = w.grp * g.ni;
+                const int hy = (w.ty * g.step_y - g.off_y) * g.seg[0].stride - g.seg[0].pad;
+                const int hx = (w.tx * g.step_x - g.off_x) * g.seg[0].stride - g.seg[0].pad;
+                for (int kb = 0; kb < g.kblocks && ok; ++kb) {
+                    ok = mbar_wait(hempty_bar(hr.s), hr.ph ^ 1u);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(hfull_bar(hr.s), (uint32_t)g.halo_bytes);
+                    tma_load_4d(sbase + g.off_halo + hr.s * g.halo_stride, &tmH, kb * kTileK, hx, hy, hn, hfull_bar(hr.s));
+                    hr.next(g.hstages);
+                    ok = mbar_wait(empty_bar(st.s), st.ph ^ 1u);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(full_bar(st.s), (uint32_t)g.tile_n * 128u);
+                    tma_load_2d(sbase + st.s * stage_bytes + kABytes, &tmB, kb * kTileK, w.nt * g.tile_n, full_bar(st.s));
+                    st.next(g.stages);
+                }
+            }
+            if (!ok) atomicCAS(g.status, 0u, timeout_word(g, 1));
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            int i = 0;
+            Ring st = {0, 0u};
+            for (int ti = blockIdx.x; ti < total_tiles && ok; ti += gridDim.x, ++i) {
+                const int b = i & 1;
+                ok = mbar_wait(acce_bar(b), ((i >> 1) & 1) ^ 1u);      // the workers have drained this accumulator
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + b * g.acc_stride;
+                for (int kb = 0; kb < g.kblocks && ok; ++kb) {
+                    const int s = st.s;
+                    ok = mbar_wait(full_bar(s), st.ph);
+                    if (!ok) break;
+                    st.next(g.stages);
+                    fence_proxy_async();
+                    tc_fence_after();
+                    const uint32_t a = sbase + s * stage_bytes, bb = a + kABytes;
+#pragma unroll
+                    for (int k4 = 0; k4 < kTileK / 16; ++k4)
+                        umma_bf16(d_tmem, umma_desc_sw128(a + k4 * 32), umma_desc_sw128(bb + k4 * 32), g.idesc, (kb > 0 || k4 > 0) ? 1u : 0u);
+                    umma_commit(empty_bar(s));
+                }
+                if (ok) umma_commit(accf_bar(b));
+            }
+            if (!ok) atomicCAS(g.status, 0u, timeout_word(g, 2));
+        }
+    } else {
+        const int wt = threadIdx.x - 64;
+        const DwUnit du = make_dw_unit(g, wt, dw_quads, dw_br);
+        const int zero_from = g.halo_cb >> 3;
+        if (zero_from < 8) {
+            // K-padding chunks are only ever written with zeros: cleared once
+            const int nz = 8 - zero_from;
+            for (int idx = wt; idx < g.stages * kTileM * nz; idx += kWorkerThreads) {
+                const int sr = idx / nz, jj = zero_from + idx - sr * nz, s = sr / kTileM, row = sr - s * kTileM;
+                st_shared16(a_chunk_addr(sbase + s * stage_bytes, row, jj), make_uint4(0u, 0u, 0u, 0u));
+            }
+            fence_proxy_async();
+        }
+        const uint32_t dww = sbase + g.off_dww;
+        const GemmSeg &sg = g.seg[0];
+        const int quarter = warp & 3, cgroup = (warp - 2) >> 2;      // accumulator lanes; which 32-column chunks
+        const int row = quarter * 32 + lane;
+        const RowLocal rl = row_local(g, row);
+        const uint32_t plo = g.act >= 1 ? 0u : 0xff80ff80u, phi = g.act == 2 ? 0x40c040c0u : 0x7f807f80u;
+        const bool wide_ok = ((reinterpret_cast<uintptr_t>(g.out) | (uintptr_t)(g.out_ctot * 2) | (uintptr_t)(g.out_coff * 2)) & 31u) == 0;
+        Ring st = {0, 0u}, hr = {0, 0u};
+        auto stencil = [&]() {
+            for (int kb = 0; kb < g.kblocks && ok; ++kb) {
+                const int s = st.s, hs = hr.s;
+                ok = mbar_wait2_warp(empty_bar(s), st.ph ^ 1u, hfull_bar(hs), hr.ph, lane);
+                if (!ok) break;
+                st.next(g.stages); hr.next(g.hstages);
+                const uint32_t a_base = sbase + s * stage_bytes, halo = sbase + g.off_halo + hs * g.halo_stride;
+                if (kW == 8 && g.halo_cb > 32) {
+                    if (sg.stride == 1) produce_dw<1, 2>(sg, g, kb, halo, dww, du, a_base);
+                    else produce_dw<2, 2>(sg, g, kb, halo, dww, du, a_base);
+                } else {
+                    if (sg.stride == 1) produce_dw<1, 1>(sg, g, kb, halo, dww, du, a_base);
+                    else produce_dw<2, 1>(sg, g, kb, halo, dww, du, a_base);
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) { mbar_arrive(full_bar(s)); mbar_arrive(hempty_bar(hs)); }
+            }
+        };
+        TileWalk ws, we;
+        ws.init(g);
+        we.init(g);
+        if (ws.ti < total_tiles) { stencil(); ws.next(g); }
+        for (int i = 0; we.ti < total_tiles; we.next(g), ++i) {
+            if (ok && ws.ti < total_tiles) { stencil(); ws.next(g); }
+            const int b = i & 1, nt = we.nt, n0 = nt * g.tile_n;
+            // the bias slice of this tile's channels (two buffers: a warp is at most one tile ahead of the others)
+            if (wt * 4 < g.tile_n)
+                *reinterpret_cast<float4 *>(sm + g.off_bias + b * 1024 + wt * 16) = __ldg(reinterpret_cast<const float4 *>(g.bias + n0) + wt);
+            const uint32_t sbias = sbase + g.off_bias + b * 1024;
+            const RowPos rq = map_row(g, we, rl, row);
+            const size_t pix = ((size_t)rq.n * g.P + rq.p) * g.Q + rq.q;
+            // the workers share a named barrier, so they agree on giving up before any of them can miss it
+            if (ok) ok = mbar_wait_warp(accf_bar(b), (i >> 1) & 1, lane);
+            if (!ok && lane == 0) *fail_flag = 1;
+            asm volatile("bar.sync 1, %0;" ::"r"(kWorkerThreads) : "memory");
+            if (*fail_flag) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * g.acc_stride;
+            const int nc32 = (g.tile_n + 31) >> 5;
+            for (int c32 = cgroup; c32 < nc32; c32 += kW / 4) {
+                float v[32];
+                const bool whole = c32 * 32 + 32 <= g.tile_n;
+                if (whole) tmem_ld32(t_lane + c32 * 32, v);
+                else tmem_ld16(t_lane + c32 * 32, v);
+                if (c32 + kW / 4 >= nc32) {
+                    // this warp's last read of the accumulator
+                    tc_fence_before();
+                    warp_arrive(acce_bar(b), lane);
+                }
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    if (h == 1 && !whole) break;
+                    const int cl = c32 * 32 + h * 16, nc = n0 + cl;
+                    uint32_t pk[8];
+#pragma unroll
+                    for (int q4 = 0; q4 < 16; q4 += 4) {
+                        const float4 bz = ld_shared_f4(sbias + (uint32_t)(cl + q4) * 4u);
+                        const float2 t0 = __fadd2_rn(make_float2(v[h * 16 + q4], v[h * 16 + q4 + 1]), make_float2(bz.x, bz.y));
+                        const float2 t1 = __fadd2_rn(make_float2(v[h * 16 + q4 + 2], v[h * 16 + q4 + 3]), make_float2(bz.z, bz.w));
+                        pk[q4 / 2] = clamp_bf16x2(pack2(t0.x, t0.y), plo, phi);
+                        pk[q4 / 2 + 1] = clamp_bf16x2(pack2(t1.x, t1.y), plo, phi);
+                    }
+                    if (!rq.valid) continue;
+                    __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(g.out) + pix * g.out_ctot + g.out_coff + nc;
+                    if (nc + 16 <= g.N && wide_ok) {
+                        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(o), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]),
+                                     "r"(pk[3]), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7]) : "memory");
+                    } else {
+                        if (nc + 8 <= g.N) *reinterpret_cast<uint4 *>(o) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        if (nc + 16 <= g.N) *reinterpret_cast<uint4 *>(o + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                    }
+                }
+            }
+            if (cgroup >= nc32) warp_arrive(acce_bar(b), lane);       // a warp without a chunk in so narrow a tile
+        }
+        if (!ok && lane == 0) atomicCAS(g.status, 0u, timeout_word(g, 3));
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)g.tmem_cols) : "memory");
+    }
+}
+
+}  // namespace xk

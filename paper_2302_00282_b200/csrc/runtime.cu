@@ -13,6 +13,7 @@
 #include <vector>
 
 #include "chain2_tc.cuh"
+#include "dwpw_tc.cuh"
 #include "gemm_tc.cuh"
 #include "graph.hpp"
 #include "kernels_bf16.cuh"
@@ -225,6 +226,10 @@ xenos_status_t runtime_bind(Graph &g, void *ws, size_t bytes, void *stream_v) {
         if ((e = cudaFuncSetAttribute(xk::gemm_chain_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, optin)) != cudaSuccess ||
             (e = cudaFuncSetAttribute(xk::gemm_chain_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, optin)) != cudaSuccess)
             return cuda_fail(g, "cudaFuncSetAttribute(gemm)", e);
+    if (any_gemm)
+        if ((e = cudaFuncSetAttribute(xk::dwpw_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, optin)) != cudaSuccess ||
+            (e = cudaFuncSetAttribute(xk::dwpw_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, optin)) != cudaSuccess)
+            return cuda_fail(g, "cudaFuncSetAttribute(dwpw)", e);
     if (any_gemm2)
         if ((e = cudaFuncSetAttribute(xk::chain2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin)) != cudaSuccess)
             return cuda_fail(g, "cudaFuncSetAttribute(chain2)", e);
@@ -484,14 +489,17 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
             // stream drains, runs its set-up (barriers, tensor memory, constant staging) and then
             // waits (griddepcontrol.wait) before it touches any activation.
             cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3((unsigned)xk::kThreads);
+            cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3((unsigned)L.block);
             cfg.dynamicSmemBytes = (size_t)L.smem_bytes; cfg.stream = stream;
             cudaLaunchAttribute at[1];
             at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
             at[0].val.programmaticStreamSerializationAllowed = 1;
             cfg.attrs = at; cfg.numAttrs = 1;
-            cudaError_t le = L.ksplit > 1 ? cudaLaunchKernelEx(&cfg, xk::gemm_chain_kernel<1>, rt->tmaps[li], *tmh, p)
-                                          : cudaLaunchKernelEx(&cfg, xk::gemm_chain_kernel<0>, rt->tmaps[li], *tmh, p);
+            cudaError_t le;
+            if (L.dw_workers == 16) le = cudaLaunchKernelEx(&cfg, xk::dwpw_kernel<16>, rt->tmaps[li], *tmh, p);
+            else if (L.dw_workers == 8) le = cudaLaunchKernelEx(&cfg, xk::dwpw_kernel<8>, rt->tmaps[li], *tmh, p);
+            else if (L.ksplit > 1) le = cudaLaunchKernelEx(&cfg, xk::gemm_chain_kernel<1>, rt->tmaps[li], *tmh, p);
+            else le = cudaLaunchKernelEx(&cfg, xk::gemm_chain_kernel<0>, rt->tmaps[li], *tmh, p);
             if (le != cudaSuccess) return cuda_fail(g, "kernel launch", le);
             break;
         }

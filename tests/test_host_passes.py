@@ -346,13 +346,13 @@ def test_reduction_split_is_automatic_only_where_units_would_idle():
     spec = graphs.mobilenet_v1()
     g, _ = compiled(spec, 32)
     L = g.plan()["launches"]
-    assert [l["ksplit"] for l in L[:-1]] == [1] * (len(L) - 1)
+    assert [l.get("ksplit", 1) for l in L[:-1]] == [1] * (len(L) - 1)
     fc = L[-1]
     assert fc["ksplit"] >= 2 and fc["m_tiles"] * fc["n_tiles"] * fc["ksplit"] <= 148 and fc["kb_per"] >= 2
     # a depthwise -> pointwise chain is cut on request only
     g1, ids = compiled(spec, 1, splits=[("pw7.relu6", dict(parts_k=8))])
     L1 = g1.plan()["launches"]
-    assert [l["ksplit"] for l in L1 if l.get("a0") == "dw"].count(8) == 1
+    assert [l.get("ksplit", 1) for l in L1 if l.get("a0") == "dw"].count(8) == 1
     assert all(l["ksplit"] == 1 for l in L1 if l.get("a0") == "stem" or l.get("epi") in (1, 2))
 
 
