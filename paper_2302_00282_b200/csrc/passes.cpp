@@ -832,6 +832,12 @@ struct Lower {
             // while SMs would stay idle, fewer images per tile spread it over more of them
             while (L.ni > 1 && (long)ceil_div(g.max_batch, L.ni) * ceil_div(round_up(N, 16), 256) * 2 <= g.hw.sm_count) --L.ni;
             while (!gapn && L.patch_rh > 1 && halo_of(L.ni, L.patch_rh, L.patch_rw) > 76 * 1024) --L.patch_rh;
+            // Small batches leave most units idle while each tile's depthwise stage runs its K blocks one after the
+            // other, at a pace set by the pixels per tile: while at least half of the units would stay idle, halve the
+            // tile's rows (the MMA tile is then partly empty, which costs nothing there).
+            while (!gapn && L.ni == 1 && L.patch_rh > 1 &&
+                   (long)g.max_batch * ceil_div(L.P, (L.patch_rh + 1) / 2) * ceil_div(L.Q, L.patch_rw) * ceil_div(round_up(N, 16), 256) * 2 <= g.hw.sm_count)
+                L.patch_rh = (L.patch_rh + 1) / 2;
             L.tiles_y = ceil_div(L.P, L.patch_rh); L.tiles_x = ceil_div(L.Q, L.patch_rw);
             L.step_y = L.patch_rh; L.step_x = L.patch_rw; L.off_y = L.off_x = 0;
             L.tile_rows = L.ni * L.patch_rh * L.patch_rw;
@@ -866,7 +872,8 @@ struct Lower {
             L.tile_n = round_up(ceil_div(N16, L.n_tiles), 16);
             // kernels are dealt to idle units first: halve the channel tile while units stay idle
             // (a linked depthwise stage is recomputed per channel tile, so it stops halving earlier)
-            const int min_tile_n = dw ? 256 : 32;
+            // (unless most units are idle anyway: then narrower channel tiles shorten every CTA's weight loads and store)
+            const int min_tile_n = dw ? ((long)L.m_tiles * L.n_tiles * 4 <= g.hw.sm_count ? 64 : 256) : 32;
             while (L.m_tiles * L.n_tiles < g.hw.sm_count && L.tile_n >= 2 * min_tile_n) {
                 int nt = L.n_tiles * 2, tn = round_up(ceil_div(N16, nt), 16);
                 if ((nt - 1) * tn >= N) break;
