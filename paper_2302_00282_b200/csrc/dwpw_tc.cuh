@@ -25,7 +25,8 @@ dwpw_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUt
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t sbase = (raw + 1023u) & ~1023u;
     uint8_t *sm = smem_raw + (sbase - raw);
-    const int stage_bytes = kABytes + g.tile_n * 128;
+    const int cols = g.n_acc * g.tile_n;                  // columns of a CTA's tile (n_acc = 2: both accumulators, 2 x 256)
+    const int stage_bytes = kABytes + cols * 128;
     const uint32_t bar_base = sbase + g.off_bar;
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto empty_bar = [&](int s) { return bar_base + 8u * (kMaxStages + s); };
@@ -86,8 +87,9 @@ dwpw_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUt
                     hr.next(g.hstages);
                     ok = mbar_wait(empty_bar(st.s), st.ph ^ 1u);
                     if (!ok) break;
-                    mbar_arrive_expect_tx(full_bar(st.s), (uint32_t)g.tile_n * 128u);
-                    tma_load_2d(sbase + st.s * stage_bytes + kABytes, &tmB, kb * kTileK, w.nt * g.tile_n, full_bar(st.s));
+                    mbar_arrive_expect_tx(full_bar(st.s), (uint32_t)cols * 128u);
+                    for (int h = 0; h < g.n_acc; ++h)
+                        tma_load_2d(sbase + st.s * stage_bytes + kABytes + h * g.tile_n * 128, &tmB, kb * kTileK, (w.nt * g.n_acc + h) * g.tile_n, full_bar(st.s));
                     st.next(g.stages);
                 }
             }
@@ -111,9 +113,11 @@ dwpw_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUt
                     fence_proxy_async();
                     tc_fence_after();
                     const uint32_t a = sbase + s * stage_bytes, bb = a + kABytes;
+                    for (int h = 0; h < g.n_acc; ++h)
 #pragma unroll
-                    for (int k4 = 0; k4 < kTileK / 16; ++k4)
-                        umma_bf16(d_tmem, umma_desc_sw128(a + k4 * 32), umma_desc_sw128(bb + k4 * 32), g.idesc, (kb > 0 || k4 > 0) ? 1u : 0u);
+                        for (int k4 = 0; k4 < kTileK / 16; ++k4)
+                            umma_bf16(d_tmem + h * g.acc_stride, umma_desc_sw128(a + k4 * 32), umma_desc_sw128(bb + h * g.tile_n * 128 + k4 * 32), g.idesc,
+                                      (kb > 0 || k4 > 0) ? 1u : 0u);
                     umma_commit(empty_bar(s));
                 }
                 if (ok) umma_commit(accf_bar(b));
@@ -166,11 +170,13 @@ dwpw_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUt
         if (ws.ti < total_tiles) { stencil(); ws.next(g); }
         for (int i = 0; we.ti < total_tiles; we.next(g), ++i) {
             if (ok && ws.ti < total_tiles) { stencil(); ws.next(g); }
-            const int b = i & 1, nt = we.nt, n0 = nt * g.tile_n;
+            const int b = i & 1, nt = we.nt, n0 = nt * cols;
             // the bias slice of this tile's channels (two buffers: a warp is at most one tile ahead of the others)
-            if (wt * 4 < g.tile_n)
-                *reinterpret_cast<float4 *>(sm + g.off_bias + b * 1024 + wt * 16) = __ldg(reinterpret_cast<const float4 *>(g.bias + n0) + wt);
-            const uint32_t sbias = sbase + g.off_bias + b * 1024;
+            // (a 512-column tile is its CTA's only tile and takes both buffers)
+            const int bbuf = g.n_acc == 2 ? 0 : b;
+            if (wt * 4 < cols)
+                *reinterpret_cast<float4 *>(sm + g.off_bias + bbuf * 1024 + wt * 16) = __ldg(reinterpret_cast<const float4 *>(g.bias + n0) + wt);
+            const uint32_t sbias = sbase + g.off_bias + bbuf * 1024;
             const RowPos rq = map_row(g, we, rl, row);
             const size_t pix = ((size_t)rq.n * g.P + rq.p) * g.Q + rq.q;
             // the workers share a named barrier, so they agree on giving up before any of them can miss it
@@ -180,10 +186,10 @@ dwpw_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUt
             if (*fail_flag) { ok = false; break; }
             tc_fence_after();
             const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * g.acc_stride;
-            const int nc32 = (g.tile_n + 31) >> 5;
+            const int nc32 = (cols + 31) >> 5;
             for (int c32 = cgroup; c32 < nc32; c32 += kW / 4) {
                 float v[32];
-                const bool whole = c32 * 32 + 32 <= g.tile_n;
+                const bool whole = c32 * 32 + 32 <= cols;
                 if (whole) tmem_ld32(t_lane + c32 * 32, v);
                 else tmem_ld16(t_lane + c32 * 32, v);
                 if (c32 + kW / 4 >= nc32) {

@@ -93,6 +93,7 @@ struct GemmParams {
     float *split_part;
     unsigned int *split_cnt;
     int launch_id;                                  // position of this launch in the plan, reported with a give-up
+    int n_acc;                                      // dwpw_kernel: channel tiles per CTA (2: one 512-column tile in both accumulators)
 };
 
 // Status word of a wait that gave up: the code, the role that waited (1 TMA, 2 MMA, 3 producer, 4 producer helping

@@ -138,6 +138,7 @@ struct Launch {
     int stem_tma = 0, stem_align = 1;                              // stem: image patch by TMA, x alignment in elements
     int a_tma = 0, a_box_bytes = 0;                                // activation operand by TMA: 1 matrix rows, 2 shifted patch
     int dw_workers = 0;                                            // > 0: depthwise -> pointwise in dwpw_kernel with that many worker warps
+    int n_acc = 1;                                                 // dwpw_kernel: channel tiles of tile_n columns per CTA (2: both accumulators hold one tile)
     // ---- two linked convolutions (LK_GEMM2): producer tile rh1 x rw1 = patch_rh x patch_rw, consumer tile rh2 x rw2
     int k2 = 1, kblocks2 = 0, n1pad = 0, halo2 = 0, rh2 = 0, rw2 = 0, act3 = 0, off_mid = 0, stage_bytes = 0;
     int off_halo = 0, off_stg = 0, off_dww = 0, off_bias = 0, off_bar = 0;                    // shared-memory layout

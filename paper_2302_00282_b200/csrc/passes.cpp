@@ -907,13 +907,34 @@ struct Lower {
                 if (L.ksplit < 2) { L.ksplit = 1; L.kb_per = 0; }
             }
         }
+        // A depthwise -> pointwise chain with at most one tile per CTA and two 256-wide channel tiles: one CTA keeps both
+        // channel tiles of its pixels (the two accumulators hold one 512-column tile; with a single tile per CTA
+        // nothing is double-buffered anyway), so the depthwise stage is computed once per pixel tile instead of once
+        // per channel tile, and the tiles get fewer rows until they cover the units again.
+        if (dw && L.epi == EPI_STORE && L.ksplit == 1 && s1.mode == AM_NONE && !rq.user && L.ni == 1 && L.tile_n == 256 &&
+            L.n_tiles % 2 == 0 && L.halo_cb == 64 && (long)L.m_tiles * L.n_tiles <= g.hw.sm_count) {
+            const int nt2 = L.n_tiles / 2;
+            int th = L.patch_rh;
+            for (int t = 1; t <= L.patch_rh; ++t)
+                if ((long)g.max_batch * ceil_div(L.P, t) * L.tiles_x * nt2 <= g.hw.sm_count) { th = t; break; }
+            const int hh = (th - 1) * dw->stride + 3;
+            const int hstride = (int)align_up((size_t)hh * L.halo_w * 128, 128);
+            const int room2 = std::min(g.hw.smem_bytes_per_cta, 227 * 1024) - 1024 - 256 - 2048 - (int)align_up((size_t)40 * src.c, 128);
+            if (2 * (16384 + 2 * 256 * 128) + 2 * hstride <= room2) {
+                L.n_acc = 2; L.n_tiles = nt2;
+                L.patch_rh = th; L.tiles_y = ceil_div(L.P, th); L.step_y = th;
+                L.tile_rows = th * L.patch_rw;
+                L.halo_h = hh; L.halo_bytes = hh * L.halo_w * 128; L.halo_stride = hstride;
+                L.m_tiles = g.max_batch * L.tiles_y * L.tiles_x;
+            }
+        }
         // two accumulators in tensor memory so the epilogue of one tile overlaps the MMAs of the next
         L.acc_stride = round_up(L.tile_n, 32);
         L.tmem_cols = 32;
         while (L.tmem_cols < 2 * L.acc_stride) L.tmem_cols *= 2;
         if (L.tmem_cols > g.hw.tmem_columns) return fail(g, XENOS_E_BAD_SPLIT, "split: accumulator tiles exceed tensor memory columns");
         // shared memory of the one persistent CTA per SM: [A|B ring][halo ring][epilogue staging][barriers]
-        int stage_bytes = 16384 + L.tile_n * 128;
+        int stage_bytes = 16384 + L.n_acc * L.tile_n * 128;
         int stg_bytes = L.epi == EPI_POOL ? 128 * (L.tile_n * 2 + 16) : (L.epi == EPI_GAP ? 128 * 33 * 4 + 512 : 0);
         stg_bytes = (int)align_up((size_t)stg_bytes, 128);
         // depthwise tap weights + bias of the linked stage (fp32 [10][C]) and two bias slices of the GEMM
@@ -1365,7 +1386,7 @@ void emit_plan_json(Graph &g) {
             jint(s, "ni", L.ni); jint(s, "step_y", L.step_y); jint(s, "step_x", L.step_x); jint(s, "off_y", L.off_y); jint(s, "off_x", L.off_x);
             jint(s, "hstages", L.hstages); jint(s, "halo_h", L.halo_h); jint(s, "halo_w", L.halo_w); jint(s, "halo_cb", L.halo_cb);
             jint(s, "halo_bytes", L.halo_bytes);
-            jint(s, "ksplit", L.ksplit); jint(s, "kb_per", L.kb_per); jint(s, "a_tma", L.a_tma); jint(s, "dw_workers", L.dw_workers);
+            jint(s, "ksplit", L.ksplit); jint(s, "kb_per", L.kb_per); jint(s, "a_tma", L.a_tma); jint(s, "dw_workers", L.dw_workers); jint(s, "n_acc", L.n_acc);
         }
         if (L.kind == LK_GEMM2) {
             jint(s, "k2", L.k2); jint(s, "cmid", L.Cmid); jint(s, "n1pad", L.n1pad); jint(s, "kblocks", L.kblocks); jint(s, "kblocks2", L.kblocks2);

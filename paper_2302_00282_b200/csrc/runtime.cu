@@ -444,6 +444,7 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
             p.stem_tma = L.stem_tma; p.stem_align = L.stem_align;
             p.a_tma = L.a_tma; p.a_box_bytes = L.a_box_bytes; p.a_cpb = L.seg[0].C / 64;
             p.off_halo = L.off_halo; p.off_stg = L.off_stg; p.off_dww = L.off_dww; p.off_bias = L.off_bias; p.off_bar = L.off_bar;
+            p.n_acc = L.n_acc;
             p.act = L.act; p.act2 = L.act2; p.epi = L.epi; p.out_ctot = L.out_ctot; p.out_coff = L.out_coff;
             p.out_f32 = L.out_dtype == XENOS_DTYPE_F32;
             p.idesc = make_idesc(L.tile_n);

@@ -226,6 +226,21 @@ def test_bf16_dw_pw(c, cout, hw, stride, batch, linked):
     assert gg.g.launch_count() == (1 if linked else 2)
 
 
+# one CTA per pixel tile keeps two 256-wide channel tiles in the two accumulators (512 and 1024 output channels,
+# stride 1 and 2, tiles that end inside the feature map, a last tile with fewer rows)
+@pytest.mark.parametrize("c,cout,hw,stride,batch", [(512, 512, 14, 1, 3), (128, 1024, 13, 2, 2), (64, 512, 30, 1, 1), (256, 520, 14, 1, 16), (512, 512, 14, 1, 32),
+                                                   (128, 1024, 14, 2, 30)])
+def test_bf16_dw_pw_two_accumulators(c, cout, hw, stride, batch):
+    def build(g):
+        x = g.cbr("dw", "input", c, 3, stride, 1, groups=c, act="relu6")
+        g.cbr("pw", x, cout, 1, act="relu6")
+    spec = _one(build, c, hw)
+    _, _, gg = check_bf16(f"dw_pw_2acc{(c, cout, hw, stride)}", spec, batch, linked=True, in_mode="bf16_nhwc",
+                          images=None if batch <= 16 else [0, batch // 2 - 1, batch - 1])
+    L = gg.g.plan()["launches"]
+    assert len(L) == 1 and L[0]["n_acc"] == (2 if cout % 512 == 0 else 1) and L[0]["dw_workers"] == 16
+
+
 def test_bf16_dw_pw_gap_fc():
     def build(g):
         x = g.cbr("dw", "input", 64, 3, 1, 1, groups=64, act="relu6")

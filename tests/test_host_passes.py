@@ -289,9 +289,10 @@ def test_gemm_split_prefers_output_channels_until_units_are_busy():
             if L["kind"] != "gemm":
                 continue
             assert L["tile_n"] % 16 == 0 and 16 <= L["tile_n"] <= 256
-            assert L["npad"] == L["tile_n"] * L["n_tiles"] and (L["n_tiles"] - 1) * L["tile_n"] < L["K"] <= L["npad"]
+            cols = L["tile_n"] * L["n_acc"]                   # columns of a CTA's tile
+            assert L["npad"] == cols * L["n_tiles"] and (L["n_tiles"] - 1) * cols < L["K"] <= L["npad"]
             assert L["grid"] == min(148, L["m_tiles"] * L["n_tiles"] * L["ksplit"])     # one persistent CTA per unit
-            if L["n_tiles"] > -(-L["K"] // 256):               # split finer than the 256-wide maximum
+            if L["n_tiles"] * L["n_acc"] > -(-L["K"] // 256):  # split finer than the 256-wide maximum
                 assert L["m_tiles"] * (L["n_tiles"] // 2) < 148   # ... only because units would idle otherwise
                 if L["a0"] == "dw":
                     # a linked depthwise stage is recomputed per channel tile: narrow tiles only while at least three
