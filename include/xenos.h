@@ -269,6 +269,24 @@ XENOS_API xenos_status_t xenos_graph_selftest_wait_expiry(xenos_graph_t *g, void
 XENOS_API xenos_status_t xenos_graph_get_plan(const xenos_graph_t *g, char *json, size_t cap,
                                               size_t *needed);
 
+/* Graph image (Section 6: the optimiser's output is an executable of the optimised model that is stored and later
+ * handed to the runtime; Section 3: it takes the place of the original model file).
+ * xenos_graph_save writes g as one self-contained byte string into host_buf (host memory, capacity cap bytes) and
+ * sets *needed to its length; with host_buf == NULL it only reports the length.  The image holds the hardware
+ * description, every tensor and operator with its parameters, the link and split requests and, if g has been
+ * compiled, the compile options.  It holds no pointer and no device address.  g is not changed and may be in any
+ * state.  Errors: XENOS_E_INVALID (needed is NULL, buffer too small).
+ * xenos_graph_load builds a new graph (owned by the library, release with xenos_graph_destroy) from the bytes bytes
+ * at host_buf.  If the saved graph was compiled, the new one is compiled with the same options (planning is
+ * deterministic: its plan equals the saved graph's byte for byte) and *workspace_bytes, when not NULL, receives the
+ * workspace it needs; otherwise the graph is returned in build state and *workspace_bytes is 0.  The caller binds a
+ * workspace as usual.  Errors: XENOS_E_INVALID for anything that is not an intact image of this library version
+ * (bad magic, version, checksum, counts or indices), or the status of the failing compile; *out is NULL then and
+ * xenos_last_error(NULL) holds the message. */
+XENOS_API xenos_status_t xenos_graph_save(const xenos_graph_t *g, void *host_buf, size_t cap, size_t *needed);
+XENOS_API xenos_status_t xenos_graph_load(const void *host_buf, size_t bytes, xenos_graph_t **out,
+                                          size_t *workspace_bytes);
+
 /* Number of kernel launches one xenos_graph_run enqueues (valid after compile). */
 XENOS_API xenos_status_t xenos_graph_launch_count(const xenos_graph_t *g, int32_t *launches);
 

@@ -43,7 +43,7 @@ class OpDesc(ctypes.Structure):
 
 EXPORTS = ["xenos_graph_create", "xenos_graph_add_input", "xenos_graph_add_op", "xenos_graph_mark_output",
            "xenos_graph_link", "xenos_graph_split", "xenos_graph_search_split", "xenos_graph_compile", "xenos_graph_bind", "xenos_graph_run",
-           "xenos_graph_profile", "xenos_graph_run_builtin_scratch", "xenos_graph_status", "xenos_graph_selftest_wait_expiry", "xenos_graph_get_plan", "xenos_graph_launch_count", "xenos_graph_destroy",
+           "xenos_graph_profile", "xenos_graph_run_builtin_scratch", "xenos_graph_status", "xenos_graph_selftest_wait_expiry", "xenos_graph_get_plan", "xenos_graph_launch_count", "xenos_graph_save", "xenos_graph_load", "xenos_graph_destroy",
            "xenos_last_error"]
 
 _lib = None
@@ -73,6 +73,8 @@ def lib() -> ctypes.CDLL:
         L.xenos_graph_selftest_wait_expiry.argtypes = [vp, vp]
         L.xenos_graph_get_plan.argtypes = [vp, ctypes.c_char_p, sz, ctypes.POINTER(sz)]
         L.xenos_graph_launch_count.argtypes = [vp, ctypes.POINTER(i32)]
+        L.xenos_graph_save.argtypes = [vp, vp, sz, ctypes.POINTER(sz)]
+        L.xenos_graph_load.argtypes = [vp, sz, ctypes.POINTER(vp), ctypes.POINTER(sz)]
         L.xenos_graph_destroy.argtypes = [vp]
         L.xenos_last_error.argtypes = [vp]
         L.xenos_last_error.restype = ctypes.c_char_p
@@ -198,6 +200,26 @@ class Graph:
         buf = ctypes.create_string_buffer(n.value)
         self._check(lib().xenos_graph_get_plan(self._h, buf, n.value, ctypes.byref(n)))
         return buf.value.decode()
+
+    def save(self) -> bytes:
+        n = ctypes.c_size_t()
+        self._check(lib().xenos_graph_save(self._h, None, 0, ctypes.byref(n)))
+        buf = ctypes.create_string_buffer(n.value)
+        self._check(lib().xenos_graph_save(self._h, buf, n.value, ctypes.byref(n)))
+        return buf.raw[:n.value]
+
+    @classmethod
+    def load(cls, image: bytes):
+        """Returns (graph, workspace_bytes); workspace_bytes is 0 when the saved graph had not been compiled."""
+        g = cls.__new__(cls)
+        g._h = ctypes.c_void_p()
+        g._keep = []
+        n = ctypes.c_size_t()
+        buf = ctypes.create_string_buffer(image, len(image))
+        rc = lib().xenos_graph_load(buf, len(image), ctypes.byref(g._h), ctypes.byref(n))
+        if rc != XENOS_OK:
+            raise XenosError(rc, lib().xenos_last_error(None).decode())
+        return g, n.value
 
     def launch_count(self) -> int:
         n = ctypes.c_int32()

@@ -8,7 +8,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libxenos.so")
-SOURCES = ["api.cpp", "graph.cpp", "passes.cpp", "search.cpp", "runtime.cu"]
+SOURCES = ["api.cpp", "graph.cpp", "passes.cpp", "search.cpp", "serialize.cpp", "runtime.cu"]
 
 
 def _nvcc() -> str:

@@ -252,6 +252,55 @@ xenos_status_t xenos_graph_compile(xenos_graph_t *gp, int32_t max_batch, int32_t
     XENOS_GUARD_END(gp)
 }
 
+xenos_status_t xenos_graph_save(const xenos_graph_t *gp, void *host_buf, size_t cap, size_t *needed) {
+    if (!gp) return XENOS_E_INVALID;
+    const Graph &g = gp->g;
+    try {
+        if (!needed) return fail(g, XENOS_E_INVALID, "save: needed is NULL");
+        std::vector<uint8_t> img;
+        save_graph(g, img);
+        *needed = img.size();
+        if (!host_buf) return XENOS_OK;              // size query
+        if (cap < img.size()) return fail(g, XENOS_E_INVALID, "save: the buffer is smaller than the image");
+        std::memcpy(host_buf, img.data(), img.size());
+        return XENOS_OK;
+    } catch (const std::exception &e) {
+        return fail(g, XENOS_E_INVALID, std::string("save: ") + e.what());
+    }
+}
+
+xenos_status_t xenos_graph_load(const void *host_buf, size_t bytes, xenos_graph_t **out, size_t *workspace_bytes) {
+    if (!out) {
+        g_create_err = "xenos_graph_load: out is NULL";
+        return XENOS_E_INVALID;
+    }
+    *out = nullptr;
+    xenos_graph_t *gp = nullptr;
+    xenos_status_t st = xenos_graph_create(nullptr, &gp);
+    if (st != XENOS_OK) return st;
+    try {
+        Graph &g = gp->g;
+        bool compiled = false;
+        st = load_graph(g, static_cast<const uint8_t *>(host_buf), bytes, &compiled);
+        if (st == XENOS_OK && compiled) {
+            size_t wsb = 0;
+            st = xenos_graph_compile(gp, g.max_batch, g.precision, &wsb);
+            if (st == XENOS_OK && workspace_bytes) *workspace_bytes = wsb;
+        } else if (st == XENOS_OK && workspace_bytes) *workspace_bytes = 0;
+        if (st != XENOS_OK) {
+            g_create_err = std::string("xenos_graph_load: ") + g.err;
+            delete gp;
+            return st;
+        }
+    } catch (const std::exception &e) {
+        g_create_err = std::string("xenos_graph_load: ") + e.what();
+        delete gp;
+        return XENOS_E_INVALID;
+    }
+    *out = gp;
+    return XENOS_OK;
+}
+
 xenos_status_t xenos_graph_bind(xenos_graph_t *gp, void *workspace_dev, size_t bytes, void *cuda_stream) {
     if (!gp) return XENOS_E_INVALID;
     XENOS_GUARD_BEGIN

@@ -220,6 +220,9 @@ uint16_t f32_to_bf16_rne(float f);
 // search.cpp
 xenos_status_t search_splits(Graph &g, int max_batch, int precision, void *ws, size_t ws_bytes, const void *const *in,
                              void *const *out, void *stream, int max_trials, int repeats, std::string &report);
+// serialize.cpp
+void save_graph(const Graph &g, std::vector<uint8_t> &out);
+xenos_status_t load_graph(Graph &g, const uint8_t *buf, size_t bytes, bool *compiled);
 // runtime.cu
 xenos_status_t runtime_bind(Graph &g, void *ws, size_t bytes, void *stream);
 xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *const *out, void *stream,

@@ -678,3 +678,24 @@ def test_bf16_stress_graph_block_at_full_size_against_the_rounding_oracle(linked
         g.act("relu", y, "relu")
     spec = _one(build, 64, 128)
     check_bf16("cfg4_block_n2", spec, 2, linked=linked, in_mode="bf16_nhwc", emulated=True)
+
+
+# ---- graph image: a loaded graph is the saved graph -----------------------------------------------------------------
+@pytest.mark.parametrize("name", ["mobilenet_v1", "squeezenet11"])
+def test_loaded_graph_image_computes_the_same_bits(name):
+    import torch
+    from paper_2302_00282_b200 import binding as xb
+    spec = getattr(graphs, name)(hw=64, classes=24) if name != "mobilenet_v1" else graphs.mobilenet_v1(hw=64, width=0.5, classes=24)
+    P = graphs.make_params(spec)
+    x = graphs.make_input(spec, 3)
+    gg = GpuGraph(spec, P, 3, linked=True)
+    y = gg.run(x)
+    g2, need = xb.Graph.load(gg.g.save())
+    assert need == gg.g.plan()["workspace_bytes"]
+    ws = torch.empty(max(need, 256), dtype=torch.uint8, device="cuda")
+    ws.fill_(0xFF)
+    g2.bind(ws.data_ptr(), ws.numel(), gg.stream)
+    xin, out = gg.upload(x), gg.alloc_out(3)
+    g2.run(3, [xin.data_ptr()], [out.data_ptr()], gg.stream)
+    g2.status(gg.stream)
+    assert gg.vec and np.array_equal(out.float().cpu().numpy(), y)

@@ -488,3 +488,69 @@ def test_stress_graph_keeps_the_bottleneck_tails_on_chip():
     g3, _ = compiled(q, 2, links=[["f3.sq", "f3.e1", "f3.e3", "f3.cat"]])
     L = [l for l in g3.plan()["launches"] if l["kind"] == "gemm2"]
     assert len(L) == 1 and L[0]["cmid"] == 32 and L[0]["n1pad"] == 64 and L[0]["K"] == 256
+
+
+# ---- graph image (Section 6: the optimised model as a stored executable) ---------------------------------------
+def _fnv1a(b: bytes) -> int:
+    h = 1469598103934665603
+    for x in b:
+        h = ((h ^ x) * 1099511628211) & 0xFFFFFFFFFFFFFFFF
+    return h
+
+
+@pytest.mark.parametrize("name,batch", [("single_chain", 1), ("mobilenet_v1", 4), ("resnet18", 2), ("squeezenet11", 2)])
+def test_graph_image_round_trip_gives_the_same_plan(name, batch):
+    spec = getattr(graphs, name)()
+    g, _ = compiled(spec, batch)
+    img = g.save()
+    g2, ws = xb.Graph.load(img)
+    assert g2.plan_text() == g.plan_text()          # same chains, tiles, offsets and packed parameters' layout
+    assert ws == g.plan()["workspace_bytes"]
+    assert g2.save() == img                         # the image of the loaded graph is the same bytes
+
+
+def test_graph_image_keeps_requests_and_build_state():
+    spec = graphs.mobilenet_v1(hw=64, width=0.5, classes=16)
+    P = graphs.make_params(spec)
+    g, ids = graph_from_spec(spec, P)
+    g.link([ids["dw3"], ids["pw3"]])
+    g.split(ids["pw3.relu6"], parts_outc=2)
+    g2, ws = xb.Graph.load(g.save())                # saved before compile: comes back in build state
+    assert ws == 0
+    with pytest.raises(xb.XenosError) as e:
+        g2.plan()
+    assert e.value.code == xb.E_STATE
+    g.compile(2, xb.PRECISION_BF16_TENSOR)
+    g2.compile(2, xb.PRECISION_BF16_TENSOR)
+    assert g2.plan_text() == g.plan_text()
+    L = [l for l in g2.plan()["launches"] if l.get("a0") == "dw"]
+    assert len(L) == 1 and L[0]["n_tiles"] == 2     # the one explicit link, with its explicit split
+
+
+def test_graph_image_rejects_what_is_not_an_intact_image():
+    g, _ = compiled(graphs.single_chain(), 1)
+    img = g.save()
+    def bad(b):
+        with pytest.raises(xb.XenosError) as e:
+            xb.Graph.load(b)
+        assert e.value.code == xb.E_INVALID
+    bad(b"")
+    bad(img[:16])
+    bad(b"NOTANIMG" + img[8:])
+    for cut in (1, 8, 9, len(img) // 2):
+        bad(img[:-cut])                             # truncated
+    flipped = bytearray(img); flipped[len(img) // 3] ^= 0x40
+    bad(bytes(flipped))                             # altered: checksum
+    def resum(b):
+        return bytes(b[:-8]) + _fnv1a(bytes(b[:-8])).to_bytes(8, "little")
+    v2 = bytearray(img); v2[8] = 2
+    bad(resum(v2))                                  # another version, intact checksum
+    # an intact checksum over fields that do not fit: a tensor count larger than the image
+    huge = bytearray(img); huge[32:40] = (1 << 40).to_bytes(8, "little")
+    bad(resum(huge))
+    # ... and an operator that names a tensor that does not exist (first tensor's producer field)
+    idx = bytearray(img)
+    off = 8 + 4 + 20 + 8 + 16                       # magic, version, hw, tensor count, c h w is_vec of tensor 0
+    idx[off:off + 4] = (12345).to_bytes(4, "little")
+    bad(resum(idx))
+    assert xb.Graph.load(img)[0].plan_text() == g.plan_text()     # the untouched image still loads
