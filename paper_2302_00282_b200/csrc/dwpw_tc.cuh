@@ -187,6 +187,65 @@ dwpw_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUt
             tc_fence_after();
             const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + b * g.acc_stride;
             const int nc32 = (cols + 31) >> 5;
+            if (g.epi == GE_GAP) {
+                // ---- global average of whole images (a CTA's only tile: the A|B ring is free and holds the slabs) ----
+                // Per pass the kW / 4 warps of a quarter take kW / 4 chunks of 32 columns: every thread parks its row's
+                // activated fp32 values in its chunk's slab [128 rows][33]; then (slab, image, column, part) items sum
+                // the rows r = part, part + parts, ... in ascending order, and the parts are added in ascending order.
+                constexpr int kSlabs = kW / 4;
+                float *slab = reinterpret_cast<float *>(sm) + cgroup * (kTileM * 33);
+                float *parts_mem = reinterpret_cast<float *>(sm) + kSlabs * (kTileM * 33);
+                const float lo1 = act_lo(g.act), hi1 = act_hi(g.act);
+                const int per = kSlabs * g.gap_imgs * 32;                       // (slab, image, column) triples
+                const int parts = per * 4 <= kWorkerThreads ? 4 : (per * 2 <= kWorkerThreads ? 2 : 1);
+                for (int c0 = 0; c0 < nc32; c0 += kSlabs) {
+                    const int c32 = c0 + cgroup;
+                    if (c32 < nc32) {
+                        float v[32];
+                        const bool whole = c32 * 32 + 32 <= cols;
+                        if (whole) tmem_ld32(t_lane + c32 * 32, v);
+                        else { tmem_ld16(t_lane + c32 * 32, v); for (int e = 16; e < 32; ++e) v[e] = 0.0f; }
+#pragma unroll
+                        for (int q4 = 0; q4 < 32; q4 += 4) {
+                            float4 bz = make_float4(0.f, 0.f, 0.f, 0.f);
+                            if (c32 * 32 + q4 < cols) bz = ld_shared_f4(sbias + (uint32_t)(c32 * 32 + q4) * 4u);
+                            slab[row * 33 + q4] = rq.valid ? fminf(fmaxf(v[q4] + bz.x, lo1), hi1) : 0.0f;
+                            slab[row * 33 + q4 + 1] = rq.valid ? fminf(fmaxf(v[q4 + 1] + bz.y, lo1), hi1) : 0.0f;
+                            slab[row * 33 + q4 + 2] = rq.valid ? fminf(fmaxf(v[q4 + 2] + bz.z, lo1), hi1) : 0.0f;
+                            slab[row * 33 + q4 + 3] = rq.valid ? fminf(fmaxf(v[q4 + 3] + bz.w, lo1), hi1) : 0.0f;
+                        }
+                    }
+                    if (c0 + kSlabs >= nc32) {
+                        // this warp's last read of the accumulator
+                        tc_fence_before();
+                        warp_arrive(acce_bar(b), lane);
+                    }
+                    asm volatile("bar.sync 1, %0;" ::"r"(kWorkerThreads) : "memory");
+                    for (int item = wt; item < per * parts; item += kWorkerThreads) {
+                        const int c = item & 31, rest = item >> 5;
+                        const int pa = rest % parts, tri = rest / parts, sl = tri % kSlabs, img = tri / kSlabs;
+                        const float *src = reinterpret_cast<float *>(sm) + sl * (kTileM * 33);
+                        float acc = 0.0f;
+                        for (int r = pa; r < g.gap_area; r += parts) acc += src[(img * g.gap_area + r) * 33 + c];
+                        parts_mem[item] = acc;
+                    }
+                    asm volatile("bar.sync 1, %0;" ::"r"(kWorkerThreads) : "memory");
+                    for (int item = wt; item < per; item += kWorkerThreads) {
+                        const int c = item & 31, tri = item >> 5, sl = tri % kSlabs, img = tri / kSlabs;
+                        const int n = we.mt * g.gap_imgs + img, nc = n0 + (c0 + sl) * 32 + c;
+                        if (c0 + sl >= nc32 || n >= g.batch || nc >= g.N) continue;
+                        float acc = 0.0f;
+                        for (int pa = 0; pa < parts; ++pa) acc += parts_mem[((tri * parts + pa) << 5) + c];
+                        acc /= (float)g.gap_rpi;
+                        const size_t oi = (size_t)n * g.out_ctot + g.out_coff + nc;
+                        if (g.out_f32) reinterpret_cast<float *>(g.out)[oi] = acc;
+                        else reinterpret_cast<__nv_bfloat16 *>(g.out)[oi] = __float2bfloat16_rn(acc);
+                    }
+                    // (the next pass's slab writes follow this pass's reads of parts_mem only; the slabs were last read
+                    // before the barrier above)
+                }
+                continue;
+            }
             for (int c32 = cgroup; c32 < nc32; c32 += kW / 4) {
                 float v[32];
                 const bool whole = c32 * 32 + 32 <= cols;

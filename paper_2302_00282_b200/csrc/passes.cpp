@@ -965,7 +965,11 @@ struct Lower {
         // for narrower ones): with a single tile the separate producer and epilogue warps of gemm_chain_kernel
         // would take turns waiting.  Measured on MobileNet at batch 32: 18.8 against 20.1 us per 14 x 14 chain; the
         // chains with many tiles per CTA are faster in gemm_chain_kernel (44 against 48 us for the first one).
-        if (dw && L.epi == EPI_STORE && L.ksplit == 1 && s1.mode == AM_NONE && L.m_tiles * L.n_tiles <= g.hw.sm_count) {
+        // (a global-average epilogue parks its slabs in the A|B ring, which a CTA's only tile has left free)
+        const int gap_workers = L.halo_cb > 32 ? 16 : 8;
+        const long gap_need = (long)(gap_workers / 4) * 128 * 33 * 4 + 4L * std::max(32 * gap_workers, (gap_workers / 4) * L.gap_imgs * 32);
+        const bool gap_fits = L.epi == EPI_GAP && L.skip < 0 && L.act2 == 0 && (long)L.stages * stage_bytes >= gap_need;
+        if (dw && (L.epi == EPI_STORE || gap_fits) && L.ksplit == 1 && s1.mode == AM_NONE && L.m_tiles * L.n_tiles <= g.hw.sm_count) {
             L.dw_workers = L.halo_cb > 32 ? 16 : 8;
             L.block = 64 + 32 * L.dw_workers;
         }
