@@ -137,6 +137,7 @@ struct Launch {
     int hstages = 0, halo_bytes = 0, halo_stride = 0, halo_cb = 0;   // depthwise halo ring (halo_h x halo_w input pixels per image)
     int stem_tma = 0, stem_align = 1;                              // stem: image patch by TMA, x alignment in elements
     int a_tma = 0, a_box_bytes = 0;                                // activation operand by TMA: 1 matrix rows, 2 shifted patch
+    int fc_small = 0;                                              // 1: fully connected layer of a small batch on the CUDA cores (fc_small_kernel)
     int dw_workers = 0;                                            // > 0: depthwise -> pointwise in dwpw_kernel with that many worker warps
     int n_acc = 1;                                                 // dwpw_kernel: channel tiles of tile_n columns per CTA (2: both accumulators hold one tile)
     // ---- two linked convolutions (LK_GEMM2): producer tile rh1 x rw1 = patch_rh x patch_rw, consumer tile rh2 x rw2

@@ -140,6 +140,57 @@ __global__ void gap_kernel(const __nv_bfloat16 *__restrict__ x, void *__restrict
     }
 }
 
+// Fully connected layer (Eq. 1 of the Xenos paper: out = W x + b) for batches of at most 32 vectors, on the CUDA
+// cores: with so few rows a 128-row MMA tile is three quarters empty and the layer is a single pass over the weight
+// matrix.  The CTA stages the input vectors [N][C] in shared memory; a warp takes one output feature at a time: its
+// lanes read the feature's weight row 16 bytes at a time (each weight leaves L2 once per CTA that needs it, once
+// from HBM), multiply it with all N vectors, and the 32 lanes' partial sums are added by butterfly shuffles (a fixed
+// order).  w is the packed [K padded][ldw] bf16 matrix of the implicit GEMM; bias, activation and output as there.
+__global__ void __launch_bounds__(256)
+fc_small_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__restrict__ w, const float *__restrict__ bias,
+                void *__restrict__ y, int N, int C, int ldw, int K, int act, int out_f32, int out_ctot, int out_coff) {
+    extern __shared__ uint4 fc_xs[];                       // [N][C / 8] chunks of 8 channels
+    const int C8 = C >> 3;
+    for (int i = threadIdx.x; i < N * C8; i += blockDim.x) fc_xs[i] = reinterpret_cast<const uint4 *>(x)[i];
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    const float lo = act >= 1 ? 0.0f : -INFINITY, hi = act == 2 ? 6.0f : INFINITY;
+    for (int o = blockIdx.x * nwarps + warp; o < K; o += gridDim.x * nwarps) {
+        float acc[32];
+#pragma unroll
+        for (int n = 0; n < 32; ++n) acc[n] = 0.0f;
+        const uint4 *wrow = reinterpret_cast<const uint4 *>(w + (size_t)o * ldw);
+        for (int ch = lane; ch < C8; ch += 32) {
+            const f8 wv = unpack8(__ldg(wrow + ch));
+#pragma unroll
+            for (int n = 0; n < 32; ++n) {
+                if (n >= N) break;
+                const f8 xv = unpack8(fc_xs[n * C8 + ch]);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) acc[n] = fmaf(wv.v[j], xv.v[j], acc[n]);
+            }
+        }
+#pragma unroll
+        for (int n = 0; n < 32; ++n) {
+            if (n >= N) break;
+            float v = acc[n];
+#pragma unroll
+            for (int s = 16; s >= 1; s >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
+            acc[n] = v;
+        }
+        // lane n stores image n
+        float mine = 0.0f;
+#pragma unroll
+        for (int n = 0; n < 32; ++n) if (n == lane) mine = acc[n];
+        if (lane < N) {
+            const float r = fminf(fmaxf(mine + bias[o], lo), hi);
+            const size_t oi = (size_t)lane * out_ctot + out_coff + o;
+            if (out_f32) reinterpret_cast<float *>(y)[oi] = r;
+            else reinterpret_cast<__nv_bfloat16 *>(y)[oi] = __float2bfloat16_rn(r);
+        }
+    }
+}
+
 __global__ void add_kernel(const __nv_bfloat16 *__restrict__ a, const __nv_bfloat16 *__restrict__ b,
                            __nv_bfloat16 *__restrict__ y, long long n8, int act) {
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n8; i += (long long)gridDim.x * blockDim.x) {

@@ -230,6 +230,9 @@ xenos_status_t runtime_bind(Graph &g, void *ws, size_t bytes, void *stream_v) {
         if ((e = cudaFuncSetAttribute(xk::dwpw_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, optin)) != cudaSuccess ||
             (e = cudaFuncSetAttribute(xk::dwpw_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, optin)) != cudaSuccess)
             return cuda_fail(g, "cudaFuncSetAttribute(dwpw)", e);
+    if (any_gemm)
+        if ((e = cudaFuncSetAttribute(xk::fc_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024)) != cudaSuccess)
+            return cuda_fail(g, "cudaFuncSetAttribute(fc)", e);
     if (any_gemm2)
         if ((e = cudaFuncSetAttribute(xk::chain2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin)) != cudaSuccess)
             return cuda_fail(g, "cudaFuncSetAttribute(chain2)", e);
@@ -414,6 +417,13 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
             break;
         }
         case LK_GEMM: {
+            if (L.fc_small) {
+                const int grid = std::min(sms, (L.K + 7) / 8);
+                xk::fc_small_kernel<<<grid, 256, (size_t)N * L.C * 2, stream>>>(
+                    (const __nv_bfloat16 *)ptr(L.seg[0].tensor), (const __nv_bfloat16 *)(ws + L.w_off), (const float *)(ws + L.b_off), ptr(L.out), N, L.C,
+                    L.kpad, L.K, L.act, L.out_dtype == XENOS_DTYPE_F32, L.out_ctot, L.out_coff);
+                break;
+            }
             xk::GemmParams p;
             std::memset(&p, 0, sizeof p);
             for (int s = 0; s < 2; ++s) {

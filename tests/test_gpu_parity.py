@@ -356,12 +356,26 @@ def test_bf16_fc_reduction_split_is_automatic_and_repeatable():
         x = g.gap("gap", "input")
         g.fc("fc", x, 1000)
     spec = _one(build, 1024, 3)
-    y, _, gg = check_bf16("fc_splitk_auto", spec, 5, linked=False, in_mode="bf16_nhwc")
+    y, _, gg = check_bf16("fc_splitk_auto", spec, 12, linked=False, in_mode="bf16_nhwc")
     L = [l for l in gg.g.plan()["launches"] if l["kind"] == "gemm"][0]
-    assert L["ksplit"] >= 2
-    x = xo.round_bf16(graphs.make_input(spec, 5))
+    assert L["ksplit"] >= 2 and not L["fc_small"]
+    x = xo.round_bf16(graphs.make_input(spec, 12))
     for _ in range(3):
         assert np.array_equal(gg.run(x), y)
+
+
+@pytest.mark.parametrize("c,k,batch,run_batch", [(1024, 1000, 1, 1), (512, 1000, 8, 8), (1536, 24, 5, 3), (40, 7, 8, 8)])
+def test_bf16_fc_of_a_few_vectors_on_cuda_cores(c, k, batch, run_batch):
+    """Up to 8 vectors: one pass over the weight matrix, no tiles (fc_small_kernel); also with fewer images than max_batch."""
+    def build(g):
+        x = g.gap("gap", "input")
+        g.fc("fc", x, k)
+    spec = _one(build, c, 2)
+    y, _, gg = check_bf16(f"fc_small{(c, k, batch)}", spec, run_batch, linked=True, in_mode="bf16_nhwc", max_batch=batch)
+    L = [l for l in gg.g.plan()["launches"] if l["kind"] == "gemm"][0]
+    assert L["fc_small"] == 1
+    x = xo.round_bf16(graphs.make_input(spec, run_batch))
+    assert np.array_equal(gg.run(x), y)
 
 
 @pytest.mark.parametrize("pool", [False, True])

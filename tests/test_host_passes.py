@@ -351,7 +351,10 @@ def test_reduction_split_is_automatic_only_where_units_would_idle():
     L = g.plan()["launches"]
     assert [l.get("ksplit", 1) for l in L[:-1]] == [1] * (len(L) - 1)
     fc = L[-1]
-    assert fc["ksplit"] >= 2 and fc["m_tiles"] * fc["n_tiles"] * fc["ksplit"] <= 148 and fc["kb_per"] >= 2
+    assert fc["ksplit"] >= 2 and fc["m_tiles"] * fc["n_tiles"] * fc["ksplit"] <= 148 and fc["kb_per"] >= 2 and not fc["fc_small"]
+    # up to 8 vectors the fc is one pass over its weights on the CUDA cores: no tiles to cut
+    fc8 = compiled(spec, 8)[0].plan()["launches"][-1]
+    assert fc8["fc_small"] == 1 and fc8["ksplit"] == 1
     # a depthwise -> pointwise chain is cut on request only
     g1, ids = compiled(spec, 1, splits=[("pw7.relu6", dict(parts_k=8))])
     L1 = g1.plan()["launches"]
