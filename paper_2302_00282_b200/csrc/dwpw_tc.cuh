@@ -36,6 +36,7 @@ dwpw_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUt
     auto hempty_bar = [&](int s) { return bar_base + 8u * (2 * kMaxStages + 4 + kMaxHaloStages + s); };
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(sm + g.off_bar + 8 * (2 * kMaxStages + 4 + 2 * kMaxHaloStages));
     volatile int *fail_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    const uint32_t dww_bar = bar_base + 8u * (2 * kMaxStages + 4 + 2 * kMaxHaloStages + 3);      // the depthwise parameters have landed
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int total_tiles = g.m_tiles * g.n_tiles;
@@ -46,22 +47,25 @@ dwpw_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUt
         for (int s = 0; s < g.stages; ++s) { mbar_init(full_bar(s), kW + 1); mbar_init(empty_bar(s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), kW); }
         for (int s = 0; s < g.hstages; ++s) { mbar_init(hfull_bar(s), 1); mbar_init(hempty_bar(s), kW); }
+        mbar_init(dww_bar, 1);
         *fail_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        // depthwise tap weights [9][C] followed by the bias [C], fp32, once per CTA: two bulk copies that the workers wait
+        // for before their first stencil (constants: no need to wait for the predecessor kernel)
+        {
+            const uint32_t C = (uint32_t)g.seg[0].C;
+            mbar_arrive_expect_tx(dww_bar, 40u * C);
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(sbase + g.off_dww), "l"(g.seg[0].dw_w), "r"(36u * C), "r"(dww_bar) : "memory");
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(sbase + g.off_dww + 36u * C), "l"(g.seg[0].dw_b), "r"(4u * C), "r"(dww_bar) : "memory");
+        }
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmH) : "memory");
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)g.tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    if (warp >= 2) {
-        // depthwise tap weights [9][C] followed by the bias [C], fp32, once per CTA
-        const int C = g.seg[0].C;
-        float4 *dst = reinterpret_cast<float4 *>(sm + g.off_dww);
-        const float4 *w4 = reinterpret_cast<const float4 *>(g.seg[0].dw_w), *b4 = reinterpret_cast<const float4 *>(g.seg[0].dw_b);
-        for (int i = threadIdx.x - 64; i < 9 * C / 4; i += kWorkerThreads) dst[i] = __ldg(w4 + i);
-        for (int i = threadIdx.x - 64; i < C / 4; i += kWorkerThreads) dst[9 * C / 4 + i] = __ldg(b4 + i);
     }
     tc_fence_before();
     __syncthreads();
@@ -145,6 +149,7 @@ dwpw_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUt
         const uint32_t plo = g.act >= 1 ? 0u : 0xff80ff80u, phi = g.act == 2 ? 0x40c040c0u : 0x7f807f80u;
         const bool wide_ok = ((reinterpret_cast<uintptr_t>(g.out) | (uintptr_t)(g.out_ctot * 2) | (uintptr_t)(g.out_coff * 2)) & 31u) == 0;
         Ring st = {0, 0u}, hr = {0, 0u};
+        ok = mbar_wait_warp(dww_bar, 0u, lane);
         auto stencil = [&]() {
             for (int kb = 0; kb < g.kblocks && ok; ++kb) {
                 const int s = st.s, hs = hr.s;
