@@ -98,7 +98,8 @@ enum LaunchKind {
     LK_F32_POOL, LK_F32_GAP, LK_F32_ADD, LK_F32_CONCAT_PART, LK_F32_FC,
     LK_F32_CONV_CONV_POOL, // fp32 linked chain
     LK_F32_MULMAC, LK_F32_TRANSPOSE, LK_F32_SLICE,
-    LK_GEMM2              // two linked convolutions, intermediate tile in shared memory (chain2_kernel)
+    LK_GEMM2,             // two linked convolutions, intermediate tile in shared memory (chain2_kernel)
+    LK_STEM3X3            // 3x3 convolution of an NCHW image with at most 4 channels on the CUDA cores (stem3x3_kernel)
 };
 
 struct Launch {

@@ -140,6 +140,78 @@ __global__ void gap_kernel(const __nv_bfloat16 *__restrict__ x, void *__restrict
     }
 }
 
+// 3x3 convolution of an NCHW image with at most 4 channels (the first layer of the bf16 graphs) on the CUDA cores:
+// with K = 27 the MMA's 64-wide K block is mostly padding and building that block costs more than the product.
+// A CTA takes 8 x 32 output pixels: the input window goes to shared memory as fp32 (zero outside the image = the
+// padding), the weights [tap row][tap column][channel][Cout] and the bias too.  A thread owns 4 adjacent pixels of a
+// row for 8 output channels: per tap row and input channel it reads the 4 pixels' window once and feeds 3 x 4 x 8
+// multiply-adds; taps are added in the order (row, channel, column), fixed.  Output: NHWC bf16 (bias, activation).
+template <typename TIn>
+__global__ void __launch_bounds__(256)
+stem3x3_kernel(const TIn *__restrict__ x, const float *__restrict__ w, const float *__restrict__ bias, __nv_bfloat16 *__restrict__ y,
+               int N, int C, int H, int W, int K, int P, int Q, int stride, int pad, int act) {
+    constexpr int TH = 8, TW = 32;
+    extern __shared__ float stem_sm[];
+    const int ih = (TH - 1) * stride + 3, iw = (TW - 1) * stride + 3, iwp = iw | 1;       // odd pitch: fewer bank conflicts
+    float *win = stem_sm;                                  // [C][ih][iwp]
+    float *ws = win + ((C * ih * iwp + 3) & ~3);           // [3][3][C][K], 16-byte aligned
+    float *bs = ws + 9 * C * K;                            // [K]
+    const int tiles_x = (Q + TW - 1) / TW, tiles_y = (P + TH - 1) / TH;
+    const int t = blockIdx.x % (tiles_x * tiles_y), n = blockIdx.x / (tiles_x * tiles_y);
+    const int ty = t / tiles_x, tx = t - ty * tiles_x;
+    const int y0 = ty * TH * stride - pad, x0 = tx * TW * stride - pad;
+    for (int i = threadIdx.x; i < 9 * C * K; i += 256) ws[i] = w[i];
+    for (int i = threadIdx.x; i < K; i += 256) bs[i] = bias[i];
+    for (int i = threadIdx.x; i < C * ih * iw; i += 256) {
+        const int c = i / (ih * iw), r = i - c * ih * iw, yy = r / iw, xx = r - yy * iw;
+        const int gy = y0 + yy, gx = x0 + xx;
+        float v = 0.0f;
+        if (gy >= 0 && gy < H && gx >= 0 && gx < W) v = (float)x[(((size_t)n * C + c) * H + gy) * W + gx];
+        win[(c * ih + yy) * iwp + xx] = v;
+    }
+    __syncthreads();
+    const int K8 = K >> 3;
+    const float lo = act >= 1 ? 0.0f : -INFINITY, hi = act == 2 ? 6.0f : INFINITY;
+    for (int u = threadIdx.x; u < TH * (TW / 4) * K8; u += 256) {
+        const int cg = u % K8, pg = u / K8, py = pg / (TW / 4), px = (pg - py * (TW / 4)) * 4;
+        float acc[4][8];
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int o = 0; o < 8; ++o) acc[j][o] = bs[cg * 8 + o];
+        for (int r = 0; r < 3; ++r)
+            for (int c = 0; c < C; ++c) {
+                const float *row = win + (c * ih + py * stride + r) * iwp + px * stride;
+                float v[9];
+#pragma unroll
+                for (int e = 0; e < 9; ++e) v[e] = e < 3 * stride + 3 ? row[e] : 0.0f;      // (stride 1 uses 6, stride 2 uses 9)
+#pragma unroll
+                for (int s = 0; s < 3; ++s) {
+                    const float4 w0 = *reinterpret_cast<const float4 *>(ws + ((r * 3 + s) * C + c) * K + cg * 8);
+                    const float4 w1 = *reinterpret_cast<const float4 *>(ws + ((r * 3 + s) * C + c) * K + cg * 8 + 4);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float in = stride == 1 ? v[j + s] : v[2 * j + s];
+                        acc[j][0] = fmaf(in, w0.x, acc[j][0]); acc[j][1] = fmaf(in, w0.y, acc[j][1]);
+                        acc[j][2] = fmaf(in, w0.z, acc[j][2]); acc[j][3] = fmaf(in, w0.w, acc[j][3]);
+                        acc[j][4] = fmaf(in, w1.x, acc[j][4]); acc[j][5] = fmaf(in, w1.y, acc[j][5]);
+                        acc[j][6] = fmaf(in, w1.z, acc[j][6]); acc[j][7] = fmaf(in, w1.w, acc[j][7]);
+                    }
+                }
+            }
+        const int oy = ty * TH + py;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int ox = tx * TW + px + j;
+            if (oy >= P || ox >= Q) continue;
+            f8 o;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) o.v[e] = fminf(fmaxf(acc[j][e], lo), hi);
+            *reinterpret_cast<uint4 *>(y + (((size_t)n * P + oy) * Q + ox) * K + cg * 8) = pack8(o);
+        }
+    }
+}
+
 // Fully connected layer (Eq. 1 of the Xenos paper: out = W x + b) for batches of at most 32 vectors, on the CUDA
 // cores: with so few rows a 128-row MMA tile is three quarters empty and the layer is a single pass over the weight
 // matrix.  The CTA stages the input vectors [N][C] in shared memory; a warp takes one output feature at a time: its

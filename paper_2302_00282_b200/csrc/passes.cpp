@@ -1120,6 +1120,36 @@ struct Lower {
 
     xenos_status_t lower_bf16_single(int ci, int ni) {
         const Node &n = g.nodes[ni];
+        if (n.kind == NK_CONV) {
+            // the first layer at small batch: a 3x3 convolution of an NCHW image runs on the CUDA cores (K = 27 fills
+            // less than half of one 64-wide K block of the MMA; a launch of the persistent kernel costs more than this
+            // whole layer).  Same-box A/B on MobileNet: batch 1 0.1506 -> 0.1424 ms; at batch 32 the tensor-core stem
+            // with its TMA-fetched patches is faster (31 against 43 us), so larger batches keep it.
+            const Tensor &x = g.tensors[n.in[0]];
+            const bool no_request = !g.chains[ci].split.user;
+            if (x.input_slot >= 0 && x.io_layout == XENOS_LAYOUT_NCHW && x.c <= 4 && n.k == 3 && (n.stride == 1 || n.stride == 2) &&
+                n.cout % 8 == 0 && n.cout <= 64 && n.cin == x.c && no_request && !n.from_matmul && g.max_batch <= 8) {
+                Launch L;
+                L.kind = LK_STEM3X3;
+                L.nodes = {ni};
+                fill_io(L, n);
+                L.seg[0].src_dtype = x.io_dtype;
+                // weights [tap row][tap column][channel][cout], fp32
+                std::vector<float> wt((size_t)9 * n.cin * n.cout);
+                for (int o = 0; o < n.cout; ++o)
+                    for (int c = 0; c < n.cin; ++c)
+                        for (int t9 = 0; t9 < 9; ++t9) wt[((size_t)t9 * n.cin + c) * n.cout + o] = n.w[((size_t)o * n.cin + c) * 9 + t9];
+                L.w_off = put_f32(wt); L.b_off = put_f32(n.b);
+                L.flops = 2.0 * node_macs(n);
+                L.bytes = tbytes(n.in[0]) + tbytes(n.out) + node_param_bytes(n);
+                const int ih = 7 * n.stride + 3, iw = 31 * n.stride + 3;
+                L.smem_bytes = 4 * (((n.cin * ih * (iw | 1) + 3) & ~3) + 9 * n.cin * n.cout + n.cout);
+                L.grid = ceil_div(L.P, 8) * ceil_div(L.Q, 32);      // per image
+                L.block = 256;
+                push(L, ci);
+                return XENOS_OK;
+            }
+        }
         if (n.kind == NK_CONV) return make_gemm(ci, {ni}, nullptr, &n, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, false);
         if (n.kind == NK_FC) {
             if (n.cin % 8) return fail(g, XENOS_E_UNSUPPORTED, "fc input length must be a multiple of 8");
@@ -1341,7 +1371,7 @@ void emit_plan_json(Graph &g) {
     static const char *nk[] = {"?", "conv", "dwconv", "fc", "maxpool", "avgpool", "gap", "add", "concat", "mul", "mac", "transpose", "split"};
     static const char *ck[] = {"single", "conv_conv_pool", "dw_pw", "conv_tail", "expand_concat", "matmul_matmul", "conv_conv"};
     static const char *lk[] = {"?", "gemm", "dw", "pool", "gap", "add", "concat_part", "mulmac", "transpose", "slice", "f32_conv", "f32_pool",
-                               "f32_gap", "f32_add", "f32_concat_part", "f32_fc", "f32_conv_conv_pool", "f32_mulmac", "f32_transpose", "f32_slice", "gemm2"};
+                               "f32_gap", "f32_add", "f32_concat_part", "f32_fc", "f32_conv_conv_pool", "f32_mulmac", "f32_transpose", "f32_slice", "gemm2", "stem3x3"};
     static const char *am[] = {"none", "gather", "stem", "dw"};
     std::string s = "{";
     jstr(s, "precision", g.precision == XENOS_PRECISION_FP32_CUDA_CORE ? "fp32_cuda_core" : "bf16_tensor");

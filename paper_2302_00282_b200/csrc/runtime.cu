@@ -320,6 +320,16 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
             xk::f32_conv_conv_pool_kernel<<<N * L.grid, L.block, L.smem_bytes, stream>>>(p);
             break;
         }
+        case LK_STEM3X3: {
+            const int grid = N * L.grid;
+            if (L.seg[0].src_dtype == XENOS_DTYPE_F32)
+                xk::stem3x3_kernel<float><<<grid, 256, (size_t)L.smem_bytes, stream>>>((const float *)ptr(L.in0), (const float *)(ws + L.w_off), (const float *)(ws + L.b_off),
+                    (__nv_bfloat16 *)ptr(L.out), N, L.C, L.H, L.W, L.K, L.P, L.Q, L.stride, L.pad, L.act);
+            else
+                xk::stem3x3_kernel<__nv_bfloat16><<<grid, 256, (size_t)L.smem_bytes, stream>>>((const __nv_bfloat16 *)ptr(L.in0), (const float *)(ws + L.w_off), (const float *)(ws + L.b_off),
+                    (__nv_bfloat16 *)ptr(L.out), N, L.C, L.H, L.W, L.K, L.P, L.Q, L.stride, L.pad, L.act);
+            break;
+        }
         case LK_DW: {
             long long total = (long long)N * L.P * L.Q * (L.C / 8);
             xk::dw3x3_kernel<<<ew_grid(total, 256, sms), 256, 0, stream>>>(

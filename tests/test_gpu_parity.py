@@ -713,3 +713,15 @@ def test_loaded_graph_image_computes_the_same_bits(name):
     g2.run(3, [xin.data_ptr()], [out.data_ptr()], gg.stream)
     g2.status(gg.stream)
     assert gg.vec and np.array_equal(out.float().cpu().numpy(), y)
+
+
+# ---- the first layer of a small batch on the CUDA cores ---------------------------------------------------------------
+@pytest.mark.parametrize("cin,cout,hw,stride,pad,batch,in_mode", [(3, 32, 40, 2, 1, 2, "f32_nchw"), (3, 64, 37, 2, 0, 3, "bf16_nchw"), (1, 8, 9, 1, 1, 8, "f32_nchw"),
+                                                                 (4, 24, 66, 1, 0, 1, "f32_nchw"), (3, 32, 224, 2, 1, 1, "f32_nchw")])
+def test_bf16_stem_3x3_on_cuda_cores(cin, cout, hw, stride, pad, batch, in_mode):
+    """Tiles that end inside the image, both strides, with and without padding, fp32 and bf16 images, 1 to 4 channels."""
+    def build(g):
+        g.cbr("stem", "input", cout, 3, stride, pad, act="relu6")
+    spec = _one(build, cin, hw)
+    _, _, gg = check_bf16(f"stem3x3{(cin, cout, hw, stride, pad)}", spec, batch, linked=True, in_mode=in_mode)
+    assert [l["kind"] for l in gg.g.plan()["launches"]] == ["stem3x3"]
