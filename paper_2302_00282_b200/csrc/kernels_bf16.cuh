@@ -160,25 +160,41 @@ stem3x3_kernel(const TIn *__restrict__ x, const float *__restrict__ w, const flo
     const int t = blockIdx.x % (tiles_x * tiles_y), n = blockIdx.x / (tiles_x * tiles_y);
     const int ty = t / tiles_x, tx = t - ty * tiles_x;
     const int y0 = ty * TH * stride - pad, x0 = tx * TW * stride - pad;
+    // the next kernel of the stream may be scheduled as soon as every CTA of this one has started
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     for (int i = threadIdx.x; i < 9 * C * K; i += 256) ws[i] = w[i];
     for (int i = threadIdx.x; i < K; i += 256) bs[i] = bias[i];
-    for (int i = threadIdx.x; i < C * ih * iw; i += 256) {
-        const int c = i / (ih * iw), r = i - c * ih * iw, yy = r / iw, xx = r - yy * iw;
-        const int gy = y0 + yy, gx = x0 + xx;
-        float v = 0.0f;
-        if (gy >= 0 && gy < H && gx >= 0 && gx < W) v = (float)x[(((size_t)n * C + c) * H + gy) * W + gx];
-        win[(c * ih + yy) * iwp + xx] = v;
+    // window rows: a warp takes a (channel, row) pair at a time, its lanes three columns each: independent loads, no
+    // division in the loop
+    {
+        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        for (int cr = warp; cr < C * ih; cr += 8) {
+            const int c = cr / ih, yy = cr - c * ih, gy = y0 + yy;
+            const bool row_in = gy >= 0 && gy < H;
+            const TIn *src = x + (((size_t)n * C + c) * H + (row_in ? gy : 0)) * W;
+            float v[3];
+#pragma unroll
+            for (int e = 0; e < 3; ++e) {
+                const int xx = lane + 32 * e, gx = x0 + xx;
+                v[e] = (row_in && xx < iw && gx >= 0 && gx < W) ? (float)src[gx] : 0.0f;
+            }
+#pragma unroll
+            for (int e = 0; e < 3; ++e) {
+                const int xx = lane + 32 * e;
+                if (xx < iw) win[cr * iwp + xx] = v[e];
+            }
+        }
     }
     __syncthreads();
     const int K8 = K >> 3;
     const float lo = act >= 1 ? 0.0f : -INFINITY, hi = act == 2 ? 6.0f : INFINITY;
     for (int u = threadIdx.x; u < TH * (TW / 4) * K8; u += 256) {
         const int cg = u % K8, pg = u / K8, py = pg / (TW / 4), px = (pg - py * (TW / 4)) * 4;
-        float acc[4][8];
+        float2 acc[4][4];
 #pragma unroll
         for (int j = 0; j < 4; ++j)
 #pragma unroll
-            for (int o = 0; o < 8; ++o) acc[j][o] = bs[cg * 8 + o];
+            for (int o = 0; o < 4; ++o) acc[j][o] = make_float2(bs[cg * 8 + 2 * o], bs[cg * 8 + 2 * o + 1]);
         for (int r = 0; r < 3; ++r)
             for (int c = 0; c < C; ++c) {
                 const float *row = win + (c * ih + py * stride + r) * iwp + px * stride;
@@ -192,10 +208,11 @@ stem3x3_kernel(const TIn *__restrict__ x, const float *__restrict__ w, const flo
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         const float in = stride == 1 ? v[j + s] : v[2 * j + s];
-                        acc[j][0] = fmaf(in, w0.x, acc[j][0]); acc[j][1] = fmaf(in, w0.y, acc[j][1]);
-                        acc[j][2] = fmaf(in, w0.z, acc[j][2]); acc[j][3] = fmaf(in, w0.w, acc[j][3]);
-                        acc[j][4] = fmaf(in, w1.x, acc[j][4]); acc[j][5] = fmaf(in, w1.y, acc[j][5]);
-                        acc[j][6] = fmaf(in, w1.z, acc[j][6]); acc[j][7] = fmaf(in, w1.w, acc[j][7]);
+                        const float2 in2 = make_float2(in, in);
+                        acc[j][0] = __ffma2_rn(in2, make_float2(w0.x, w0.y), acc[j][0]);
+                        acc[j][1] = __ffma2_rn(in2, make_float2(w0.z, w0.w), acc[j][1]);
+                        acc[j][2] = __ffma2_rn(in2, make_float2(w1.x, w1.y), acc[j][2]);
+                        acc[j][3] = __ffma2_rn(in2, make_float2(w1.z, w1.w), acc[j][3]);
                     }
                 }
             }
@@ -206,7 +223,7 @@ stem3x3_kernel(const TIn *__restrict__ x, const float *__restrict__ w, const flo
             if (oy >= P || ox >= Q) continue;
             f8 o;
 #pragma unroll
-            for (int e = 0; e < 8; ++e) o.v[e] = fminf(fmaxf(acc[j][e], lo), hi);
+            for (int e = 0; e < 4; ++e) { o.v[2 * e] = fminf(fmaxf(acc[j][e].x, lo), hi); o.v[2 * e + 1] = fminf(fmaxf(acc[j][e].y, lo), hi); }
             *reinterpret_cast<uint4 *>(y + (((size_t)n * P + oy) * Q + ox) * K + cg * 8) = pack8(o);
         }
     }

@@ -1124,7 +1124,7 @@ struct Lower {
             // the first layer at small batch: a 3x3 convolution of an NCHW image runs on the CUDA cores (K = 27 fills
             // less than half of one 64-wide K block of the MMA; a launch of the persistent kernel costs more than this
             // whole layer).  Same-box A/B on MobileNet: batch 1 0.1506 -> 0.1424 ms; at batch 32 the tensor-core stem
-            // with its TMA-fetched patches is faster (31 against 43 us), so larger batches keep it.
+            // with its TMA-fetched patches is faster (30 against 35.5 us), so larger batches keep it.
             const Tensor &x = g.tensors[n.in[0]];
             const bool no_request = !g.chains[ci].split.user;
             if (x.input_slot >= 0 && x.io_layout == XENOS_LAYOUT_NCHW && x.c <= 4 && n.k == 3 && (n.stride == 1 || n.stride == 2) &&
