@@ -94,6 +94,10 @@ struct GemmParams {
     unsigned int *split_cnt;
     int launch_id;                                  // position of this launch in the plan, reported with a give-up
     int n_acc;                                      // dwpw_kernel: channel tiles per CTA (2: one 512-column tile in both accumulators)
+    // global average of images with more than 128 pixels (1x1 convolution, rows by TMA): an image is cut into gap_parts
+    // tiles of 128 rows; a tile leaves its column sums in split_part [image][part][split_ld], and the tile that arrives
+    // last at the image's counter (split_cnt) adds the parts in ascending order and stores the mean
+    int gap_parts;
 };
 
 // Status word of a wait that gave up: the code, the role that waited (1 TMA, 2 MMA, 3 producer, 4 producer helping
@@ -909,7 +913,8 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                     if (!ok) break;
                     mbar_arrive_expect_tx(full_bar(st.s), (uint32_t)g.tile_n * 128u + (tma_a ? (uint32_t)g.a_box_bytes : 0u));
                     if (g.a_tma == 1) {
-                        tma_load_2d(sbase + st.s * stage_bytes, &tmH, kb * kTileK, w.mt * g.tile_rows, full_bar(st.s));
+                        const int arow = (kSplit && g.gap_parts > 1) ? (w.mt / g.gap_parts) * g.gap_rpi + (w.mt % g.gap_parts) * kTileM : w.mt * g.tile_rows;
+                        tma_load_2d(sbase + st.s * stage_bytes, &tmH, kb * kTileK, arow, full_bar(st.s));
                     } else if (g.a_tma == 2) {
                         const int tap = kb / g.a_cpb, cb = kb - tap * g.a_cpb;
                         const int tr = tap / g.seg[0].k, ts = tap - tr * g.seg[0].k;
@@ -1151,7 +1156,10 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                     *reinterpret_cast<float4 *>(sm + g.off_bias + bias_buf * 1024 + et * 16) = __ldg(reinterpret_cast<const float4 *>(g.bias + nt * g.tile_n) + et);
             }
             const uint32_t sbias = sbase + g.off_bias + bias_buf * 1024;
-            const RowPos rq = map_row(g, w, rl, row);
+            RowPos rq = map_row(g, w, rl, row);
+            const bool gparts = kSplit && g.gap_parts > 1;
+            const int gp_img = gparts ? mt / g.gap_parts : 0, gp_t = gparts ? mt - gp_img * g.gap_parts : 0;
+            if (gparts) rq.valid = gp_t * kTileM + row < g.gap_rpi;      // rows of this image inside this tile
             const int n0 = nt * g.tile_n;
             const size_t pix = ((size_t)rq.n * g.P + rq.p) * g.Q + rq.q;
             // The four epilogue warps share named barriers (bias slice, pool and average staging), so they
@@ -1339,10 +1347,15 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                         epi_bar();
                         for (int item = et; item < per; item += kEpilogueThreads) {
                             const int c = item & 31, img = item >> 5;
-                            const int n = mt * g.gap_imgs + img;
+                            const int n = gparts ? gp_img : mt * g.gap_imgs + img;
                             if (c >= ncols || n >= g.batch || nc0 + c >= g.N) continue;
                             float acc = 0.0f;
                             for (int pa = 0; pa < parts; ++pa) acc += part[((img * parts + pa) << 5) + c];
+                            if (gparts) {
+                                // this tile's share of the image's column sum
+                                __stcg(g.split_part + ((size_t)gp_img * g.gap_parts + gp_t) * g.split_ld + nc0 + c, acc);
+                                continue;
+                            }
                             acc /= (float)g.gap_rpi;
                             const size_t oi = (size_t)n * g.out_ctot + g.out_coff + nc0 + c;
                             if (g.out_f32) reinterpret_cast<float *>(g.out)[oi] = acc;
@@ -1350,6 +1363,29 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                         }
                     }
                 }
+            }
+            if (gparts) {
+                // the image's tiles meet at its counter; the one that arrives last adds the parts in ascending order
+                __threadfence();
+                epi_bar();
+                unsigned int *cnt = g.split_cnt + 2 * ((size_t)gp_img * g.n_tiles + nt);
+                if (et == 0) fail_flag[1] = atomicAdd(cnt, 1u) == (unsigned int)(g.gap_parts - 1) ? 1 : 0;
+                epi_bar();
+                if (fail_flag[1]) {
+                    __threadfence();
+                    for (int col = et; col < g.tile_n; col += kEpilogueThreads) {
+                        const int nc = n0 + col;
+                        if (nc >= g.N || gp_img >= g.batch) continue;
+                        float acc = 0.0f;
+                        for (int t = 0; t < g.gap_parts; ++t) acc += __ldcg(g.split_part + ((size_t)gp_img * g.gap_parts + t) * g.split_ld + nc);
+                        acc /= (float)g.gap_rpi;
+                        const size_t oi = (size_t)gp_img * g.out_ctot + g.out_coff + nc;
+                        if (g.out_f32) reinterpret_cast<float *>(g.out)[oi] = acc;
+                        else reinterpret_cast<__nv_bfloat16 *>(g.out)[oi] = __float2bfloat16_rn(acc);
+                    }
+                    if (et == 0) *cnt = 0u;      // ready for the next run
+                }
+                epi_bar();      // (fail_flag[1] is read before the next tile rewrites it)
             }
             if (g.epi == GE_POOL) {
                 epi_bar();

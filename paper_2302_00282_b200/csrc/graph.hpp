@@ -134,6 +134,7 @@ struct Launch {
     int stages = 0, smem_bytes = 0, tmem_cols = 0, pipe_bytes = 0;
     int ni = 1, step_y = 0, step_x = 0, off_y = 0, off_x = 0;      // PATCH tiles: images, tile pitch, origin offset
     int gap_imgs = 0, gap_area = 0, gap_rpi = 0;                                 // global-average epilogue
+    int gap_parts = 1;                                                           // > 1: an image is averaged over that many 128-row tiles
     int acc_stride = 0;                                            // columns between the two accumulators
     int hstages = 0, halo_bytes = 0, halo_stride = 0, halo_cb = 0;   // depthwise halo ring (halo_h x halo_w input pixels per image)
     int stem_tma = 0, stem_align = 1;                              // stem: image patch by TMA, x alignment in elements

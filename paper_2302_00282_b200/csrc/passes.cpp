@@ -349,7 +349,10 @@ static bool try_match(const LinkCtx &cx, int a, Allowed allowed, Chain &out, boo
             out.pattern = "ConvX -> ZPooling (CBR-MaxPooling)";
             return true;
         }
-        if (B.kind == NK_GAP && cx.rows(a) <= 128 && !nchw_in) {
+        // (an image of more than 128 pixels is averaged over several tiles when the convolution is 1x1 on 64-channel
+        // blocks: its rows are then plain rows of the activation matrix)
+        if (B.kind == NK_GAP && !nchw_in &&
+            (cx.rows(a) <= 128 || (A.k == 1 && A.stride == 1 && A.pad == 0 && A.cin % 64 == 0 && g.precision != XENOS_PRECISION_FP32_CUDA_CORE))) {
             out.kind = CK_CONV_TAIL;
             out.nodes = {a, b};
             out.pattern = "ConvX -> ZPooling (CBR-AvgPooling, global)";
@@ -736,6 +739,14 @@ struct Lower {
             L.imgs_per_tile = 128 / L.rows_per_image;
             L.tile_rows = L.imgs_per_tile * L.rows_per_image;
             L.gap_imgs = L.imgs_per_tile; L.gap_area = L.rows_per_image; L.gap_rpi = L.rows_per_image;
+            if (L.rows_per_image > 128) {
+                // several tiles per image: 128 rows each, their column sums combined by the tile that finishes last
+                if (dw || shortcut || expand2 || M.k != 1 || M.stride != 1 || M.pad != 0 || src.c % 64)
+                    return fail(g, XENOS_E_UNSUPPORTED, "internal: global average over more than 128 pixels needs a 1x1 convolution on 64-channel blocks");
+                L.gap_parts = ceil_div(L.rows_per_image, 128);
+                L.imgs_per_tile = 1; L.tile_rows = 128;
+                L.gap_imgs = 1; L.gap_area = 128;
+            }
         }
         // Where a 64-channel K block of the activation operand is a box of the NHWC tensor (stride 1, channels a
         // multiple of 64, no second K segment), TMA fetches it and writes the operand layout itself: the rows of
@@ -858,7 +869,7 @@ struct Lower {
         const SplitRequest &rq = ch.split;
         int N16 = round_up(N, 16);
         if (L.map_mode == MAP_PATCH) L.m_tiles = ceil_div(g.max_batch, L.ni) * L.tiles_y * L.tiles_x;
-        else if (L.epi == EPI_GAP) L.m_tiles = ceil_div(g.max_batch, L.imgs_per_tile);
+        else if (L.epi == EPI_GAP) L.m_tiles = L.gap_parts > 1 ? g.max_batch * L.gap_parts : ceil_div(g.max_batch, L.imgs_per_tile);
         else L.m_tiles = ceil_div(g.max_batch * L.rows_per_image, 128);
         if (rq.user && (rq.h > 1 || rq.w > 1))
             return fail(g, XENOS_E_BAD_SPLIT, "split: tensor-core chains cut rows / columns into 128-row tiles themselves; only parts_outc can be set");
@@ -1306,6 +1317,10 @@ xenos_status_t plan_workspace(Graph &g) {
             L.split_cnt_off = off + g.cnt_bytes;
             g.cnt_bytes += align_up((size_t)L.m_tiles * L.n_tiles * 8, 16);      // [arrived, reduced] per tile
             g.split_bytes = std::max(g.split_bytes, (size_t)L.ksplit * g.max_batch * L.rows_per_image * L.npad * 4);
+        } else if (L.kind == LK_GEMM && L.gap_parts > 1) {
+            L.split_cnt_off = off + g.cnt_bytes;
+            g.cnt_bytes += align_up((size_t)g.max_batch * L.n_tiles * 8, 16);   // one counter per (image, channel tile)
+            g.split_bytes = std::max(g.split_bytes, (size_t)g.max_batch * L.gap_parts * L.npad * 4);
         }
     g.cnt_bytes = align_up(g.cnt_bytes, 256);
     off += g.cnt_bytes;
@@ -1426,7 +1441,7 @@ void emit_plan_json(Graph &g) {
             jint(s, "ni", L.ni); jint(s, "step_y", L.step_y); jint(s, "step_x", L.step_x); jint(s, "off_y", L.off_y); jint(s, "off_x", L.off_x);
             jint(s, "hstages", L.hstages); jint(s, "halo_h", L.halo_h); jint(s, "halo_w", L.halo_w); jint(s, "halo_cb", L.halo_cb);
             jint(s, "halo_bytes", L.halo_bytes);
-            jint(s, "ksplit", L.ksplit); jint(s, "kb_per", L.kb_per); jint(s, "a_tma", L.a_tma); jint(s, "fc_small", L.fc_small); jint(s, "dw_workers", L.dw_workers); jint(s, "n_acc", L.n_acc);
+            jint(s, "ksplit", L.ksplit); jint(s, "kb_per", L.kb_per); jint(s, "a_tma", L.a_tma); jint(s, "fc_small", L.fc_small); jint(s, "dw_workers", L.dw_workers); jint(s, "n_acc", L.n_acc); jint(s, "gap_parts", L.gap_parts);
         }
         if (L.kind == LK_GEMM2) {
             jint(s, "k2", L.k2); jint(s, "cmid", L.Cmid); jint(s, "n1pad", L.n1pad); jint(s, "kblocks", L.kblocks); jint(s, "kblocks2", L.kblocks2);

@@ -464,13 +464,13 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
             p.stem_tma = L.stem_tma; p.stem_align = L.stem_align;
             p.a_tma = L.a_tma; p.a_box_bytes = L.a_box_bytes; p.a_cpb = L.seg[0].C / 64;
             p.off_halo = L.off_halo; p.off_stg = L.off_stg; p.off_dww = L.off_dww; p.off_bias = L.off_bias; p.off_bar = L.off_bar;
-            p.n_acc = L.n_acc;
+            p.n_acc = L.n_acc; p.gap_parts = L.gap_parts;
             p.act = L.act; p.act2 = L.act2; p.epi = L.epi; p.out_ctot = L.out_ctot; p.out_coff = L.out_coff;
             p.out_f32 = L.out_dtype == XENOS_DTYPE_F32;
             p.idesc = make_idesc(L.tile_n);
             p.launch_id = (int)li;
             if (L.map_mode == MAP_PATCH) p.m_tiles = ((N + L.ni - 1) / L.ni) * L.tiles_y * L.tiles_x;
-            else if (L.epi == EPI_GAP) p.m_tiles = (N + L.imgs_per_tile - 1) / L.imgs_per_tile;
+            else if (L.epi == EPI_GAP) p.m_tiles = L.gap_parts > 1 ? N * L.gap_parts : (N + L.imgs_per_tile - 1) / L.imgs_per_tile;
             else p.m_tiles = (int)(((long long)N * L.rows_per_image + 127) / 128);
             // the halo tensor map of a linked depthwise stage points at the stage's input; when that
             // is a caller buffer its address is only known now
@@ -519,7 +519,7 @@ xenos_status_t runtime_run(Graph &g, int batch, const void *const *in, void *con
             cudaError_t le;
             if (L.dw_workers == 16) le = cudaLaunchKernelEx(&cfg, xk::dwpw_kernel<16>, rt->tmaps[li], *tmh, p);
             else if (L.dw_workers == 8) le = cudaLaunchKernelEx(&cfg, xk::dwpw_kernel<8>, rt->tmaps[li], *tmh, p);
-            else if (L.ksplit > 1) le = cudaLaunchKernelEx(&cfg, xk::gemm_chain_kernel<1>, rt->tmaps[li], *tmh, p);
+            else if (L.ksplit > 1 || L.gap_parts > 1) le = cudaLaunchKernelEx(&cfg, xk::gemm_chain_kernel<1>, rt->tmaps[li], *tmh, p);
             else le = cudaLaunchKernelEx(&cfg, xk::gemm_chain_kernel<0>, rt->tmaps[li], *tmh, p);
             if (le != cudaSuccess) return cuda_fail(g, "kernel launch", le);
             break;

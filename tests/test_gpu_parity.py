@@ -280,6 +280,23 @@ def test_bf16_conv_gap_linked():
     assert gg.g.launch_count() == 1
 
 
+@pytest.mark.parametrize("c,cout,hw,batch,run_batch", [(512, 1000, 13, 3, 3), (64, 40, 12, 5, 4), (128, 264, 23, 2, 2), (64, 16, 16, 33, 33)])
+def test_bf16_conv_gap_over_several_tiles(c, cout, hw, batch, run_batch):
+    """Images of more than 128 pixels: each 128-row tile leaves its column sums, the tile that arrives last at the image's
+    counter adds them in ascending order (2, 2, 5 and 2 tiles per image; a last tile of 41, 16, 17 and 128 rows; fewer images
+    than max_batch; more tiles than units); run twice: the counters must be back at zero."""
+    def build(g):
+        x = g.cbr("cls", "input", cout, 1, act="relu", bn=False, bias=True)
+        g.gap("gap", x)
+    spec = _one(build, c, hw)
+    y, _, gg = check_bf16(f"conv_gap_parts{(c, cout, hw)}", spec, run_batch, linked=True, in_mode="bf16_nhwc", max_batch=batch)
+    L = gg.g.plan()["launches"]
+    assert len(L) == 1 and L[0]["gap_parts"] == -(-hw * hw // 128)
+    x = xo.round_bf16(graphs.make_input(spec, run_batch))
+    for _ in range(2):
+        assert np.array_equal(gg.run(x), y)
+
+
 @pytest.mark.parametrize("hw,batch", [(4, 9), (2, 40), (1, 7)])
 def test_bf16_conv_gap_many_images_per_tile(hw, batch):
     """Small images: a 128-row tile holds several whole images and the average runs without partial sums."""
