@@ -344,6 +344,13 @@ static bool try_match(const LinkCtx &cx, int a, Allowed allowed, Chain &out, boo
             int th, tw, rh, rw;
             const Tensor &po = g.tensors[B.out];
             if (!pool_patch(B.k, B.stride, po.h, po.w, th, tw, rh, rw)) return false;
+            // An image convolution with its max pool is linked on request only: the pool's tiles overlap (27 % more
+            // convolution rows for a 3x3 stride-2 pool) and the pooling pass of the epilogue costs what the separate pool
+            // kernel costs.  Measured at batch 32, linked against the two kernels: 96 vs 77 us (7x7 stem, 64 channels),
+            // 73 vs 50 us (3x3 stem, 64 channels), 166 vs 125 us (3x3, 24 channels).  Images wider than 256 pixels keep
+            // the link: there the convolution alone loses its TMA-fetched patches (0.83 vs 4.4 ms at 512 x 512).
+            // At batch 1 the link wins (one launch less: 0.221 vs 0.231 ms for the whole 3x3-stem graph).
+            if (by_model && nchw_in && g.max_batch >= 8 && g.tensors[A.in[0]].w <= 256 && g.tensors[A.in[0]].h <= 256) return false;
             out.kind = CK_CONV_TAIL;
             out.nodes = {a, b};
             out.pattern = "ConvX -> ZPooling (CBR-MaxPooling)";

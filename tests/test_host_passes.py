@@ -558,3 +558,17 @@ def test_graph_image_rejects_what_is_not_an_intact_image():
     idx[off:off + 4] = (12345).to_bytes(4, "little")
     bad(resum(idx))
     assert xb.Graph.load(img)[0].plan_text() == g.plan_text()     # the untouched image still loads
+
+
+def test_image_convolution_and_max_pool_link_by_measured_cost():
+    """At batch 8 and above an image convolution and its max pool run as two kernels (measured faster), unless the image is
+    wider than 256 pixels or the link is requested; at small batch they are linked."""
+    spec = graphs.resnet18()
+    def first_chain(batch, **kw):
+        pl = compiled(spec, batch, **kw)[0].plan()
+        return [pl["nodes"][i]["kind"] for i in pl["chains"][0]["nodes"]]
+    assert first_chain(1) == ["conv", "maxpool"]
+    assert first_chain(32) == ["conv"]
+    assert first_chain(32, links=[["stem", "mp"]]) == ["conv", "maxpool"]
+    pl = compiled(graphs.resnet50_stress(), 8)[0].plan()
+    assert [pl["nodes"][i]["kind"] for i in pl["chains"][0]["nodes"]] == ["conv", "maxpool"]
