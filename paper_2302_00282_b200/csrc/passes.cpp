@@ -347,9 +347,11 @@ static bool try_match(const LinkCtx &cx, int a, Allowed allowed, Chain &out, boo
             // An image convolution with its max pool is linked on request only: the pool's tiles overlap (27 % more
             // convolution rows for a 3x3 stride-2 pool) and the pooling pass of the epilogue costs what the separate pool
             // kernel costs.  Measured at batch 32, linked against the two kernels: 96 vs 77 us (7x7 stem, 64 channels),
-            // 73 vs 50 us (3x3 stem, 64 channels), 166 vs 125 us (3x3, 24 channels).  Images wider than 256 pixels keep
-            // the link: there the convolution alone loses its TMA-fetched patches (0.83 vs 4.4 ms at 512 x 512).
+            // 73 vs 50 us (3x3 stem, 64 channels), 166 vs 125 us (3x3, 24 channels), 830 vs 788 us (7x7 stem at 512 x 512,
+            // batch 64).
             // At batch 1 the link wins (one launch less: 0.221 vs 0.231 ms for the whole 3x3-stem graph).
+            // Images wider than 256 pixels keep the link: the difference is small there and the link saves the
+            // convolution's output, the largest tensor of the graph (1.07 GB written and read at 512 x 512, batch 64).
             if (by_model && nchw_in && g.max_batch >= 8 && g.tensors[A.in[0]].w <= 256 && g.tensors[A.in[0]].h <= 256) return false;
             out.kind = CK_CONV_TAIL;
             out.nodes = {a, b};
@@ -795,6 +797,8 @@ struct Lower {
                 long best = -1;
                 for (int tw = 1; tw <= std::min(L.Q, 128); ++tw) {
                     int th = std::min(L.P, 128 / tw);
+                    // (tiles whose input patch the copy engine can fetch: at most 256 columns and rows)
+                    if (tw > 1 && ((tw - 1) * M.stride + (M.k > 4 ? 10 : M.k) + 8 > 256 || (th - 1) * M.stride + M.k > 256)) continue;
                     long tiles = (long)ceil_div(L.P, th) * ceil_div(L.Q, tw);
                     if (best < 0 || tiles < best || (tiles == best && tw > L.patch_rw)) { best = tiles; L.patch_rh = th; L.patch_rw = tw; }
                 }

@@ -562,7 +562,8 @@ def test_graph_image_rejects_what_is_not_an_intact_image():
 
 def test_image_convolution_and_max_pool_link_by_measured_cost():
     """At batch 8 and above an image convolution and its max pool run as two kernels (measured faster), unless the image is
-    wider than 256 pixels or the link is requested; at small batch they are linked."""
+    wider than 256 pixels or the link is requested; at small batch they are linked.  An unlinked image convolution's tiles
+    keep their input patch within the copy engine's 256 x 256 box, also for a 512 x 512 image."""
     spec = graphs.resnet18()
     def first_chain(batch, **kw):
         pl = compiled(spec, batch, **kw)[0].plan()
@@ -572,3 +573,6 @@ def test_image_convolution_and_max_pool_link_by_measured_cost():
     assert first_chain(32, links=[["stem", "mp"]]) == ["conv", "maxpool"]
     pl = compiled(graphs.resnet50_stress(), 8)[0].plan()
     assert [pl["nodes"][i]["kind"] for i in pl["chains"][0]["nodes"]] == ["conv", "maxpool"]
+    pl = compiled(graphs.resnet50_stress(), 8, linked=False)[0].plan()
+    stem = pl["launches"][0]
+    assert stem["a0"] == "stem" and (stem["patch_rw"] - 1) * 2 + 18 <= 256 and stem["hstages"] >= 2      # hstages: patches by TMA
