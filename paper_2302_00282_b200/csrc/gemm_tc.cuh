@@ -1072,7 +1072,11 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant
                     gr1[i] = gather_row(g.seg[1], r4);       // (unused without a second segment)
                 }
                 if (gj + 8 * tk.kb0) gather_advance(gs0, gj + 8 * tk.kb0, g.seg[0].C >> 3, g.seg[0].k);
-                if (g.seg[1].mode == GA_GATHER && gj) gather_advance(gs1, gj, g.seg[1].C >> 3, g.seg[1].k);
+                if (g.seg[1].mode == GA_GATHER) {
+                    // (a chunk of a split reduction may begin inside the second segment)
+                    const int adv = gj + 8 * max(0, tk.kb0 - g.seg[0].kblocks);
+                    if (adv) gather_advance(gs1, adv, g.seg[1].C >> 3, g.seg[1].k);
+                }
             }
             for (int kb = tk.kb0; kb < tk.kb1 && ok; ++kb) {
                 const int s = st.s;

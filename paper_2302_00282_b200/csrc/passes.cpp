@@ -334,7 +334,12 @@ static bool try_match(const LinkCtx &cx, int a, Allowed allowed, Chain &out, boo
             }
             out.nodes.push_back(b);
             int c = cx.sole(b);
-            if (c >= 0 && allowed(c) && g.nodes[c].kind == NK_GAP && cx.rows(b) <= 128) {
+            // (a global average is not attached to a long reduction that would run on a handful of units: the epilogue
+            // with the average cannot take part in a reduction split, and at batch 1 the 72 K blocks of ResNet-18's last
+            // convolution then run one after the other on 16 units, 38 us against 14 + 6 us as two kernels)
+            const long gap_tiles = (long)((g.max_batch * cx.rows(b) + 127) / 128) * ((A.cout + 31) / 32);
+            const bool serial_k = by_model && (long)A.k * A.k * A.cin >= 16 * 64 && gap_tiles * 2 <= g.hw.sm_count;
+            if (c >= 0 && allowed(c) && g.nodes[c].kind == NK_GAP && cx.rows(b) <= 128 && !serial_k) {
                 out.nodes.push_back(c);
                 out.pattern += " -> ZPooling (global average)";
             }
@@ -918,10 +923,13 @@ struct Lower {
                 (long)g.max_batch * src.c * 2 <= 160 * 1024 && !(src.input_slot >= 0 && src.io_dtype != XENOS_DTYPE_BF16))
                 L.fc_small = 1;
             const bool plain = !L.fc_small && s0.mode == AM_GATHER && (L.map_mode == MAP_FLAT || L.a_tma == 2);
-            const bool can = (plain || s0.mode == AM_DW) && s1.mode == AM_NONE && L.epi == EPI_STORE;
+            // (a linked shortcut convolution, the second K segment of a gathered convolution, is cut with it: the chunks
+            // are blocks of the concatenated K)
+            const bool can = ((plain || s0.mode == AM_DW) && s1.mode == AM_NONE && L.epi == EPI_STORE) ||
+                             (plain && L.map_mode == MAP_FLAT && !L.a_tma && s1.mode == AM_GATHER && L.epi == EPI_STORE);
             int want = 1;
             if (rq.user && rq.k > 1) {
-                if (!can) return fail(g, XENOS_E_UNSUPPORTED, "split: parts_k applies to a convolution, depthwise -> pointwise chain or fc that stores its tile (no image stem, second K segment or pooling epilogue)");
+                if (!can) return fail(g, XENOS_E_UNSUPPORTED, "split: parts_k applies to a convolution, depthwise -> pointwise chain or fc that stores its tile (no image stem or pooling epilogue)");
                 if (rq.k > L.kblocks) return fail(g, XENOS_E_BAD_SPLIT, "split: parts_k exceeds the number of 64-element K blocks");
                 want = rq.k;
             } else if (!rq.user && can && plain && L.kblocks >= 4 && (long)L.m_tiles * L.n_tiles * 2 <= g.hw.sm_count) {

@@ -367,6 +367,25 @@ def test_bf16_shortcut_block_with_reduction_split():
     assert gg.g.plan()["launches"][1]["ksplit"] == 3
 
 
+@pytest.mark.parametrize("parts_k", [2, 5, 10, 19])
+def test_bf16_shortcut_convolution_is_cut_with_its_block(parts_k):
+    """A linked shortcut convolution is the second K segment of the block's last convolution (18 + 1 K blocks here, the
+    second one 64 of 128 channels wide... both cut as one K): chunks that end inside the first segment, that begin inside
+    the second (19 chunks of one block), and a stride-2 shortcut; two runs agree bit for bit."""
+    def build(g):
+        y = g.cbr("c1", "input", 128, 3, 2, 1)
+        y = g.cbr("c2", y, 128, 3, 1, 1, act=None)
+        skip = g.cbr("proj", "input", 128, 1, 2, 0, act=None)
+        y = g.add("add", y, skip)
+        g.act("relu", y, "relu")
+    spec = _one(build, 64, 13)
+    y, _, gg = check_bf16(f"shortcut_proj_splitk{parts_k}", spec, 3, linked=True, in_mode="bf16_nhwc", splits=[("add", dict(parts_k=parts_k))])
+    L = gg.g.plan()["launches"][1]
+    assert L["a1"] == "gather" and L["kblocks"] == 19 and L["ksplit"] == parts_k
+    x = xo.round_bf16(graphs.make_input(spec, 3))
+    assert np.array_equal(gg.run(x), y)
+
+
 def test_bf16_fc_reduction_split_is_automatic_and_repeatable():
     """fc with few rows and a long reduction: the planner cuts K by itself (the other dimensions leave the units idle)."""
     def build(g):
