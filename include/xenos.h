@@ -166,9 +166,10 @@ XENOS_API xenos_status_t xenos_graph_link(xenos_graph_t *g, const xenos_id_t *op
  * kernel's (tap, channel) order and in blocks of 64 elements, is cut into parts_k chunks
  * of equal size (the last may be shorter); each chunk's partial sums are fp32 and are
  * added in ascending chunk order, so results do not vary from run to run, but they are not
- * bit-equal to the unsplit plan.  parts_k applies to tensor-core convolutions and fc
- * without a linked depthwise stage, image stem, linked shortcut convolution or pooling
- * epilogue (XENOS_E_UNSUPPORTED otherwise, from compile).
+ * bit-equal to the unsplit plan.  parts_k applies to tensor-core convolutions (a linked
+ * shortcut convolution is cut with its block: the chunks are blocks of the concatenated
+ * reduction), depthwise -> pointwise chains and fc that store their tile; not to an image
+ * stem or a pooling / global-average epilogue (XENOS_E_UNSUPPORTED, from compile).
  * XENOS_E_BAD_SPLIT (from this call or from compile) if a count exceeds the extent it
  * divides, leaves a chunk empty or breaks a kernel limit. */
 XENOS_API xenos_status_t xenos_graph_split(xenos_graph_t *g, xenos_id_t op, int32_t parts_outc,
